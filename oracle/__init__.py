@@ -1,0 +1,14 @@
+"""CPU oracle (fp64, plain loops) for the fused attention / fused linear patterns.
+
+Test infrastructure only: imported by ``tests/``, by the smoke check and by the
+benchmark's CPU-baseline leg.  The CUDA product path never imports this package.
+"""
+from .ref import (  # noqa: F401
+    attn,
+    attn_probs,
+    attn_decode,
+    linear_bias_gelu,
+    gelu_tanh,
+    num_threads,
+    build,
+)

@@ -1,0 +1,194 @@
+/*
+ * forge_ref.c -- CPU oracle for fused scaled-dot-product attention and the fused
+ * Linear + bias + tanh-GELU.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain, fp64 statement of what
+ * the fused patterns compute.  It is used by the tests, by the smoke check and by
+ * the benchmark's CPU-baseline leg; the product (the CUDA library) never links,
+ * loads or calls it, and shares no code, header, table or helper with it.
+ *
+ * What it follows:
+ *   - attention: the unfused chain  Q.K^T -> scale -> [mask] -> softmax -> .V
+ *     (Eq. 8) whose result the fused operator must preserve, i.e.
+ *     softmax(scale * Q K^T) V (Eq. 9) with the mask applied as exclusion of
+ *     keys before the softmax.  Grouped-query heads: query head h reads KV head
+ *     h / (Hq / Hkv).
+ *   - decode: the same definition with one query row per (batch, head) over the
+ *     first lens[b] rows of a KV cache.  The number of splits is not part of the
+ *     definition (the split/combine is an identity in exact arithmetic).
+ *   - linear: y = gelu_tanh(x W + b) for W stored [K, N] (Listing 6 / Eq. 11:
+ *     matmul, element-wise bias add, activation, one dispatch).
+ *
+ * There is no blocking, fusion, online rescaling or reordering here: scores for a
+ * row are all computed, the maximum is taken, exponentials are normalised, and
+ * the weighted sum over V is formed, in that order.  OpenMP, when enabled, only
+ * distributes independent (batch, head) pairs or output rows over threads.
+ *
+ * Layouts (row-major, last index fastest):
+ *   q, out : [B, Hq, Sq, D]     k, v : [B, Hkv, Skv, D]     lens : int32 [B]
+ *   probs  : [B, Hq, Sq, Skv]
+ *   x : [M, K]   w : [K, N]   b : [N]   y : [M, N]
+ *
+ * mask_kind: 0 none, 1 causal, 2 key padding (key j valid iff j < lens[b]),
+ *            3 causal and key padding.
+ * Causal alignment when Sq != Skv is bottom-right: query i sees keys
+ * j <= i + (Skv - Sq).  lens[b] is clamped to [0, Skv].  A row with no allowed
+ * key produces zeros (and an all-zero probability row).
+ *
+ * Every function returns 0 on success, 1 on an invalid argument.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+
+static int kv_limit(int mask_kind, const int32_t *lens, int b, int Skv)
+{
+    int n = Skv;
+    if (mask_kind & 2) {
+        n = lens[b];
+        if (n < 0) n = 0;
+        if (n > Skv) n = Skv;
+    }
+    return n;
+}
+
+/* 1 if key j is visible to query i under the mask. */
+static int allowed(int mask_kind, int i, int j, int Sq, int Skv, int kvlen)
+{
+    if (j >= kvlen) return 0;
+    if ((mask_kind & 1) && j > i + (Skv - Sq)) return 0;
+    return 1;
+}
+
+static int check_attn_args(const void *q, const void *k, const void *v, const void *out,
+                           int B, int Hq, int Hkv, int Sq, int Skv, int D,
+                           int mask_kind, const int32_t *lens)
+{
+    if (!q || !k || !v || !out) return 1;
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Skv <= 0 || D <= 0) return 1;
+    if (Hq % Hkv != 0) return 1;
+    if (mask_kind < 0 || mask_kind > 3) return 1;
+    if ((mask_kind & 2) && !lens) return 1;
+    return 0;
+}
+
+/*
+ * One attention row (Eq. 9 restricted to the allowed keys).  p has room for Skv
+ * doubles and receives the probabilities (exact 0.0 where masked).
+ */
+static void attn_row(const double *qrow, const double *kmat, const double *vmat, double *orow,
+                     double *p, int i, int Sq, int Skv, int D, int mask_kind, int kvlen, double scale)
+{
+    double m = -INFINITY;
+    int any = 0;
+    for (int j = 0; j < Skv; ++j) {
+        if (!allowed(mask_kind, i, j, Sq, Skv, kvlen)) { p[j] = 0.0; continue; }
+        double s = 0.0;
+        for (int d = 0; d < D; ++d) s += qrow[d] * kmat[(size_t)j * D + d];
+        s *= scale;
+        p[j] = s;
+        if (!any || s > m) m = s;
+        any = 1;
+    }
+    for (int d = 0; d < D; ++d) orow[d] = 0.0;
+    if (!any) return;
+
+    double denom = 0.0;
+    for (int j = 0; j < Skv; ++j) {
+        if (!allowed(mask_kind, i, j, Sq, Skv, kvlen)) continue;
+        p[j] = exp(p[j] - m);
+        denom += p[j];
+    }
+    for (int j = 0; j < Skv; ++j) {
+        if (!allowed(mask_kind, i, j, Sq, Skv, kvlen)) continue;
+        p[j] /= denom;
+        for (int d = 0; d < D; ++d) orow[d] += p[j] * vmat[(size_t)j * D + d];
+    }
+}
+
+static int attn_impl(const double *q, const double *k, const double *v, double *out, double *probs,
+                     int B, int Hq, int Hkv, int Sq, int Skv, int D,
+                     int mask_kind, const int32_t *lens, double scale)
+{
+    if (check_attn_args(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens)) return 1;
+    const int G = Hq / Hkv;
+    int failed = 0;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int b = 0; b < B; ++b) {
+        for (int h = 0; h < Hq; ++h) {
+            const int kvh = h / G;
+            const int kvlen = kv_limit(mask_kind, lens, b, Skv);
+            const double *kmat = k + ((size_t)b * Hkv + kvh) * (size_t)Skv * D;
+            const double *vmat = v + ((size_t)b * Hkv + kvh) * (size_t)Skv * D;
+            double *scratch = probs ? NULL : (double *)malloc(sizeof(double) * (size_t)Skv);
+            if (!probs && !scratch) { failed = 1; continue; }
+            for (int i = 0; i < Sq; ++i) {
+                size_t row = ((size_t)b * Hq + h) * (size_t)Sq + i;
+                double *p = probs ? probs + row * (size_t)Skv : scratch;
+                attn_row(q + row * D, kmat, vmat, out + row * D, p, i, Sq, Skv, D, mask_kind, kvlen, scale);
+            }
+            free(scratch);
+        }
+    }
+    return failed;
+}
+
+/* Fused attention result (Eq. 8 / Eq. 9). */
+int forge_ref_attn(const double *q, const double *k, const double *v, double *out,
+                   int B, int Hq, int Hkv, int Sq, int Skv, int D,
+                   int mask_kind, const int32_t *lens, double scale)
+{
+    return attn_impl(q, k, v, out, NULL, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale);
+}
+
+/* Same, and also returns the probability matrix softmax(mask(scale Q K^T)) that the
+ * unfused chain of Eq. 8 would have materialised.  For small shapes. */
+int forge_ref_attn_probs(const double *q, const double *k, const double *v, double *out, double *probs,
+                         int B, int Hq, int Hkv, int Sq, int Skv, int D,
+                         int mask_kind, const int32_t *lens, double scale)
+{
+    if (!probs) return 1;
+    return attn_impl(q, k, v, out, probs, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale);
+}
+
+/*
+ * Decode step: q, out [B, Hq, D]; caches [B, Hkv, Smax, D]; sequence b attends its
+ * first lens[b] cached rows.  This is Eq. 9 with a single query row per head.
+ */
+int forge_ref_attn_decode(const double *q, const double *k_cache, const double *v_cache, double *out,
+                          int B, int Hq, int Hkv, int Smax, int D, const int32_t *lens, double scale)
+{
+    if (!lens) return 1;
+    return attn_impl(q, k_cache, v_cache, out, NULL, B, Hq, Hkv, 1, Smax, D, 2, lens, scale);
+}
+
+/* tanh form of GELU: 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3))). */
+double forge_ref_gelu_tanh(double z)
+{
+    const double c = sqrt(2.0 / M_PI);
+    return 0.5 * z * (1.0 + tanh(c * (z + 0.044715 * z * z * z)));
+}
+
+/* y[m, n] = gelu_tanh(b[n] + sum_k x[m, k] w[k, n])  (Listing 6 / Eq. 11). */
+int forge_ref_linear_bias_gelu(const double *x, const double *w, const double *b, double *y,
+                               int M, int N, int K)
+{
+    if (!x || !w || !b || !y || M <= 0 || N <= 0 || K <= 0) return 1;
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        for (int n = 0; n < N; ++n) {
+            double acc = 0.0;
+            for (int kk = 0; kk < K; ++kk) acc += x[(size_t)m * K + kk] * w[(size_t)kk * N + n];
+            y[(size_t)m * N + n] = forge_ref_gelu_tanh(acc + b[n]);
+        }
+    }
+    return 0;
+}
+
+/* Number of OpenMP threads the loops above will use (1 when built without OpenMP). */
+#ifdef _OPENMP
+#include <omp.h>
+int forge_ref_num_threads(void) { return omp_get_max_threads(); }
+#else
+int forge_ref_num_threads(void) { return 1; }
+#endif

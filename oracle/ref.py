@@ -1,0 +1,122 @@
+"""ctypes binding for ``forge_ref.c`` (the CPU oracle).  Test infrastructure only.
+
+Arrays are numpy fp64, C-contiguous; ``lens`` is int32.  Shapes follow the C file:
+q/out [B,Hq,Sq,D], k/v [B,Hkv,Skv,D]; decode q/out [B,Hq,D], caches [B,Hkv,Smax,D];
+linear x [M,K], w [K,N], b [N].
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "forge_ref.c")
+_LIB = os.path.join(_HERE, "libforge_ref.so")
+_lib = None
+
+_dp = ctypes.POINTER(ctypes.c_double)
+_ip = ctypes.POINTER(ctypes.c_int32)
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (plain -O2, no fast-math) if it is missing or stale."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.run(["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-o", tmp, _SRC, "-lm"], check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        i = ctypes.c_int
+        lib.forge_ref_attn.argtypes = [_dp, _dp, _dp, _dp, i, i, i, i, i, i, i, _ip, ctypes.c_double]
+        lib.forge_ref_attn_probs.argtypes = [_dp, _dp, _dp, _dp, _dp, i, i, i, i, i, i, i, _ip, ctypes.c_double]
+        lib.forge_ref_attn_decode.argtypes = [_dp, _dp, _dp, _dp, i, i, i, i, i, _ip, ctypes.c_double]
+        lib.forge_ref_linear_bias_gelu.argtypes = [_dp, _dp, _dp, _dp, i, i, i]
+        lib.forge_ref_gelu_tanh.argtypes = [ctypes.c_double]
+        lib.forge_ref_gelu_tanh.restype = ctypes.c_double
+        lib.forge_ref_num_threads.restype = i
+        _lib = lib
+    return _lib
+
+
+def _f64(a):
+    return np.ascontiguousarray(a, dtype=np.float64)
+
+
+def _ptr(a):
+    return a.ctypes.data_as(_dp)
+
+
+def _lens_ptr(lens):
+    if lens is None:
+        return None, None
+    l32 = np.ascontiguousarray(lens, dtype=np.int32)
+    return l32, l32.ctypes.data_as(_ip)
+
+
+def _check(status, what):
+    if status != 0:
+        raise ValueError(f"{what}: invalid argument (status {status})")
+
+
+def attn(q, k, v, mask_kind=0, lens=None, scale=1.0):
+    q, k, v = _f64(q), _f64(k), _f64(v)
+    B, Hq, Sq, D = q.shape
+    _, Hkv, Skv, _ = k.shape
+    assert k.shape == v.shape == (B, Hkv, Skv, D)
+    out = np.empty_like(q)
+    keep, lp = _lens_ptr(lens)
+    _check(_load().forge_ref_attn(_ptr(q), _ptr(k), _ptr(v), _ptr(out), B, Hq, Hkv, Sq, Skv, D,
+                                  int(mask_kind), lp, float(scale)), "forge_ref_attn")
+    return out
+
+
+def attn_probs(q, k, v, mask_kind=0, lens=None, scale=1.0):
+    q, k, v = _f64(q), _f64(k), _f64(v)
+    B, Hq, Sq, D = q.shape
+    _, Hkv, Skv, _ = k.shape
+    assert k.shape == v.shape == (B, Hkv, Skv, D)
+    out = np.empty_like(q)
+    probs = np.empty((B, Hq, Sq, Skv), dtype=np.float64)
+    keep, lp = _lens_ptr(lens)
+    _check(_load().forge_ref_attn_probs(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(probs), B, Hq, Hkv,
+                                        Sq, Skv, D, int(mask_kind), lp, float(scale)), "forge_ref_attn_probs")
+    return out, probs
+
+
+def attn_decode(q, k_cache, v_cache, lens, scale=1.0):
+    q, k_cache, v_cache = _f64(q), _f64(k_cache), _f64(v_cache)
+    B, Hq, D = q.shape
+    _, Hkv, Smax, _ = k_cache.shape
+    assert k_cache.shape == v_cache.shape == (B, Hkv, Smax, D)
+    out = np.empty_like(q)
+    keep, lp = _lens_ptr(lens)
+    _check(_load().forge_ref_attn_decode(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(out), B, Hq, Hkv,
+                                         Smax, D, lp, float(scale)), "forge_ref_attn_decode")
+    return out
+
+
+def linear_bias_gelu(x, w, b):
+    x, w, b = _f64(x), _f64(w), _f64(b)
+    M, K = x.shape
+    K2, N = w.shape
+    assert K2 == K and b.shape == (N,)
+    y = np.empty((M, N), dtype=np.float64)
+    _check(_load().forge_ref_linear_bias_gelu(_ptr(x), _ptr(w), _ptr(b), _ptr(y), M, N, K),
+           "forge_ref_linear_bias_gelu")
+    return y
+
+
+def gelu_tanh(z: float) -> float:
+    return float(_load().forge_ref_gelu_tanh(float(z)))
+
+
+def num_threads() -> int:
+    return int(_load().forge_ref_num_threads())

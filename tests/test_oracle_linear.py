@@ -1,0 +1,87 @@
+"""Pins for the Linear + bias + tanh-GELU oracle (CPU only)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+
+RNG = np.random.default_rng(7)
+
+
+def test_gelu_closed_forms_and_invariants():
+    assert oracle.gelu_tanh(0.0) == 0.0
+    for z in [0.1, 0.5, 1.0, 2.0, 3.3, 7.0]:
+        # odd tanh => gelu(z) - gelu(-z) = z
+        assert abs(oracle.gelu_tanh(z) - oracle.gelu_tanh(-z) - z) < 1e-15 * max(1.0, z)
+    assert abs(oracle.gelu_tanh(30.0) - 30.0) < 1e-12       # saturates to identity
+    assert abs(oracle.gelu_tanh(-30.0)) < 1e-12             # and to zero
+    # the minimum of tanh-GELU is about -0.17 near z = -0.75; it is negative only for z < 0
+    assert -0.171 < oracle.gelu_tanh(-0.75) < -0.169
+
+
+def test_gelu_is_the_tanh_form_not_erf():
+    """tanh-GELU(1) = 0.841192; the erf form gives 0.841345, 1.5e-4 away."""
+    erf_form = 0.5 * (1.0 + math.erf(1.0 / math.sqrt(2.0)))
+    assert abs(oracle.gelu_tanh(1.0) - 0.841192) < 5e-7
+    assert abs(oracle.gelu_tanh(1.0) - erf_form) > 1e-4
+
+
+def test_gelu_against_torch_library():
+    z = np.concatenate([np.linspace(-8, 8, 2001), RNG.standard_normal(1000) * 3])
+    ref = torch.nn.functional.gelu(torch.from_numpy(z), approximate="tanh").numpy()
+    got = np.array([oracle.gelu_tanh(t) for t in z])
+    np.testing.assert_allclose(got, ref, rtol=0, atol=2e-15)
+
+
+def _gelu_np(z):
+    return torch.nn.functional.gelu(torch.from_numpy(np.asarray(z, dtype=np.float64)), approximate="tanh").numpy()
+
+
+def test_linear_k1_outer_product():
+    x = RNG.standard_normal((5, 1)); w = RNG.standard_normal((1, 7)); b = RNG.standard_normal(7)
+    np.testing.assert_allclose(oracle.linear_bias_gelu(x, w, b), _gelu_np(x * w + b), rtol=0, atol=1e-15)
+
+
+def test_linear_identity_weight():
+    n = 6
+    x = RNG.standard_normal((n, n)); b = RNG.standard_normal(n)
+    np.testing.assert_allclose(oracle.linear_bias_gelu(x, np.eye(n), b), _gelu_np(x + b), rtol=0, atol=1e-15)
+
+
+def test_linear_all_ones():
+    M, N, K = 3, 4, 9
+    b = np.array([0.0, -9.0, 0.5, -8.0])
+    y = oracle.linear_bias_gelu(np.ones((M, K)), np.ones((K, N)), b)
+    np.testing.assert_allclose(y, np.broadcast_to(_gelu_np(K + b), (M, N)), rtol=0, atol=1e-14)
+    assert (y[:, 1] == 0.0).all()  # K + b = 0 exactly
+
+
+def test_linear_layout_is_x_times_w_kn():
+    """Non-square, asymmetric operands: a transposed or [N,K]-indexed W would fail."""
+    M, N, K = 4, 3, 5
+    x = RNG.standard_normal((M, K)); w = RNG.standard_normal((K, N)); b = RNG.standard_normal(N)
+    y = oracle.linear_bias_gelu(x, w, b)
+    np.testing.assert_allclose(y, _gelu_np(x @ w + b), rtol=0, atol=1e-14)
+    # other loop order, accumulated column by column
+    z = np.zeros((M, N))
+    for n in range(N):
+        for k in range(K):
+            for m in range(M):
+                z[m, n] += x[m, k] * w[k, n]
+    np.testing.assert_allclose(y, _gelu_np(z + b[None, :]), rtol=0, atol=1e-14)
+
+
+def test_linear_against_torch_library():
+    M, N, K = 33, 17, 29
+    x = RNG.standard_normal((M, K)); w = RNG.standard_normal((K, N)) * 0.2; b = RNG.standard_normal(N)
+    ref = torch.nn.functional.gelu(
+        torch.nn.functional.linear(torch.from_numpy(x), torch.from_numpy(w).t(), torch.from_numpy(b)),
+        approximate="tanh").numpy()
+    np.testing.assert_allclose(oracle.linear_bias_gelu(x, w, b), ref, rtol=0, atol=1e-13)
+
+
+def test_linear_invalid_arguments():
+    with pytest.raises((ValueError, AssertionError)):
+        oracle.linear_bias_gelu(np.zeros((2, 3)), np.zeros((4, 2)), np.zeros(2))

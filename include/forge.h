@@ -1,0 +1,160 @@
+/*
+ * forge.h -- C ABI of the B200 (sm_100a) library for the fused patterns that the
+ * attention-fusion and operator-fusion passes of the FORGE-UGC compiler produce:
+ *
+ *   - fused scaled-dot-product attention: the chain  Q.K^T -> scale -> [mask] ->
+ *     softmax -> .V  collapsed into one operator (Section 4.3 "Pass 4: Attention
+ *     Fusion", Eq. 8 and Eq. 9), with grouped-query heads and a split-KV decode
+ *     variant;
+ *   - fused Linear + bias + GELU: matmul, element-wise bias add and activation in
+ *     one dispatch, the linear output never materialised (Section 4.3 "Pass 5:
+ *     Operator Fusion", Listing 6 and Eq. 11).
+ *
+ * Conventions shared by every entry point
+ *   - Unless a parameter says HOST, pointers are DEVICE pointers owned by the
+ *     caller.  The library never frees or keeps them and allocates no device
+ *     memory.  Pointers must be 16-byte aligned.
+ *   - Tensors are dense, row-major, last index fastest:
+ *       q, out : [B, Hq, Sq, D]        k, v : [B, Hkv, Skv, D]        lens : int32 [B]
+ *   - Query head h reads KV head h / (Hq / Hkv)  (consecutive grouping).
+ *   - All work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is the
+ *     legacy default stream).  No entry point synchronises unless it says so.
+ *   - Arguments are validated on the host before anything is launched.  The return
+ *     value is a forge_status; nothing throws.
+ *   - mask_kind: FORGE_MASK_NONE, FORGE_MASK_CAUSAL, FORGE_MASK_PADDING (key j of
+ *     sequence b is valid iff j < lens[b]) or FORGE_MASK_CAUSAL_PADDING.  A masked
+ *     key gets probability exactly 0.  Causal alignment for Sq != Skv is
+ *     bottom-right: query i sees keys j <= i + (Skv - Sq).  lens lives on the
+ *     device, so it cannot be checked on the host: kernels clamp lens[b] to
+ *     [0, Skv]; a query row with no visible key yields zeros.
+ *   - Dropout, which the matched chain may contain, is the identity at inference
+ *     and is not implemented.
+ */
+#ifndef FORGE_H_
+#define FORGE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum forge_status {
+    FORGE_OK = 0,
+    FORGE_ERR_INVALID_ARG = 1, /* NULL pointer, non-positive size, Hq % Hkv != 0, misaligned pointer, lens missing */
+    FORGE_ERR_UNSUPPORTED = 2, /* valid request with no kernel: D not in {64,128}, row stride not a multiple of 16 bytes, ... */
+    FORGE_ERR_WORKSPACE = 3,   /* workspace too small */
+    FORGE_ERR_CUDA = 4,        /* a CUDA runtime/driver call failed; see forge_last_cuda_error() */
+    FORGE_ERR_TIMEOUT = 5      /* a bounded wait inside a kernel expired; reported by forge_check_status() */
+} forge_status;
+
+enum {
+    FORGE_MASK_NONE = 0,
+    FORGE_MASK_CAUSAL = 1,
+    FORGE_MASK_PADDING = 2,
+    FORGE_MASK_CAUSAL_PADDING = 3
+};
+
+/*
+ * Fused attention, bf16 in / fp32 accumulate / bf16 out:
+ *     out[b,h,i,:] = sum_j softmax_j(scale * q[b,h,i,:].k[b,h/G,j,:] over visible j) * v[b,h/G,j,:]
+ * (Eq. 9 with the optional scale and mask nodes of Eq. 8 folded in; scores and
+ * probabilities never reach global memory).  D must be 64 or 128.  `lens` may be
+ * NULL unless mask_kind has the padding bit.  Tensor-core path (tcgen05, TMEM
+ * accumulators, TMA-staged K/V).
+ */
+int forge_attn_fused(const void* q, const void* k, const void* v, void* out,
+                     int B, int Hq, int Hkv, int Sq, int Skv, int D,
+                     int mask_kind, const int32_t* lens, float scale, void* stream);
+
+/*
+ * Same operator with fp32 tensors in and out (fp32 FMA arithmetic, no reduced
+ * precision inside).  D must be 64 or 128.
+ */
+int forge_attn_fused_f32(const void* q, const void* k, const void* v, void* out,
+                         int B, int Hq, int Hkv, int Sq, int Skv, int D,
+                         int mask_kind, const int32_t* lens, float scale, void* stream);
+
+/*
+ * Decode step of the same operator (Eq. 9 with one query row per head) over a KV
+ * cache, split along the cached sequence:
+ *     q, out : [B, Hq, D] bf16       k_cache, v_cache : [B, Hkv, Smax, D] bf16
+ * Sequence b attends rows 0 .. lens[b]-1 of its cache (lens[b] clamped to
+ * [0, Smax]; 0 gives zeros).  Split s of sequence b covers rows
+ * [s*c, min((s+1)*c, lens[b])) with c = ceil(lens[b] / num_splits); each split
+ * produces a partial (running max, running sum, unnormalised output) in
+ * `workspace` (fp32), and a combine step merges them.  Empty splits are skipped.
+ * The result does not depend on num_splits beyond rounding.
+ * workspace: at least forge_attn_decode_workspace_bytes(...) bytes, 16-byte
+ * aligned, contents need no initialisation and are overwritten.  Two calls that
+ * may overlap on the GPU must not share a workspace.
+ * 1 <= num_splits <= 64; D must be 64 or 128; Hq / Hkv must be 1, 2, 4 or 8.
+ */
+int forge_attn_decode_splitkv(const void* q, const void* k_cache, const void* v_cache, void* out,
+                              int B, int Hq, int Hkv, int Smax, int D,
+                              const int32_t* lens, int num_splits, float scale,
+                              void* workspace, size_t workspace_bytes, void* stream);
+
+/* Bytes of workspace forge_attn_decode_splitkv needs; 0 for invalid arguments. */
+size_t forge_attn_decode_workspace_bytes(int B, int Hq, int D, int num_splits);
+
+/*
+ * Fused Linear + bias + tanh-GELU (Listing 6 / Eq. 11):
+ *     y[m,n] = gelu_tanh(b[n] + sum_k x[m,k] * w[k,n]),
+ *     gelu_tanh(z) = 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3)))
+ * x [M,K], w [K,N] (GPT-2 c_fc layout), b [N], y [M,N]; bf16 in and out, fp32
+ * accumulation, bias and activation applied to the fp32 accumulator before the
+ * single rounding to bf16.  K and N must be multiples of 8 (16-byte rows).
+ * Tensor-core path (tcgen05, TMEM accumulators, TMA-staged operands).
+ */
+int forge_linear_bias_gelu(const void* x, const void* w, const void* b, void* y,
+                           int M, int N, int K, void* stream);
+
+/*
+ * Host-buffer variants: the same operators for callers whose tensors live in
+ * HOST memory (pinned memory makes the copies asynchronous).  Inputs are copied
+ * to `dev_scratch`, the operator runs there, and the result is copied back to the
+ * host pointer, all on `stream`; the call returns without synchronising.
+ * dev_scratch is DEVICE memory of at least forge_*_host_scratch_bytes(...) bytes,
+ * 256-byte aligned, owned by the caller.  `lens` is a HOST pointer here.
+ */
+size_t forge_attn_host_scratch_bytes(int B, int Hq, int Hkv, int Sq, int Skv, int D, int elem_bytes);
+int forge_attn_fused_host(const void* q, const void* k, const void* v, void* out,
+                          int B, int Hq, int Hkv, int Sq, int Skv, int D,
+                          int mask_kind, const int32_t* lens, float scale,
+                          void* dev_scratch, size_t dev_scratch_bytes, void* stream);
+int forge_attn_fused_f32_host(const void* q, const void* k, const void* v, void* out,
+                              int B, int Hq, int Hkv, int Sq, int Skv, int D,
+                              int mask_kind, const int32_t* lens, float scale,
+                              void* dev_scratch, size_t dev_scratch_bytes, void* stream);
+size_t forge_attn_decode_host_scratch_bytes(int B, int Hq, int Hkv, int Smax, int D, int num_splits);
+int forge_attn_decode_splitkv_host(const void* q, const void* k_cache, const void* v_cache, void* out,
+                                   int B, int Hq, int Hkv, int Smax, int D,
+                                   const int32_t* lens, int num_splits, float scale,
+                                   void* dev_scratch, size_t dev_scratch_bytes, void* stream);
+size_t forge_linear_host_scratch_bytes(int M, int N, int K);
+int forge_linear_bias_gelu_host(const void* x, const void* w, const void* b, void* y,
+                                int M, int N, int K,
+                                void* dev_scratch, size_t dev_scratch_bytes, void* stream);
+
+/*
+ * Synchronises `stream`, then reports whether any kernel launched by this library
+ * since the last call gave up on a bounded wait (FORGE_ERR_TIMEOUT) and clears the
+ * flag.  Returns FORGE_OK otherwise, FORGE_ERR_CUDA if the stream itself failed.
+ */
+int forge_check_status(void* stream);
+
+/* Human-readable name of a forge_status value (static storage). */
+const char* forge_status_string(int status);
+
+/* The cudaError_t (as int) behind the most recent FORGE_ERR_CUDA on this thread. */
+int forge_last_cuda_error(void);
+
+/* Number of kernels this library has launched in this process (for accounting). */
+unsigned long long forge_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FORGE_H_ */

@@ -1,0 +1,217 @@
+"""Python binding of the C ABI in ``include/forge.h`` (argument marshalling only).
+
+Every function takes torch tensors (used purely as owners of device or pinned host
+memory), checks shapes and dtypes, and passes raw pointers, sizes and the current
+CUDA stream to ``libforge.so``.  All arithmetic happens inside the library's kernels.
+There is no fallback: if the library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libforge.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
+MASK_NONE, MASK_CAUSAL, MASK_PADDING, MASK_CAUSAL_PADDING = range(4)
+
+# name -> (restype, argtypes); mirrors include/forge.h
+_vp, _i, _f, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+_ATTN = [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _i, _vp, _f]
+_DEC = [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _i, _f]
+SIGNATURES = {
+    "forge_attn_fused": (_i, _ATTN + [_vp]),
+    "forge_attn_fused_f32": (_i, _ATTN + [_vp]),
+    "forge_attn_decode_splitkv": (_i, _DEC + [_vp, _sz, _vp]),
+    "forge_attn_decode_workspace_bytes": (_sz, [_i, _i, _i, _i]),
+    "forge_linear_bias_gelu": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
+    "forge_attn_host_scratch_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _i]),
+    "forge_attn_fused_host": (_i, _ATTN + [_vp, _sz, _vp]),
+    "forge_attn_fused_f32_host": (_i, _ATTN + [_vp, _sz, _vp]),
+    "forge_attn_decode_host_scratch_bytes": (_sz, [_i, _i, _i, _i, _i, _i]),
+    "forge_attn_decode_splitkv_host": (_i, _DEC + [_vp, _sz, _vp]),
+    "forge_linear_host_scratch_bytes": (_sz, [_i, _i, _i]),
+    "forge_linear_bias_gelu_host": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
+    "forge_check_status": (_i, [_vp]),
+    "forge_status_string": (ctypes.c_char_p, [_i]),
+    "forge_last_cuda_error": (_i, []),
+    "forge_launch_count": (ctypes.c_ulonglong, []),
+}
+
+_lib = None
+
+
+class ForgeError(RuntimeError):
+    def __init__(self, fn: str, status: int):
+        self.status = status
+        lib = load()
+        name = lib.forge_status_string(status).decode()
+        extra = f" (cudaError {lib.forge_last_cuda_error()})" if status == ERR_CUDA else ""
+        super().__init__(f"{fn} failed: {name}{extra}")
+
+
+def load() -> ctypes.CDLL:
+    """Loads ``libforge.so`` (built by ``paper_2604_16498_b200.build``).  Raises if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2604_16498_b200.build` "
+                               "(there is no fallback implementation)")
+        lib = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = lib
+    return _lib
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> int:
+    if not (t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise ValueError(f"{name}: expected a contiguous CUDA tensor of {dtype}")
+    return t.data_ptr()
+
+
+def _host(t: torch.Tensor, dtype, name: str) -> int:
+    if t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise ValueError(f"{name}: expected a contiguous host tensor of {dtype}")
+    return t.data_ptr()
+
+
+def _check(fn: str, status: int) -> None:
+    if status != OK:
+        raise ForgeError(fn, status)
+
+
+def _attn_dims(q, k, v):
+    B, Hq, Sq, D = q.shape
+    Bk, Hkv, Skv, Dk = k.shape
+    if (Bk, Dk) != (B, D) or tuple(v.shape) != tuple(k.shape):
+        raise ValueError("q [B,Hq,Sq,D], k/v [B,Hkv,Skv,D] expected")
+    return B, Hq, Hkv, Sq, Skv, D
+
+
+def attn_fused(q, k, v, mask_kind=MASK_NONE, lens=None, scale=None, out=None):
+    """forge_attn_fused: bf16 tensors q [B,Hq,Sq,D], k/v [B,Hkv,Skv,D] on the GPU."""
+    B, Hq, Hkv, Sq, Skv, D = _attn_dims(q, k, v)
+    out = torch.empty_like(q) if out is None else out
+    scale = D ** -0.5 if scale is None else scale
+    lp = None if lens is None else _dev(lens, torch.int32, "lens")
+    _check("forge_attn_fused", load().forge_attn_fused(
+        _dev(q, torch.bfloat16, "q"), _dev(k, torch.bfloat16, "k"), _dev(v, torch.bfloat16, "v"),
+        _dev(out, torch.bfloat16, "out"), B, Hq, Hkv, Sq, Skv, D, int(mask_kind), lp, float(scale), _stream()))
+    return out
+
+
+def attn_fused_f32(q, k, v, mask_kind=MASK_NONE, lens=None, scale=None, out=None):
+    """forge_attn_fused_f32: the same operator on fp32 tensors."""
+    B, Hq, Hkv, Sq, Skv, D = _attn_dims(q, k, v)
+    out = torch.empty_like(q) if out is None else out
+    scale = D ** -0.5 if scale is None else scale
+    lp = None if lens is None else _dev(lens, torch.int32, "lens")
+    _check("forge_attn_fused_f32", load().forge_attn_fused_f32(
+        _dev(q, torch.float32, "q"), _dev(k, torch.float32, "k"), _dev(v, torch.float32, "v"),
+        _dev(out, torch.float32, "out"), B, Hq, Hkv, Sq, Skv, D, int(mask_kind), lp, float(scale), _stream()))
+    return out
+
+
+def attn_decode_workspace_bytes(B, Hq, D, num_splits) -> int:
+    return int(load().forge_attn_decode_workspace_bytes(B, Hq, D, num_splits))
+
+
+def attn_decode_splitkv(q, k_cache, v_cache, lens, num_splits, scale=None, out=None, workspace=None):
+    """forge_attn_decode_splitkv: q [B,Hq,D], caches [B,Hkv,Smax,D] (bf16), lens int32 [B]."""
+    B, Hq, D = q.shape
+    Bk, Hkv, Smax, Dk = k_cache.shape
+    if (Bk, Dk) != (B, D) or tuple(v_cache.shape) != tuple(k_cache.shape):
+        raise ValueError("q [B,Hq,D], caches [B,Hkv,Smax,D] expected")
+    out = torch.empty_like(q) if out is None else out
+    scale = D ** -0.5 if scale is None else scale
+    need = attn_decode_workspace_bytes(B, Hq, D, num_splits)
+    if workspace is None:
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=q.device)
+    _check("forge_attn_decode_splitkv", load().forge_attn_decode_splitkv(
+        _dev(q, torch.bfloat16, "q"), _dev(k_cache, torch.bfloat16, "k_cache"),
+        _dev(v_cache, torch.bfloat16, "v_cache"), _dev(out, torch.bfloat16, "out"),
+        B, Hq, Hkv, Smax, D, _dev(lens, torch.int32, "lens"), int(num_splits), float(scale),
+        _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream()))
+    return out
+
+
+def linear_bias_gelu(x, w, b, out=None):
+    """forge_linear_bias_gelu: x [M,K], w [K,N], b [N] (bf16) -> gelu_tanh(x @ w + b) [M,N]."""
+    M, K = x.shape
+    K2, N = w.shape
+    if K2 != K or tuple(b.shape) != (N,):
+        raise ValueError("x [M,K], w [K,N], b [N] expected")
+    out = torch.empty((M, N), dtype=torch.bfloat16, device=x.device) if out is None else out
+    _check("forge_linear_bias_gelu", load().forge_linear_bias_gelu(
+        _dev(x, torch.bfloat16, "x"), _dev(w, torch.bfloat16, "w"), _dev(b, torch.bfloat16, "b"),
+        _dev(out, torch.bfloat16, "out"), M, N, K, _stream()))
+    return out
+
+
+# ---- host-buffer variants: tensors in (pinned) host memory, device scratch from the caller ----
+def attn_host_scratch_bytes(B, Hq, Hkv, Sq, Skv, D, elem_bytes) -> int:
+    return int(load().forge_attn_host_scratch_bytes(B, Hq, Hkv, Sq, Skv, D, elem_bytes))
+
+
+def attn_fused_host(q, k, v, out, scratch, mask_kind=MASK_NONE, lens=None, scale=None):
+    """forge_attn_fused_host / forge_attn_fused_f32_host, chosen by q.dtype.  Asynchronous."""
+    B, Hq, Hkv, Sq, Skv, D = _attn_dims(q, k, v)
+    f32 = q.dtype == torch.float32
+    dt = torch.float32 if f32 else torch.bfloat16
+    scale = D ** -0.5 if scale is None else scale
+    lp = None if lens is None else _host(lens, torch.int32, "lens")
+    fn = "forge_attn_fused_f32_host" if f32 else "forge_attn_fused_host"
+    _check(fn, getattr(load(), fn)(
+        _host(q, dt, "q"), _host(k, dt, "k"), _host(v, dt, "v"), _host(out, dt, "out"),
+        B, Hq, Hkv, Sq, Skv, D, int(mask_kind), lp, float(scale),
+        _dev(scratch, torch.uint8, "scratch"), scratch.numel(), _stream()))
+    return out
+
+
+def attn_decode_host_scratch_bytes(B, Hq, Hkv, Smax, D, num_splits) -> int:
+    return int(load().forge_attn_decode_host_scratch_bytes(B, Hq, Hkv, Smax, D, num_splits))
+
+
+def attn_decode_splitkv_host(q, k_cache, v_cache, lens, num_splits, out, scratch, scale=None):
+    B, Hq, D = q.shape
+    _, Hkv, Smax, _ = k_cache.shape
+    scale = D ** -0.5 if scale is None else scale
+    bf = torch.bfloat16
+    _check("forge_attn_decode_splitkv_host", load().forge_attn_decode_splitkv_host(
+        _host(q, bf, "q"), _host(k_cache, bf, "k_cache"), _host(v_cache, bf, "v_cache"), _host(out, bf, "out"),
+        B, Hq, Hkv, Smax, D, _host(lens, torch.int32, "lens"), int(num_splits), float(scale),
+        _dev(scratch, torch.uint8, "scratch"), scratch.numel(), _stream()))
+    return out
+
+
+def linear_host_scratch_bytes(M, N, K) -> int:
+    return int(load().forge_linear_host_scratch_bytes(M, N, K))
+
+
+def linear_bias_gelu_host(x, w, b, out, scratch):
+    M, K = x.shape
+    _, N = w.shape
+    bf = torch.bfloat16
+    _check("forge_linear_bias_gelu_host", load().forge_linear_bias_gelu_host(
+        _host(x, bf, "x"), _host(w, bf, "w"), _host(b, bf, "b"), _host(out, bf, "out"), M, N, K,
+        _dev(scratch, torch.uint8, "scratch"), scratch.numel(), _stream()))
+    return out
+
+
+def check_status() -> None:
+    """Synchronises the current stream and raises if a kernel gave up on a bounded wait."""
+    _check("forge_check_status", load().forge_check_status(_stream()))
+
+
+def launch_count() -> int:
+    return int(load().forge_launch_count())

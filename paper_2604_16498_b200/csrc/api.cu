@@ -1,0 +1,230 @@
+// Host-side plumbing of the C ABI: status strings, error bookkeeping, launch counter,
+// the device status word, tensor-map encoding and the host-buffer variants.
+#include <atomic>
+#include <cstring>
+
+#include "forge_common.cuh"
+#include "tmap.cuh"
+
+namespace forge {
+
+namespace {
+thread_local int tl_last_cuda_error = 0;
+std::atomic<unsigned long long> g_launches{0};
+__device__ int g_device_status = 0;
+}  // namespace
+
+void set_last_cuda_error(cudaError_t e) { tl_last_cuda_error = static_cast<int>(e); }
+void count_launch(int n) { g_launches.fetch_add(static_cast<unsigned long long>(n), std::memory_order_relaxed); }
+
+int* device_status_word() {
+    // Resolved per device: the symbol has one instance per device that loads the module.
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+    static int* cache[64] = {nullptr};
+    if (dev < 0 || dev >= 64) return nullptr;
+    if (!cache[dev]) {
+        void* p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_device_status);
+        if (e != cudaSuccess) { set_last_cuda_error(e); return nullptr; }
+        cache[dev] = static_cast<int*>(p);
+    }
+    return cache[dev];
+}
+
+bool encode_tmap_bf16_sw128(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
+                            const uint64_t* strides_bytes, const uint32_t* box) {
+    using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static EncodeFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres);
+        if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !p) {
+            set_last_cuda_error(e != cudaSuccess ? e : cudaErrorUnknown);
+            return false;
+        }
+        fn = reinterpret_cast<EncodeFn>(p);
+    }
+    cuuint64_t gdim[5];
+    cuuint64_t gstride[5];
+    cuuint32_t gbox[5];
+    cuuint32_t estride[5];
+    for (int i = 0; i < rank; ++i) {
+        gdim[i] = dims[i];
+        gbox[i] = box[i];
+        estride[i] = 1;
+        if (i + 1 < rank) gstride[i] = strides_bytes[i];
+    }
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, static_cast<cuuint32_t>(rank), const_cast<void*>(base),
+                    gdim, gstride, gbox, estride, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_last_cuda_error(cudaErrorInvalidValue);
+        return false;
+    }
+    return true;
+}
+
+}  // namespace forge
+
+extern "C" const char* forge_status_string(int status) {
+    switch (status) {
+        case FORGE_OK: return "FORGE_OK";
+        case FORGE_ERR_INVALID_ARG: return "FORGE_ERR_INVALID_ARG";
+        case FORGE_ERR_UNSUPPORTED: return "FORGE_ERR_UNSUPPORTED";
+        case FORGE_ERR_WORKSPACE: return "FORGE_ERR_WORKSPACE";
+        case FORGE_ERR_CUDA: return "FORGE_ERR_CUDA";
+        case FORGE_ERR_TIMEOUT: return "FORGE_ERR_TIMEOUT";
+        default: return "FORGE_ERR_UNKNOWN";
+    }
+}
+
+extern "C" int forge_last_cuda_error(void) { return forge::tl_last_cuda_error; }
+
+extern "C" unsigned long long forge_launch_count(void) {
+    return forge::g_launches.load(std::memory_order_relaxed);
+}
+
+extern "C" int forge_check_status(void* stream) {
+    using namespace forge;
+    FORGE_CUDA_TRY(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    int* word = device_status_word();
+    if (!word) return FORGE_ERR_CUDA;
+    int host = 0;
+    FORGE_CUDA_TRY(cudaMemcpy(&host, word, sizeof(int), cudaMemcpyDeviceToHost));
+    if (host != 0) {
+        FORGE_CUDA_TRY(cudaMemset(word, 0, sizeof(int)));
+        return FORGE_ERR_TIMEOUT;
+    }
+    return FORGE_OK;
+}
+
+// ------------------------------------------------------------------ host-buffer variants
+namespace {
+inline size_t up256(size_t n) { return (n + 255) & ~(size_t)255; }
+}  // namespace
+
+extern "C" size_t forge_attn_host_scratch_bytes(int B, int Hq, int Hkv, int Sq, int Skv, int D, int elem_bytes) {
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Skv <= 0 || D <= 0 || elem_bytes <= 0) return 0;
+    const size_t qo = (size_t)B * Hq * Sq * D * elem_bytes;
+    const size_t kv = (size_t)B * Hkv * Skv * D * elem_bytes;
+    return 2 * up256(qo) + 2 * up256(kv) + up256((size_t)B * 4);
+}
+
+static int attn_host_impl(bool f32, const void* q, const void* k, const void* v, void* out,
+                          int B, int Hq, int Hkv, int Sq, int Skv, int D,
+                          int mask_kind, const int32_t* lens, float scale,
+                          void* dev_scratch, size_t dev_scratch_bytes, void* stream) {
+    using namespace forge;
+    if (!q || !k || !v || !out || !dev_scratch) return FORGE_ERR_INVALID_ARG;
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Skv <= 0 || D <= 0) return FORGE_ERR_INVALID_ARG;
+    if ((mask_kind & FORGE_MASK_PADDING) && !lens) return FORGE_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(dev_scratch) & 255u) return FORGE_ERR_INVALID_ARG;
+    const int es = f32 ? 4 : 2;
+    if (dev_scratch_bytes < forge_attn_host_scratch_bytes(B, Hq, Hkv, Sq, Skv, D, es)) return FORGE_ERR_WORKSPACE;
+    const size_t qo = (size_t)B * Hq * Sq * D * es, kv = (size_t)B * Hkv * Skv * D * es;
+    char* p = static_cast<char*>(dev_scratch);
+    void* dq = p; p += up256(qo);
+    void* dk = p; p += up256(kv);
+    void* dv = p; p += up256(kv);
+    void* dout = p; p += up256(qo);
+    int32_t* dlens = reinterpret_cast<int32_t*>(p);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    FORGE_CUDA_TRY(cudaMemcpyAsync(dq, q, qo, cudaMemcpyHostToDevice, s));
+    FORGE_CUDA_TRY(cudaMemcpyAsync(dk, k, kv, cudaMemcpyHostToDevice, s));
+    FORGE_CUDA_TRY(cudaMemcpyAsync(dv, v, kv, cudaMemcpyHostToDevice, s));
+    if (lens) FORGE_CUDA_TRY(cudaMemcpyAsync(dlens, lens, (size_t)B * 4, cudaMemcpyHostToDevice, s));
+    int st = f32 ? forge_attn_fused_f32(dq, dk, dv, dout, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens ? dlens : nullptr,
+                                        scale, stream)
+                 : forge_attn_fused(dq, dk, dv, dout, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens ? dlens : nullptr,
+                                    scale, stream);
+    if (st != FORGE_OK) return st;
+    FORGE_CUDA_TRY(cudaMemcpyAsync(out, dout, qo, cudaMemcpyDeviceToHost, s));
+    return FORGE_OK;
+}
+
+extern "C" int forge_attn_fused_host(const void* q, const void* k, const void* v, void* out,
+                                     int B, int Hq, int Hkv, int Sq, int Skv, int D,
+                                     int mask_kind, const int32_t* lens, float scale,
+                                     void* dev_scratch, size_t dev_scratch_bytes, void* stream) {
+    return attn_host_impl(false, q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, dev_scratch,
+                          dev_scratch_bytes, stream);
+}
+
+extern "C" int forge_attn_fused_f32_host(const void* q, const void* k, const void* v, void* out,
+                                         int B, int Hq, int Hkv, int Sq, int Skv, int D,
+                                         int mask_kind, const int32_t* lens, float scale,
+                                         void* dev_scratch, size_t dev_scratch_bytes, void* stream) {
+    return attn_host_impl(true, q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, dev_scratch,
+                          dev_scratch_bytes, stream);
+}
+
+extern "C" size_t forge_attn_decode_host_scratch_bytes(int B, int Hq, int Hkv, int Smax, int D, int num_splits) {
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || Smax <= 0 || D <= 0 || num_splits <= 0) return 0;
+    const size_t qo = (size_t)B * Hq * D * 2, kv = (size_t)B * Hkv * Smax * D * 2;
+    return 2 * up256(qo) + 2 * up256(kv) + up256((size_t)B * 4) +
+           up256(forge_attn_decode_workspace_bytes(B, Hq, D, num_splits));
+}
+
+extern "C" int forge_attn_decode_splitkv_host(const void* q, const void* k_cache, const void* v_cache, void* out,
+                                              int B, int Hq, int Hkv, int Smax, int D,
+                                              const int32_t* lens, int num_splits, float scale,
+                                              void* dev_scratch, size_t dev_scratch_bytes, void* stream) {
+    using namespace forge;
+    if (!q || !k_cache || !v_cache || !out || !lens || !dev_scratch) return FORGE_ERR_INVALID_ARG;
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || Smax <= 0 || D <= 0 || num_splits <= 0) return FORGE_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(dev_scratch) & 255u) return FORGE_ERR_INVALID_ARG;
+    if (dev_scratch_bytes < forge_attn_decode_host_scratch_bytes(B, Hq, Hkv, Smax, D, num_splits))
+        return FORGE_ERR_WORKSPACE;
+    const size_t qo = (size_t)B * Hq * D * 2, kv = (size_t)B * Hkv * Smax * D * 2;
+    const size_t wsb = forge_attn_decode_workspace_bytes(B, Hq, D, num_splits);
+    char* p = static_cast<char*>(dev_scratch);
+    void* dq = p; p += up256(qo);
+    void* dk = p; p += up256(kv);
+    void* dv = p; p += up256(kv);
+    void* dout = p; p += up256(qo);
+    int32_t* dlens = reinterpret_cast<int32_t*>(p); p += up256((size_t)B * 4);
+    void* ws = p;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    FORGE_CUDA_TRY(cudaMemcpyAsync(dq, q, qo, cudaMemcpyHostToDevice, s));
+    FORGE_CUDA_TRY(cudaMemcpyAsync(dk, k_cache, kv, cudaMemcpyHostToDevice, s));
+    FORGE_CUDA_TRY(cudaMemcpyAsync(dv, v_cache, kv, cudaMemcpyHostToDevice, s));
+    FORGE_CUDA_TRY(cudaMemcpyAsync(dlens, lens, (size_t)B * 4, cudaMemcpyHostToDevice, s));
+    int st = forge_attn_decode_splitkv(dq, dk, dv, dout, B, Hq, Hkv, Smax, D, dlens, num_splits, scale, ws, wsb,
+                                       stream);
+    if (st != FORGE_OK) return st;
+    FORGE_CUDA_TRY(cudaMemcpyAsync(out, dout, qo, cudaMemcpyDeviceToHost, s));
+    return FORGE_OK;
+}
+
+extern "C" size_t forge_linear_host_scratch_bytes(int M, int N, int K) {
+    if (M <= 0 || N <= 0 || K <= 0) return 0;
+    return up256((size_t)M * K * 2) + up256((size_t)K * N * 2) + up256((size_t)N * 2) + up256((size_t)M * N * 2);
+}
+
+extern "C" int forge_linear_bias_gelu_host(const void* x, const void* w, const void* b, void* y,
+                                           int M, int N, int K,
+                                           void* dev_scratch, size_t dev_scratch_bytes, void* stream) {
+    using namespace forge;
+    if (!x || !w || !b || !y || !dev_scratch) return FORGE_ERR_INVALID_ARG;
+    if (M <= 0 || N <= 0 || K <= 0) return FORGE_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(dev_scratch) & 255u) return FORGE_ERR_INVALID_ARG;
+    if (dev_scratch_bytes < forge_linear_host_scratch_bytes(M, N, K)) return FORGE_ERR_WORKSPACE;
+    const size_t xb = (size_t)M * K * 2, wb = (size_t)K * N * 2, bb = (size_t)N * 2, yb = (size_t)M * N * 2;
+    char* p = static_cast<char*>(dev_scratch);
+    void* dx = p; p += up256(xb);
+    void* dw = p; p += up256(wb);
+    void* db = p; p += up256(bb);
+    void* dy = p;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    FORGE_CUDA_TRY(cudaMemcpyAsync(dx, x, xb, cudaMemcpyHostToDevice, s));
+    FORGE_CUDA_TRY(cudaMemcpyAsync(dw, w, wb, cudaMemcpyHostToDevice, s));
+    FORGE_CUDA_TRY(cudaMemcpyAsync(db, b, bb, cudaMemcpyHostToDevice, s));
+    int st = forge_linear_bias_gelu(dx, dw, db, dy, M, N, K, stream);
+    if (st != FORGE_OK) return st;
+    FORGE_CUDA_TRY(cudaMemcpyAsync(y, dy, yb, cudaMemcpyDeviceToHost, s));
+    return FORGE_OK;
+}

@@ -1,0 +1,54 @@
+// Shared host-side plumbing of the library: status bookkeeping, launch counting,
+// argument checks.  Nothing here computes anything of the operators.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cstddef>
+#include <cstdint>
+
+#include "../../include/forge.h"
+
+namespace forge {
+
+// Per-thread record of the last failing CUDA call (returned by forge_last_cuda_error()).
+void set_last_cuda_error(cudaError_t e);
+// Counts a kernel launch (returned by forge_launch_count()).
+void count_launch(int n = 1);
+// Device-side status word, set by kernels whose bounded waits expire.
+int* device_status_word();   // device address, resolved once per process
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Checks a launch: returns FORGE_OK or records the error and returns FORGE_ERR_CUDA.
+inline int finish_launch(int nkernels) {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { set_last_cuda_error(e); return FORGE_ERR_CUDA; }
+    count_launch(nkernels);
+    return FORGE_OK;
+}
+
+#define FORGE_CUDA_TRY(expr)                                         \
+    do {                                                             \
+        cudaError_t e__ = (expr);                                    \
+        if (e__ != cudaSuccess) {                                    \
+            ::forge::set_last_cuda_error(e__);                       \
+            return FORGE_ERR_CUDA;                                   \
+        }                                                            \
+    } while (0)
+
+// Common validation of the attention entry points' scalar arguments and pointers.
+inline int check_attn_args(const void* q, const void* k, const void* v, const void* out,
+                           int B, int Hq, int Hkv, int Sq, int Skv, int D,
+                           int mask_kind, const int32_t* lens) {
+    if (!q || !k || !v || !out) return FORGE_ERR_INVALID_ARG;
+    if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Skv <= 0 || D <= 0) return FORGE_ERR_INVALID_ARG;
+    if (Hq % Hkv != 0) return FORGE_ERR_INVALID_ARG;
+    if (mask_kind < 0 || mask_kind > 3) return FORGE_ERR_INVALID_ARG;
+    if ((mask_kind & FORGE_MASK_PADDING) && !lens) return FORGE_ERR_INVALID_ARG;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return FORGE_ERR_INVALID_ARG;
+    if (lens && (reinterpret_cast<uintptr_t>(lens) & 3u)) return FORGE_ERR_INVALID_ARG;
+    if (D != 64 && D != 128) return FORGE_ERR_UNSUPPORTED;
+    return FORGE_OK;
+}
+
+}  // namespace forge

@@ -1,0 +1,245 @@
+// Fused Linear + bias + tanh-GELU (Listing 6 / Eq. 11): Y = gelu_tanh(X W + b) in one kernel.
+// The fp32 accumulator lives in tensor memory; bias and activation are applied to it as it is
+// read back, before the single rounding to bf16 -- the linear output never reaches memory.
+//
+// Persistent, warp-specialised kernel, one CTA per SM:
+//   warp 0    : TMA producer  (X tile 128 x 64, W tile 64 x BN per stage, 128-byte swizzle)
+//   warp 1    : tcgen05.mma issuer (one elected lane), owns the TMEM allocation
+//   warps 2-5 : epilogue (TMEM -> registers -> +bias -> GELU -> bf16 -> global)
+// Two TMEM accumulators: the epilogue of tile i overlaps the main loop of tile i+1.
+// X [M,K] is the K-major A operand; W [K,N] (N contiguous) is the MN-major B operand, so no
+// transposed copy of the weights is needed.
+#include <cuda_bf16.h>
+
+#include "forge_common.cuh"
+#include "sm100_ptx.cuh"
+#include "tmap.cuh"
+
+namespace forge {
+namespace {
+
+using namespace ptx;
+
+constexpr int kBM = 128;
+constexpr int kBK = 64;
+constexpr int kThreads = 192;
+constexpr int kEpiThreads = 128;
+constexpr int kAccStride = 256;   // TMEM columns between the two accumulators
+constexpr int kTmemCols = 512;
+
+template <int BN, int STAGES>
+struct LinearSmem {
+    static constexpr int kABytes = kBM * kBK * 2;        // 16 KB
+    static constexpr int kBBytes = kBK * BN * 2;         // 64 rows of K x BN
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kBarOffset = STAGES * kStageBytes;
+    // barriers: full[S], empty[S], tmem_full[2], tmem_empty[2]; then the TMEM base, then bias[2][BN]
+    static constexpr int kBiasOffset = kBarOffset + (2 * STAGES + 4) * 8 + 16;
+    static constexpr int kTotal = kBiasOffset + 2 * BN * 4;
+    static constexpr int kAlloc = kTotal + 1024;         // slack to align the base to 1024 bytes
+};
+
+__device__ __forceinline__ float gelu_tanh_f32(float z) {
+    // 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3)))
+    const float u = 0.7978845608028654f * z * fmaf(0.044715f * z, z, 1.0f);
+    float t;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(u));
+    const float hz = 0.5f * z;
+    return fmaf(hz, t, hz);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+template <int BN, int STAGES>
+__global__ void __launch_bounds__(kThreads, 1)
+linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+                        const __nv_bfloat16* __restrict__ bias, __nv_bfloat16* __restrict__ y,
+                        int M, int N, int K, int* __restrict__ status) {
+    using L = LinearSmem<BN, STAGES>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::kBarOffset);
+    uint64_t* empty = full + STAGES;
+    uint64_t* tmem_full = empty + STAGES;
+    uint64_t* tmem_empty = tmem_full + 2;
+    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+    float* s_bias = reinterpret_cast<float*>(smem + L::kBiasOffset);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tiles_m = (M + kBM - 1) / kBM, tiles_n = (N + BN - 1) / BN;
+    const int num_tiles = tiles_m * tiles_n;
+    const int kblocks = (K + kBK - 1) / kBK;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < STAGES; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&tmem_full[i], 1); mbar_init(&tmem_empty[i], kEpiThreads / 32); }
+        fence_mbar_init();
+        prefetch_tmap(&tmap_x);
+        prefetch_tmap(&tmap_w);
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_base_slot, kTmemCols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_base_slot;
+    bool failed = false;
+
+    if (warp == 0) {
+        if (elect_one()) {
+            int stage = 0;
+            uint32_t phase = 0;
+            for (int tile = blockIdx.x; tile < num_tiles && !failed; tile += gridDim.x) {
+                const int m0 = (tile / tiles_n) * kBM, n0 = (tile % tiles_n) * BN;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!mbar_wait(&empty[stage], phase ^ 1)) { failed = true; break; }
+                    uint8_t* sa = smem + stage * L::kStageBytes;
+                    uint8_t* sb = sa + L::kABytes;
+                    mbar_expect_tx(&full[stage], L::kStageBytes);
+                    tma_load_2d(sa, &tmap_x, &full[stage], kb * kBK, m0);
+#pragma unroll
+                    for (int c = 0; c < BN / 64; ++c)
+                        tma_load_2d(sb + c * (kBK * 128), &tmap_w, &full[stage], n0 + c * 64, kb * kBK);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (elect_one()) {
+            constexpr uint32_t idesc = make_idesc_bf16(kBM, BN, /*a_mn_major=*/false, /*b_mn_major=*/true);
+            int stage = 0;
+            uint32_t phase = 0;
+            int it = 0;
+            for (int tile = blockIdx.x; tile < num_tiles && !failed; tile += gridDim.x, ++it) {
+                const int acc = it & 1;
+                const uint32_t acc_phase = (it >> 1) & 1;
+                if (!mbar_wait(&tmem_empty[acc], acc_phase ^ 1)) { failed = true; break; }
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + acc * kAccStride;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!mbar_wait(&full[stage], phase)) { failed = true; break; }
+                    tc_fence_after_sync();
+                    const uint32_t sa = smem_u32(smem + stage * L::kStageBytes);
+                    const uint32_t sb = sa + L::kABytes;
+#pragma unroll
+                    for (int k = 0; k < kBK / 16; ++k) {
+                        // A: 16 K-elements = 32 bytes further along the 128-byte swizzled row
+                        const uint64_t a_desc = make_smem_desc(sa + k * 32, 16, 1024);
+                        // B: 16 K-rows = two 1024-byte groups further; 64-column chunks are kBK*128 bytes apart
+                        const uint64_t b_desc = make_smem_desc(sb + k * 2048, kBK * 128, 1024);
+                        mma_ss(d_tmem, a_desc, b_desc, idesc, (kb | k) != 0);
+                    }
+                    mma_commit(&empty[stage]);  // the stage is free once these MMAs have read it
+                    if (++stage == STAGES) { stage = 0; phase ^= 1; }
+                }
+                if (failed) break;
+                mma_commit(&tmem_full[acc]);
+            }
+        }
+    } else {
+        const int quarter = warp & 3;            // TMEM lane quarter this warp may access
+        const int etid = (warp - 2) * 32 + lane; // 0..127
+        int it = 0;
+        for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
+            const int m0 = (tile / tiles_n) * kBM, n0 = (tile % tiles_n) * BN;
+            const int acc = it & 1;
+            const uint32_t acc_phase = (it >> 1) & 1;
+            float* bias_s = s_bias + acc * BN;
+            for (int i = etid; i < BN; i += kEpiThreads)
+                bias_s[i] = (n0 + i < N) ? __bfloat162float(bias[n0 + i]) : 0.f;
+            asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+            // A warp that gave up keeps taking part in the named barrier above (so the others never
+            // wait for it there) but skips the work.
+            if (!failed && !mbar_wait(&tmem_full[acc], acc_phase)) failed = true;
+            if (failed) continue;
+            tc_fence_after_sync();
+            const int row = m0 + quarter * 32 + lane;
+            const uint32_t taddr = tmem_base + acc * kAccStride + (static_cast<uint32_t>(quarter * 32) << 16);
+            __nv_bfloat16* yrow = y + (size_t)row * N + n0;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld_x32(taddr + c * 32, r);
+                tmem_ld_wait();
+                uint32_t packed[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const float z0 = __uint_as_float(r[2 * i]) + bias_s[c * 32 + 2 * i];
+                    const float z1 = __uint_as_float(r[2 * i + 1]) + bias_s[c * 32 + 2 * i + 1];
+                    packed[i] = pack_bf16(gelu_tanh_f32(z0), gelu_tanh_f32(z1));
+                }
+                if (row < M) {
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        if (n0 + c * 32 + v * 8 < N)  // N is a multiple of 8: an 8-column group is all in or all out
+                            *reinterpret_cast<uint4*>(yrow + c * 32 + v * 8) =
+                                make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+                    }
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tmem_empty[acc]);
+        }
+    }
+
+    if (failed) {
+        atomicExch(status, 1);
+        // give copies and MMAs that are still in flight time to land before TMEM and smem go away
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+template <int BN, int STAGES>
+int launch_linear(const void* x, const void* w, const void* b, void* y, int M, int N, int K, cudaStream_t s) {
+    using L = LinearSmem<BN, STAGES>;
+    CUtensorMap tmap_x, tmap_w;
+    {
+        const uint64_t dims[2] = {(uint64_t)K, (uint64_t)M};
+        const uint64_t strides[1] = {(uint64_t)K * 2};
+        const uint32_t box[2] = {kBK, kBM};
+        if (!encode_tmap_bf16_sw128(&tmap_x, x, 2, dims, strides, box)) return FORGE_ERR_CUDA;
+    }
+    {
+        const uint64_t dims[2] = {(uint64_t)N, (uint64_t)K};
+        const uint64_t strides[1] = {(uint64_t)N * 2};
+        const uint32_t box[2] = {64, kBK};
+        if (!encode_tmap_bf16_sw128(&tmap_w, w, 2, dims, strides, box)) return FORGE_ERR_CUDA;
+    }
+    int* status = device_status_word();
+    if (!status) return FORGE_ERR_CUDA;
+    int dev = 0, sms = 0;
+    FORGE_CUDA_TRY(cudaGetDevice(&dev));
+    FORGE_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    auto kernel = linear_bias_gelu_kernel<BN, STAGES>;
+    FORGE_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kAlloc));
+    const int tiles = ((M + kBM - 1) / kBM) * ((N + BN - 1) / BN);
+    const int grid = tiles < sms ? tiles : sms;
+    kernel<<<grid, kThreads, L::kAlloc, s>>>(tmap_x, tmap_w, static_cast<const __nv_bfloat16*>(b),
+                                             static_cast<__nv_bfloat16*>(y), M, N, K, status);
+    return finish_launch(1);
+}
+
+}  // namespace
+}  // namespace forge
+
+extern "C" int forge_linear_bias_gelu(const void* x, const void* w, const void* b, void* y,
+                                      int M, int N, int K, void* stream) {
+    using namespace forge;
+    if (!x || !w || !b || !y) return FORGE_ERR_INVALID_ARG;
+    if (M <= 0 || N <= 0 || K <= 0) return FORGE_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(w) || !aligned16(b) || !aligned16(y)) return FORGE_ERR_INVALID_ARG;
+    if ((K % 8) != 0 || (N % 8) != 0) return FORGE_ERR_UNSUPPORTED;
+    return launch_linear<192, 5>(x, w, b, y, M, N, K, static_cast<cudaStream_t>(stream));
+}

@@ -155,7 +155,7 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
             asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
             // A warp that gave up keeps taking part in the named barrier above (so the others never
             // wait for it there) but skips the work.
-            if (!failed && !mbar_wait(&tmem_full[acc], acc_phase)) failed = true;
+            if (!failed && !warp_wait(&tmem_full[acc], acc_phase)) failed = true;
             if (failed) continue;
             tc_fence_after_sync();
             const int row = m0 + quarter * 32 + lane;

@@ -100,6 +100,35 @@ int forge_attn_decode_splitkv(const void* q, const void* k_cache, const void* v_
 size_t forge_attn_decode_workspace_bytes(int B, int Hq, int D, int num_splits);
 
 /*
+ * forge_attn_decode_splitkv for callers that cannot provide a workspace because they cannot
+ * allocate device memory at all (the paper has no counterpart to this entry point; it exists
+ * for deployment reasons only).  Typical cases: a serving process whose device-memory plan is
+ * frozen once it has started, a plugin inside a host runtime that owns the allocator, a latency
+ * path that must avoid the device-wide synchronisation cudaMalloc implies.
+ *
+ * The split partials go to a fixed array of FORGE_DECODE_STATIC_SCRATCH_BYTES that is compiled
+ * into the library's device image; every GPU that loads the library holds that much memory until
+ * the process exits.  The call itself allocates and frees nothing, on the host or on the device.
+ * Inputs, `out` and `lens` are still the caller's device buffers, with the same meaning, layout
+ * and limits as forge_attn_decode_splitkv, and the result is the same.
+ *
+ *   - Problems whose partials do not fit, i.e. forge_attn_decode_workspace_bytes(B, Hq, D,
+ *     num_splits) > FORGE_DECODE_STATIC_SCRATCH_BYTES, are refused with FORGE_ERR_WORKSPACE and
+ *     nothing is launched (B=16, Hq=32, D=128, 16 splits needs 4.1 MiB).
+ *   - The first call on each device looks up the array's device address (the device must be
+ *     current).  Make that first call outside any stream capture; later calls do no set-up.
+ *   - All calls on a device share the one array, and it keeps whatever the previous call left
+ *     there.  The kernels overwrite every slot they later read, so nothing needs clearing, but
+ *     two calls that may run at the same time on one GPU (different streams, threads or
+ *     processes sharing the context) race on it and give wrong results: serialise them, or use
+ *     forge_attn_decode_splitkv with one workspace per concurrent call.
+ */
+#define FORGE_DECODE_STATIC_SCRATCH_BYTES (8u << 20)
+int forge_attn_decode_splitkv_static(const void* q, const void* k_cache, const void* v_cache, void* out,
+                                     int B, int Hq, int Hkv, int Smax, int D,
+                                     const int32_t* lens, int num_splits, float scale, void* stream);
+
+/*
  * Fused Linear + bias + tanh-GELU (Listing 6 / Eq. 11):
  *     y[m,n] = gelu_tanh(b[n] + sum_k x[m,k] * w[k,n]),
  *     gelu_tanh(z) = 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3)))

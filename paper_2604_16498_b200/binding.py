@@ -27,6 +27,7 @@ SIGNATURES = {
     "forge_attn_fused_f32": (_i, _ATTN + [_vp]),
     "forge_attn_decode_splitkv": (_i, _DEC + [_vp, _sz, _vp]),
     "forge_attn_decode_workspace_bytes": (_sz, [_i, _i, _i, _i]),
+    "forge_attn_decode_splitkv_static": (_i, _DEC + [_vp]),
     "forge_linear_bias_gelu": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
     "forge_attn_host_scratch_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _i]),
     "forge_attn_fused_host": (_i, _ATTN + [_vp, _sz, _vp]),
@@ -142,6 +143,26 @@ def attn_decode_splitkv(q, k_cache, v_cache, lens, num_splits, scale=None, out=N
         _dev(v_cache, torch.bfloat16, "v_cache"), _dev(out, torch.bfloat16, "out"),
         B, Hq, Hkv, Smax, D, _dev(lens, torch.int32, "lens"), int(num_splits), float(scale),
         _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream()))
+    return out
+
+
+DECODE_STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def attn_decode_splitkv_static(q, k_cache, v_cache, lens, num_splits, out, scale=None):
+    """forge_attn_decode_splitkv_static: the decode step for callers that cannot allocate a
+    workspace.  The partials go to a fixed 8 MiB array inside the library (shared by all calls on
+    the device, so calls must not overlap); larger problems raise ForgeError(ERR_WORKSPACE).
+    `out` is the caller's buffer: nothing is allocated here either."""
+    B, Hq, D = q.shape
+    Bk, Hkv, Smax, Dk = k_cache.shape
+    if (Bk, Dk) != (B, D) or tuple(v_cache.shape) != tuple(k_cache.shape):
+        raise ValueError("q [B,Hq,D], caches [B,Hkv,Smax,D] expected")
+    scale = D ** -0.5 if scale is None else scale
+    _check("forge_attn_decode_splitkv_static", load().forge_attn_decode_splitkv_static(
+        _dev(q, torch.bfloat16, "q"), _dev(k_cache, torch.bfloat16, "k_cache"),
+        _dev(v_cache, torch.bfloat16, "v_cache"), _dev(out, torch.bfloat16, "out"),
+        B, Hq, Hkv, Smax, D, _dev(lens, torch.int32, "lens"), int(num_splits), float(scale), _stream()))
     return out
 
 

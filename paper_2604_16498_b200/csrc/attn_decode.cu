@@ -11,6 +11,8 @@
 // cached row is read exactly once.
 #include <cuda_bf16.h>
 
+#include <mutex>
+
 #include "forge_common.cuh"
 
 namespace forge {
@@ -273,4 +275,60 @@ extern "C" int forge_attn_decode_splitkv(const void* q, const void* k_cache, con
     else
         decode_combine_kernel<128><<<B * Hq, 128, 0, s>>>(ws_o, ws_ml, static_cast<__nv_bfloat16*>(out), num_splits);
     return finish_launch(1);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Decode without a caller workspace.
+//
+// Some callers cannot hand over scratch memory because they cannot allocate any: a serving loop
+// whose device-memory plan is frozen after start-up, a plugin living inside a host runtime that
+// owns the allocator, or code on a latency path where cudaMalloc's implicit device synchronisation
+// is not acceptable.  For them the split partials live in a fixed array that is part of the
+// library's device image.  Every GPU that loads the library carries this array until the process
+// exits, whether or not the entry point is ever called.
+namespace forge {
+namespace {
+
+static __device__ __align__(256) unsigned char g_decode_static_scratch[FORGE_DECODE_STATIC_SCRATCH_BYTES];
+
+// In host code the array's name is only a handle for the runtime, not a device address; the address
+// has to be asked for, once per device, with that device current.
+void* static_scratch_for_current_device() {
+    constexpr int kMaxDevices = 64;
+    static void* cache[kMaxDevices] = {nullptr};
+    static std::mutex mu;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        set_last_cuda_error(cudaErrorInvalidDevice);
+        return nullptr;
+    }
+    std::lock_guard<std::mutex> lock(mu);
+    if (!cache[dev]) {
+        void* ptr = nullptr;
+        const cudaError_t e = cudaGetSymbolAddress(&ptr, g_decode_static_scratch);
+        if (e != cudaSuccess || !ptr) {
+            set_last_cuda_error(e != cudaSuccess ? e : cudaErrorInvalidSymbol);
+            return nullptr;
+        }
+        cache[dev] = ptr;
+    }
+    return cache[dev];
+}
+
+}  // namespace
+}  // namespace forge
+
+extern "C" int forge_attn_decode_splitkv_static(const void* q, const void* k_cache, const void* v_cache, void* out,
+                                                int B, int Hq, int Hkv, int Smax, int D,
+                                                const int32_t* lens, int num_splits, float scale, void* stream) {
+    using namespace forge;
+    if (B <= 0 || Hq <= 0 || D <= 0 || num_splits <= 0) return FORGE_ERR_INVALID_ARG;
+    // the partials of this problem, B * Hq * num_splits * (D + 2) * 4 bytes, must fit the fixed array
+    const size_t need = forge_attn_decode_workspace_bytes(B, Hq, D, num_splits);
+    if (need > (size_t)FORGE_DECODE_STATIC_SCRATCH_BYTES) return FORGE_ERR_WORKSPACE;
+    if (!q || !k_cache || !v_cache || !out || !lens) return FORGE_ERR_INVALID_ARG;
+    void* scratch = static_scratch_for_current_device();
+    if (!scratch) return FORGE_ERR_CUDA;
+    return forge_attn_decode_splitkv(q, k_cache, v_cache, out, B, Hq, Hkv, Smax, D, lens, num_splits, scale,
+                                     scratch, (size_t)FORGE_DECODE_STATIC_SCRATCH_BYTES, stream);
 }

@@ -5,10 +5,11 @@
 //     M = max_s m_s,   L = sum_s 2^(m_s - M) l_s,   out = sum_s 2^(m_s - M) O_s / L
 // (scores are kept in log2 units: they are pre-multiplied by scale * log2(e)).
 //
-// The kernel is bound by streaming K and V from HBM: every lane issues 128-bit loads that
-// cover whole 128-byte lines, K and V loads of a group of keys are issued together, and the
-// G = Hq / Hkv query heads that share a KV head are processed by the same CTA so that each
-// cached row is read exactly once.
+// The kernel is bound by streaming K and V from HBM: every lane issues 128-bit loads straight
+// into MMA fragments (no shared-memory staging), K and V loads of a block of rows are issued
+// together, and the G = Hq / Hkv query heads that share a KV head are processed by the same CTA
+// so that each cached row is read exactly once.  The dot products run on warp-level tensor-core
+// MMAs (m16n8k16) only because fp32 FMAs with shuffle reductions were bound by instruction issue.
 #include <cuda_bf16.h>
 
 #include <mutex>
@@ -20,7 +21,7 @@ namespace {
 
 constexpr int kWarps = 4;
 constexpr int kThreads = kWarps * 32;
-constexpr int kU = 4;  // 128-bit loads in flight per lane and per tensor
+constexpr int kBlockKeys = 16;  // cached rows per warp iteration
 
 __device__ __forceinline__ uint4 ld_stream(const void* p) {
     uint4 r;
@@ -29,29 +30,44 @@ __device__ __forceinline__ uint4 ld_stream(const void* p) {
                  : "l"(p));
     return r;
 }
-// bf16 pair packed in 32 bits -> two floats (exact widening)
-__device__ __forceinline__ float bf_lo(uint32_t w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float bf_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
-__device__ __forceinline__ void unpack8(const uint4& r, float (&f)[8]) {
-    f[0] = bf_lo(r.x); f[1] = bf_hi(r.x); f[2] = bf_lo(r.y); f[3] = bf_hi(r.y);
-    f[4] = bf_lo(r.z); f[5] = bf_hi(r.z); f[6] = bf_lo(r.w); f[7] = bf_hi(r.w);
+
+// D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col).  Lane = (g = lane / 4, c = lane % 4):
+//   A: a0 = (row g, k 2c..2c+1)  a1 = (row g+8, k 2c..)  a2 = (row g, k 2c+8..)  a3 = (row g+8, k 2c+8..)
+//   B: b0 = (k 2c..2c+1, col g)  b1 = (k 2c+8.., col g)
+//   D: d0 = (row g, col 2c)  d1 = (row g, col 2c+1)  d2 = (row g+8, col 2c)  d3 = (row g+8, col 2c+1)
+__device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, "
+                 "{%8, %9}, {%0, %1, %2, %3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// grid = (num_splits, Hkv, B)
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// grid = (num_splits, Hkv, B).  Each warp walks its share of the split in blocks of 16 cached rows:
+//   S[head, key]  = Q K^T   as m16n8k16 with A = Q (rows = the G heads, padded with zero rows) and
+//                   B = K rows straight from global memory (the contraction runs over the head
+//                   dimension in whatever order the 16-byte loads deliver it, the same for Q and K);
+//   online softmax on the accumulator fragment (lane (g, c) owns head g, keys 2c, 2c+1 of each 8);
+//   O^T[dim, head] += V^T P^T  with A = pairs of V rows interleaved with byte permutes and B = the
+//                   probabilities exactly where the first MMA left them.
+// The arithmetic is a few instructions per cached row, so the kernel is bound by the HBM stream.
 template <int D, int G>
 __global__ void __launch_bounds__(kThreads)
 decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ kc,
                     const __nv_bfloat16* __restrict__ vc, const int32_t* __restrict__ lens,
                     float* __restrict__ ws_o, float* __restrict__ ws_ml,
                     int Hq, int Hkv, int Smax, int num_splits, float scale_log2) {
-    constexpr int LPK = D / 8;     // lanes that share one cached row (16 bytes each)
-    constexpr int KPL = 32 / LPK;  // rows covered by one warp-wide load
-    constexpr int KPI = KPL * kU;  // rows per warp iteration
+    constexpr int NKB = D / 32;  // 32-dim blocks of the head dimension (two k16 MMAs each)
+    constexpr int NHB = D / 64;  // 64-dim blocks of the output (four 16-dim MMAs each)
 
     const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int sub = lane / LPK;    // which of the KPL rows of a load this lane reads
-    const int chunk = lane % LPK;  // which 8 dims of the row
+    const int g = lane >> 2, c = lane & 3;
 
     const int len = min(max(lens[b], 0), Smax);
     const int per = (len + num_splits - 1) / num_splits;
@@ -62,132 +78,144 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     __shared__ float sm_l[kWarps][G];
     __shared__ __align__(16) float sm_acc[kWarps][G][D];
 
-    // query rows of the G heads, pre-scaled; each lane keeps its 8 dims
-    float qf[G][8];
+    // Q fragment: head g (zero rows for g >= G), 8 dims at c*8 of every 32-dim block
+    uint32_t qr[NKB][4];
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
-        const uint4 raw = *reinterpret_cast<const uint4*>(q + ((size_t)b * Hq + kvh * G + g) * D + chunk * 8);
-        unpack8(raw, qf[g]);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) qf[g][i] *= scale_log2;
+    for (int kb = 0; kb < NKB; ++kb) {
+        uint4 raw = make_uint4(0, 0, 0, 0);
+        if (g < G) raw = *reinterpret_cast<const uint4*>(q + ((size_t)b * Hq + kvh * G + g) * D + kb * 32 + c * 8);
+        qr[kb][0] = raw.x; qr[kb][1] = raw.y; qr[kb][2] = raw.z; qr[kb][3] = raw.w;
     }
 
-    float m_run[G], l_run[G], acc[G][8];
+    float m_run = -INFINITY, l_run = 0.f;  // of head g (lanes with g >= G carry dummies)
+    float acc[NHB][4][4];                  // O^T fragments: [64-dim block][16-dim MMA][d0..d3]
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
-        m_run[g] = -INFINITY;
-        l_run[g] = 0.f;
+    for (int hb = 0; hb < NHB; ++hb)
 #pragma unroll
-        for (int i = 0; i < 8; ++i) acc[g][i] = 0.f;
-    }
+        for (int t = 0; t < 4; ++t)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[hb][t][i] = 0.f;
 
-    const __nv_bfloat16* kbase = kc + ((size_t)b * Hkv + kvh) * (size_t)Smax * D + chunk * 8;
-    const __nv_bfloat16* vbase = vc + ((size_t)b * Hkv + kvh) * (size_t)Smax * D + chunk * 8;
+    const __nv_bfloat16* kbase = kc + ((size_t)b * Hkv + kvh) * (size_t)Smax * D;
+    const __nv_bfloat16* vbase = vc + ((size_t)b * Hkv + kvh) * (size_t)Smax * D;
 
-    for (int j0 = s0 + warp * KPI; j0 < s1; j0 += kWarps * KPI) {
-        uint4 kr[kU], vr[kU];
+    for (int j0 = s0 + warp * kBlockKeys; j0 < s1; j0 += kWarps * kBlockKeys) {
+        // K: rows j0 + u*8 + g, 16 bytes at dims kb*32 + c*8.  V: rows j0 + {2c, 2c+1, 2c+8, 2c+9},
+        // 16 bytes at dims hb*64 + g*8.  Rows at or beyond s1 are not read (zeros).
+        uint4 kr[2][NKB], vr[4][NHB];
 #pragma unroll
-        for (int u = 0; u < kU; ++u) {
-            const int j = j0 + u * KPL + sub;
-            if (j < s1) {
-                kr[u] = ld_stream(kbase + (size_t)j * D);
-                vr[u] = ld_stream(vbase + (size_t)j * D);
-            } else {
-                kr[u] = make_uint4(0, 0, 0, 0);
-                vr[u] = make_uint4(0, 0, 0, 0);
+        for (int u = 0; u < 2; ++u) {
+            const int j = j0 + u * 8 + g;
+#pragma unroll
+            for (int kb = 0; kb < NKB; ++kb)
+                kr[u][kb] = (j < s1) ? ld_stream(kbase + (size_t)j * D + kb * 32 + c * 8) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int j = j0 + 2 * c + (r & 1) + (r >> 1) * 8;
+#pragma unroll
+            for (int hb = 0; hb < NHB; ++hb)
+                vr[r][hb] = (j < s1) ? ld_stream(vbase + (size_t)j * D + hb * 64 + g * 8) : make_uint4(0, 0, 0, 0);
+        }
+
+        // scores: s[u][0..1] = head g, keys j0 + u*8 + 2c + {0, 1}  (s[u][2..3] belong to zero rows)
+        float s[2][4];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            s[u][0] = s[u][1] = s[u][2] = s[u][3] = 0.f;
+#pragma unroll
+            for (int kb = 0; kb < NKB; ++kb) {
+                mma16816(s[u], qr[kb][0], 0u, qr[kb][1], 0u, kr[u][kb].x, kr[u][kb].y);
+                mma16816(s[u], qr[kb][2], 0u, qr[kb][3], 0u, kr[u][kb].z, kr[u][kb].w);
             }
         }
-        float s[kU][G];
+        float mt = -INFINITY;
 #pragma unroll
-        for (int u = 0; u < kU; ++u) {
-            float kf[8];
-            unpack8(kr[u], kf);
+        for (int u = 0; u < 2; ++u)
 #pragma unroll
-            for (int g = 0; g < G; ++g) {
-                float d = 0.f;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) d = fmaf(qf[g][i], kf[i], d);
-                s[u][g] = d;
+            for (int i = 0; i < 2; ++i) {
+                const bool ok = (j0 + u * 8 + 2 * c + i) < s1;
+                s[u][i] = ok ? s[u][i] * scale_log2 : -INFINITY;
+                mt = fmaxf(mt, s[u][i]);
             }
-        }
-        // sum the partial dot products over the LPK lanes of a row (all of them get the total)
+        mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 1));
+        mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 2));
+        const float m_new = fmaxf(m_run, mt);
+        const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
+        float alpha = exp2f(m_run - m_ref);  // 0 on the first block (m_run = -inf)
+        m_run = m_new;
+        float p[2][2];
 #pragma unroll
-        for (int o = 1; o < LPK; o <<= 1)
+        for (int u = 0; u < 2; ++u)
 #pragma unroll
-            for (int u = 0; u < kU; ++u)
-#pragma unroll
-                for (int g = 0; g < G; ++g) s[u][g] += __shfl_xor_sync(0xffffffffu, s[u][g], o);
+            for (int i = 0; i < 2; ++i) p[u][i] = exp2f(s[u][i] - m_ref);  // masked key: exactly 0
+        if (g >= G) { alpha = 1.f; p[0][0] = p[0][1] = p[1][0] = p[1][1] = 0.f; }
+        l_run = l_run * alpha + (p[0][0] + p[0][1]) + (p[1][0] + p[1][1]);
 
-        float alpha[G], m_ref[G];
+        // rescale the accumulators: this lane holds output columns (heads) 2c and 2c+1
+        const float a_even = __shfl_sync(0xffffffffu, alpha, (2 * c) * 4);
+        const float a_odd = __shfl_sync(0xffffffffu, alpha, (2 * c + 1) * 4);
+        if (__any_sync(0xffffffffu, alpha != 1.f)) {
 #pragma unroll
-        for (int g = 0; g < G; ++g) {
-            float mt = -INFINITY;
+            for (int hb = 0; hb < NHB; ++hb)
 #pragma unroll
-            for (int u = 0; u < kU; ++u) {
-                const bool ok = (j0 + u * KPL + sub) < s1;
-                s[u][g] = ok ? s[u][g] : -INFINITY;
-                mt = fmaxf(mt, s[u][g]);
-            }
-#pragma unroll
-            for (int o = LPK; o < 32; o <<= 1) mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, o));
-            const float m_new = fmaxf(m_run[g], mt);
-            m_ref[g] = (m_new == -INFINITY) ? 0.f : m_new;
-            alpha[g] = exp2f(m_run[g] - m_ref[g]);
-            m_run[g] = m_new;
+                for (int t = 0; t < 4; ++t) {
+                    acc[hb][t][0] *= a_even; acc[hb][t][1] *= a_odd;
+                    acc[hb][t][2] *= a_even; acc[hb][t][3] *= a_odd;
+                }
         }
+
+        // P^T as the B operand: k-slots (2c, 2c+1) = keys 2c, 2c+1; k-slots (2c+8, 2c+9) = keys 2c+8, 2c+9
+        const uint32_t pb0 = pack_bf16x2(p[0][0], p[0][1]);
+        const uint32_t pb1 = pack_bf16x2(p[1][0], p[1][1]);
 #pragma unroll
-        for (int g = 0; g < G; ++g) {
-            l_run[g] *= alpha[g];
+        for (int hb = 0; hb < NHB; ++hb) {
+            // interleave two V rows: word w of a row holds dims 2w, 2w+1 -> (row_a[d], row_b[d]) pairs
+            const uint32_t va[4] = {vr[0][hb].x, vr[0][hb].y, vr[0][hb].z, vr[0][hb].w};
+            const uint32_t vb[4] = {vr[1][hb].x, vr[1][hb].y, vr[1][hb].z, vr[1][hb].w};
+            const uint32_t vc_[4] = {vr[2][hb].x, vr[2][hb].y, vr[2][hb].z, vr[2][hb].w};
+            const uint32_t vd[4] = {vr[3][hb].x, vr[3][hb].y, vr[3][hb].z, vr[3][hb].w};
+            uint32_t ab[8], cd[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) acc[g][i] *= alpha[g];
-        }
-#pragma unroll
-        for (int u = 0; u < kU; ++u) {
-            float vf[8];
-            unpack8(vr[u], vf);
-#pragma unroll
-            for (int g = 0; g < G; ++g) {
-                const float p = exp2f(s[u][g] - m_ref[g]);  // masked row: exactly 0
-                l_run[g] += p;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) acc[g][i] = fmaf(p, vf[i], acc[g][i]);
+            for (int w = 0; w < 4; ++w) {
+                ab[2 * w] = __byte_perm(va[w], vb[w], 0x5410);
+                ab[2 * w + 1] = __byte_perm(va[w], vb[w], 0x7632);
+                cd[2 * w] = __byte_perm(vc_[w], vd[w], 0x5410);
+                cd[2 * w + 1] = __byte_perm(vc_[w], vd[w], 0x7632);
             }
+            // MMA t: row g = dim hb*64 + g*8 + t, row g+8 = dim hb*64 + g*8 + 4 + t
+#pragma unroll
+            for (int t = 0; t < 4; ++t) mma16816(acc[hb][t], ab[t], ab[4 + t], cd[t], cd[4 + t], pb0, pb1);
         }
     }
 
-    // merge the KPL row-groups of the warp (they share m_run), then the warps via shared memory
+    // the 4 lanes of a head hold partial sums over their own keys
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+    if (g < G && c == 0) { sm_m[warp][g] = m_run; sm_l[warp][g] = l_run; }
 #pragma unroll
-    for (int o = LPK; o < 32; o <<= 1) {
+    for (int hb = 0; hb < NHB; ++hb)
 #pragma unroll
-        for (int g = 0; g < G; ++g) {
-            l_run[g] += __shfl_xor_sync(0xffffffffu, l_run[g], o);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) acc[g][i] += __shfl_xor_sync(0xffffffffu, acc[g][i], o);
+        for (int t = 0; t < 4; ++t) {
+            const int d0 = hb * 64 + g * 8 + t;
+            if (2 * c < G) { sm_acc[warp][2 * c][d0] = acc[hb][t][0]; sm_acc[warp][2 * c][d0 + 4] = acc[hb][t][2]; }
+            if (2 * c + 1 < G) { sm_acc[warp][2 * c + 1][d0] = acc[hb][t][1]; sm_acc[warp][2 * c + 1][d0 + 4] = acc[hb][t][3]; }
         }
-    }
-    if (sub == 0) {
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-            if (chunk == 0) { sm_m[warp][g] = m_run[g]; sm_l[warp][g] = l_run[g]; }
-#pragma unroll
-            for (int i = 0; i < 8; ++i) sm_acc[warp][g][chunk * 8 + i] = acc[g][i];
-        }
-    }
     __syncthreads();
     for (int idx = tid; idx < G * D; idx += kThreads) {
-        const int g = idx / D, d = idx % D;
+        const int hg = idx / D, d = idx % D;
         float M = -INFINITY;
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) M = fmaxf(M, sm_m[w][g]);
+        for (int w = 0; w < kWarps; ++w) M = fmaxf(M, sm_m[w][hg]);
         const float Mref = (M == -INFINITY) ? 0.f : M;
         float L = 0.f, O = 0.f;
 #pragma unroll
         for (int w = 0; w < kWarps; ++w) {
-            const float wgt = exp2f(sm_m[w][g] - Mref);
-            L = fmaf(wgt, sm_l[w][g], L);
-            O = fmaf(wgt, sm_acc[w][g][d], O);
+            const float wgt = exp2f(sm_m[w][hg] - Mref);
+            L = fmaf(wgt, sm_l[w][hg], L);
+            O = fmaf(wgt, sm_acc[w][hg][d], O);
         }
-        const size_t slot = ((size_t)b * Hq + kvh * G + g) * num_splits + split;
+        const size_t slot = ((size_t)b * Hq + kvh * G + hg) * num_splits + split;
         ws_o[slot * D + d] = O;
         if (d == 0) { ws_ml[slot * 2] = M; ws_ml[slot * 2 + 1] = L; }
     }

@@ -3,13 +3,19 @@
 // ranges; each range yields a partial (running max m, running sum l, unnormalised output)
 // and the combine step merges the partials:
 //     M = max_s m_s,   L = sum_s 2^(m_s - M) l_s,   out = sum_s 2^(m_s - M) O_s / L
-// (scores are kept in log2 units: they are pre-multiplied by scale * log2(e)).
+// (scores are kept in log2 units: they are multiplied by scale * log2(e)).
 //
-// The kernel is bound by streaming K and V from HBM: every lane issues 128-bit loads straight
-// into MMA fragments (no shared-memory staging), K and V loads of a block of rows are issued
-// together, and the G = Hq / Hkv query heads that share a KV head are processed by the same CTA
-// so that each cached row is read exactly once.  The dot products run on warp-level tensor-core
-// MMAs (m16n8k16) only because fp32 FMAs with shuffle reductions were bound by instruction issue.
+// The work is bound by streaming K and V from HBM once, and HBM only delivers its bandwidth
+// with a deep queue of requests (pure streaming with 48 KB in flight per SM reaches 4.2 TB/s on
+// this part, with 250 KB 5.8 TB/s).  So the split kernel is persistent and every warp is an
+// independent worker: it owns whole (batch, kv head, split) items, keeps a private ring of
+// 16-row blocks in shared memory filled by 16-byte asynchronous copies that run ahead across
+// item boundaries (8 warps x 24 KB in flight per SM, 512 contiguous bytes per instruction,
+// zero-fill instead of reads past the end of a split), and writes its partial straight from
+// registers.  No warp ever waits for another one.  The G = Hq / Hkv query heads that share a KV
+// head are processed together, so every cached row is read exactly once.  The dot products run
+// on warp-level tensor-core MMAs (m16n8k16) with fragments read from the swizzled ring; fp32 FMAs
+// with shuffle reductions were bound by instruction issue.
 #include <cuda_bf16.h>
 
 #include <mutex>
@@ -19,17 +25,31 @@
 namespace forge {
 namespace {
 
-constexpr int kWarps = 4;
+constexpr int kWarps = 8;
 constexpr int kThreads = kWarps * 32;
-constexpr int kBlockKeys = 16;  // cached rows per warp iteration
+constexpr int kBlockKeys = 16;             // cached rows per ring stage
+constexpr int kWarpRingBytes = 24 * 1024;  // per warp
 
-__device__ __forceinline__ uint4 ld_stream(const void* p) {
+// 16-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros and reads nothing.
+__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gsrc, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_dst), "l"(gsrc), "r"(src_bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 r;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
-                 : "l"(p));
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
     return r;
 }
+// Position of 16-byte chunk k of cached row r inside the row's shared-memory image.  Bits 1-2 of the
+// chunk index are XORed with a function of the row so that both fragment reads are free of bank
+// conflicts: per quarter-warp, K reads touch rows (r, r+1) x 4 consecutive chunks and V reads touch
+// rows (r, r+2, r+4, r+6) x 2 consecutive chunks.
+__device__ __forceinline__ int swz(int r, int k) { return k ^ ((((r >> 1) & 3) << 1) ^ ((r & 1) << 2)); }
 
 // D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col).  Lane = (g = lane / 4, c = lane % 4):
 //   A: a0 = (row g, k 2c..2c+1)  a1 = (row g+8, k 2c..)  a2 = (row g, k 2c+8..)  a3 = (row g+8, k 2c+8..)
@@ -48,177 +68,261 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// grid = (num_splits, Hkv, B).  Each warp walks its share of the split in blocks of 16 cached rows:
+// One (batch, kv head, split) work item and its range of cached rows.
+struct Item {
+    int b, kvh, split, s0, s1;
+};
+__device__ __forceinline__ Item make_item(int idx, const int32_t* lens, int Hkv, int Smax, int num_splits) {
+    Item it;
+    it.split = idx % num_splits;
+    const int bk = idx / num_splits;
+    it.kvh = bk % Hkv;
+    it.b = bk / Hkv;
+    const int len = min(max(lens[it.b], 0), Smax);
+    const int per = (len + num_splits - 1) / num_splits;
+    it.s0 = it.split * per;
+    it.s1 = min(it.s0 + per, len);
+    if (it.s1 < it.s0) it.s1 = it.s0;
+    return it;
+}
+
+// Worker w (= warp) takes items w, w + workers, ...; consecutive items go to different SMs.
 //   S[head, key]  = Q K^T   as m16n8k16 with A = Q (rows = the G heads, padded with zero rows) and
-//                   B = K rows straight from global memory (the contraction runs over the head
-//                   dimension in whatever order the 16-byte loads deliver it, the same for Q and K);
+//                   B = K rows (the contraction runs over the head dimension in whatever order the
+//                   16-byte chunks deliver it, the same for Q and K);
 //   online softmax on the accumulator fragment (lane (g, c) owns head g, keys 2c, 2c+1 of each 8);
 //   O^T[dim, head] += V^T P^T  with A = pairs of V rows interleaved with byte permutes and B = the
 //                   probabilities exactly where the first MMA left them.
-// The arithmetic is a few instructions per cached row, so the kernel is bound by the HBM stream.
 template <int D, int G>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, 1)
 decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ kc,
                     const __nv_bfloat16* __restrict__ vc, const int32_t* __restrict__ lens,
                     float* __restrict__ ws_o, float* __restrict__ ws_ml,
-                    int Hq, int Hkv, int Smax, int num_splits, float scale_log2) {
+                    int B, int Hq, int Hkv, int Smax, int num_splits, float scale_log2) {
     constexpr int NKB = D / 32;  // 32-dim blocks of the head dimension (two k16 MMAs each)
     constexpr int NHB = D / 64;  // 64-dim blocks of the output (four 16-dim MMAs each)
+    constexpr int kRowBytes = D * 2;
+    constexpr int kCPR = kRowBytes / 16;                  // 16-byte chunks per row
+    constexpr int kTensorBytes = kBlockKeys * kRowBytes;  // 16 rows of K (or of V)
+    constexpr int kStageBytes = 2 * kTensorBytes;
+    constexpr int kStages = kWarpRingBytes / kStageBytes;  // 3 for D = 128, 6 for D = 64
+    static_assert(kStages >= 2, "ring too small");
 
-    const int split = blockIdx.x, kvh = blockIdx.y, b = blockIdx.z;
+    extern __shared__ __align__(128) uint8_t ring_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, c = lane & 3;
+    const uint32_t ring = static_cast<uint32_t>(__cvta_generic_to_shared(ring_raw)) + warp * kWarpRingBytes;
 
-    const int len = min(max(lens[b], 0), Smax);
-    const int per = (len + num_splits - 1) / num_splits;
-    const int s0 = split * per;
-    const int s1 = min(s0 + per, len);
+    const int num_items = B * Hkv * num_splits;
+    const int workers = gridDim.x * kWarps;
+    const int worker = warp * gridDim.x + blockIdx.x;
 
-    __shared__ float sm_m[kWarps][G];
-    __shared__ float sm_l[kWarps][G];
-    __shared__ __align__(16) float sm_acc[kWarps][G][D];
-
-    // Q fragment: head g (zero rows for g >= G), 8 dims at c*8 of every 32-dim block
-    uint32_t qr[NKB][4];
+    // ---- prefetch cursor: runs kStages - 1 blocks ahead of the compute, across item boundaries
+    int p_idx = worker, p_j0 = 0, p_s1 = 0;
+    const __nv_bfloat16 *p_k = kc, *p_v = vc;
+    int p_n = 0;  // blocks issued
+    auto p_open = [&]() {  // position the cursor on the first block of the next non-empty item
+        while (p_idx < num_items) {
+            const Item it = make_item(p_idx, lens, Hkv, Smax, num_splits);
+            if (it.s1 > it.s0) {
+                p_j0 = it.s0;
+                p_s1 = it.s1;
+                p_k = kc + ((size_t)it.b * Hkv + it.kvh) * (size_t)Smax * D;
+                p_v = vc + ((size_t)it.b * Hkv + it.kvh) * (size_t)Smax * D;
+                return;
+            }
+            p_idx += workers;
+        }
+    };
+    auto issue = [&]() {  // lane l of copy i moves chunk i*32 + l of the block's 16 rows
+        if (p_idx < num_items) {
+            const uint32_t dst = ring + (p_n % kStages) * kStageBytes;
 #pragma unroll
-    for (int kb = 0; kb < NKB; ++kb) {
-        uint4 raw = make_uint4(0, 0, 0, 0);
-        if (g < G) raw = *reinterpret_cast<const uint4*>(q + ((size_t)b * Hq + kvh * G + g) * D + kb * 32 + c * 8);
-        qr[kb][0] = raw.x; qr[kb][1] = raw.y; qr[kb][2] = raw.z; qr[kb][3] = raw.w;
+            for (int i = 0; i < kTensorBytes / 512; ++i) {
+                const int id = i * 32 + lane, r = id / kCPR, k = id % kCPR;
+                const uint32_t ok = (p_j0 + r < p_s1) ? 16u : 0u;  // rows past the split: zeros, nothing read
+                const size_t goff = (size_t)(p_j0 + (ok ? r : 0)) * D + k * 8;
+                const uint32_t soff = r * kRowBytes + swz(r, k) * 16;
+                cp_async16(dst + soff, p_k + goff, ok);
+                cp_async16(dst + kTensorBytes + soff, p_v + goff, ok);
+            }
+            ++p_n;
+            p_j0 += kBlockKeys;
+            if (p_j0 >= p_s1) { p_idx += workers; p_open(); }
+        }
+        cp_async_commit();  // an empty group keeps the group count uniform
+    };
+    p_open();
+#pragma unroll
+    for (int i = 0; i < kStages - 1; ++i) issue();
+
+    // Q fragment of an item: head g (zero rows for g >= G), 8 dims at c*8 of every 32-dim block
+    auto load_q = [&](const Item& it, uint32_t (&qr)[NKB][4]) {
+#pragma unroll
+        for (int kb = 0; kb < NKB; ++kb) {
+            uint4 raw = make_uint4(0, 0, 0, 0);
+            if (g < G)
+                raw = *reinterpret_cast<const uint4*>(q + ((size_t)it.b * Hq + it.kvh * G + g) * D + kb * 32 + c * 8);
+            qr[kb][0] = raw.x; qr[kb][1] = raw.y; qr[kb][2] = raw.z; qr[kb][3] = raw.w;
+        }
+    };
+
+    Item nxt = {0, 0, 0, 0, 0};
+    uint32_t qn[NKB][4];
+    if (worker < num_items) {
+        nxt = make_item(worker, lens, Hkv, Smax, num_splits);
+        load_q(nxt, qn);
     }
-
-    float m_run = -INFINITY, l_run = 0.f;  // of head g (lanes with g >= G carry dummies)
-    float acc[NHB][4][4];                  // O^T fragments: [64-dim block][16-dim MMA][d0..d3]
+    int n = 0;  // blocks consumed
+    for (int idx = worker; idx < num_items; idx += workers) {
+        const Item it = nxt;
+        uint32_t qr[NKB][4];
 #pragma unroll
-    for (int hb = 0; hb < NHB; ++hb)
+        for (int kb = 0; kb < NKB; ++kb)
 #pragma unroll
-        for (int t = 0; t < 4; ++t)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) acc[hb][t][i] = 0.f;
-
-    const __nv_bfloat16* kbase = kc + ((size_t)b * Hkv + kvh) * (size_t)Smax * D;
-    const __nv_bfloat16* vbase = vc + ((size_t)b * Hkv + kvh) * (size_t)Smax * D;
-
-    for (int j0 = s0 + warp * kBlockKeys; j0 < s1; j0 += kWarps * kBlockKeys) {
-        // K: rows j0 + u*8 + g, 16 bytes at dims kb*32 + c*8.  V: rows j0 + {2c, 2c+1, 2c+8, 2c+9},
-        // 16 bytes at dims hb*64 + g*8.  Rows at or beyond s1 are not read (zeros).
-        uint4 kr[2][NKB], vr[4][NHB];
-#pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int j = j0 + u * 8 + g;
-#pragma unroll
-            for (int kb = 0; kb < NKB; ++kb)
-                kr[u][kb] = (j < s1) ? ld_stream(kbase + (size_t)j * D + kb * 32 + c * 8) : make_uint4(0, 0, 0, 0);
-        }
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            const int j = j0 + 2 * c + (r & 1) + (r >> 1) * 8;
-#pragma unroll
-            for (int hb = 0; hb < NHB; ++hb)
-                vr[r][hb] = (j < s1) ? ld_stream(vbase + (size_t)j * D + hb * 64 + g * 8) : make_uint4(0, 0, 0, 0);
+            for (int i = 0; i < 4; ++i) qr[kb][i] = qn[kb][i];
+        if (idx + workers < num_items) {  // fetch the next item's range and Q rows early
+            nxt = make_item(idx + workers, lens, Hkv, Smax, num_splits);
+            load_q(nxt, qn);
         }
 
-        // scores: s[u][0..1] = head g, keys j0 + u*8 + 2c + {0, 1}  (s[u][2..3] belong to zero rows)
-        float s[2][4];
+        float m_run = -INFINITY, l_run = 0.f;  // of head g (lanes with g >= G carry dummies)
+        float acc[NHB][4][4];                  // O^T fragments: [64-dim block][16-dim MMA][d0..d3]
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            s[u][0] = s[u][1] = s[u][2] = s[u][3] = 0.f;
+        for (int hb = 0; hb < NHB; ++hb)
 #pragma unroll
-            for (int kb = 0; kb < NKB; ++kb) {
-                mma16816(s[u], qr[kb][0], 0u, qr[kb][1], 0u, kr[u][kb].x, kr[u][kb].y);
-                mma16816(s[u], qr[kb][2], 0u, qr[kb][3], 0u, kr[u][kb].z, kr[u][kb].w);
+            for (int t = 0; t < 4; ++t)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[hb][t][i] = 0.f;
+
+        for (int j0 = it.s0; j0 < it.s1; j0 += kBlockKeys, ++n) {
+            issue();                       // refills the stage that was read in the previous iteration
+            cp_async_wait<kStages - 1>();  // this lane's copies of block n have landed
+            __syncwarp();                  // ... and everyone else's
+            const uint32_t sa = ring + (n % kStages) * kStageBytes;
+            // K fragment: rows u*8 + g, chunk kb*4 + c.  V fragment: rows {2c, 2c+1, 2c+8, 2c+9}, chunk hb*8 + g.
+            uint4 kr[2][NKB], vr[4][NHB];
+#pragma unroll
+            for (int u = 0; u < 2; ++u)
+#pragma unroll
+                for (int kb = 0; kb < NKB; ++kb)
+                    kr[u][kb] = lds128(sa + (u * 8 + g) * kRowBytes + swz(u * 8 + g, kb * 4 + c) * 16);
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const int row = 2 * c + (r & 1) + (r >> 1) * 8;
+#pragma unroll
+                for (int hb = 0; hb < NHB; ++hb)
+                    vr[r][hb] = lds128(sa + kTensorBytes + row * kRowBytes + swz(row, hb * 8 + g) * 16);
+            }
+            __syncwarp();  // all fragment reads done before this stage is refilled
+
+            // scores: s[u][0..1] = head g, keys j0 + u*8 + 2c + {0, 1}  (s[u][2..3] belong to zero rows)
+            float s[2][4];
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                // two accumulation chains per key group (shorter dependent MMA sequences)
+                float s2[4] = {0.f, 0.f, 0.f, 0.f};
+                s[u][0] = s[u][1] = s[u][2] = s[u][3] = 0.f;
+#pragma unroll
+                for (int kb = 0; kb < NKB; ++kb) {
+                    mma16816(s[u], qr[kb][0], 0u, qr[kb][1], 0u, kr[u][kb].x, kr[u][kb].y);
+                    mma16816(s2, qr[kb][2], 0u, qr[kb][3], 0u, kr[u][kb].z, kr[u][kb].w);
+                }
+                s[u][0] += s2[0];
+                s[u][1] += s2[1];
+            }
+            float mt = -INFINITY;
+#pragma unroll
+            for (int u = 0; u < 2; ++u)
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const bool ok = (j0 + u * 8 + 2 * c + i) < it.s1;
+                    s[u][i] = ok ? s[u][i] * scale_log2 : -INFINITY;
+                    mt = fmaxf(mt, s[u][i]);
+                }
+            mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 1));
+            mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 2));
+            const float m_new = fmaxf(m_run, mt);
+            const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
+            float alpha = exp2f(m_run - m_ref);  // 0 on the first block (m_run = -inf)
+            m_run = m_new;
+            float p[2][2];
+#pragma unroll
+            for (int u = 0; u < 2; ++u)
+#pragma unroll
+                for (int i = 0; i < 2; ++i) p[u][i] = exp2f(s[u][i] - m_ref);  // masked key: exactly 0
+            if (g >= G) { alpha = 1.f; p[0][0] = p[0][1] = p[1][0] = p[1][1] = 0.f; }
+            l_run = l_run * alpha + (p[0][0] + p[0][1]) + (p[1][0] + p[1][1]);
+
+            // rescale the accumulators: this lane holds output columns (heads) 2c and 2c+1
+            const float a_even = __shfl_sync(0xffffffffu, alpha, (2 * c) * 4);
+            const float a_odd = __shfl_sync(0xffffffffu, alpha, (2 * c + 1) * 4);
+            if (__any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll
+                for (int hb = 0; hb < NHB; ++hb)
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        acc[hb][t][0] *= a_even; acc[hb][t][1] *= a_odd;
+                        acc[hb][t][2] *= a_even; acc[hb][t][3] *= a_odd;
+                    }
+            }
+
+            // P^T as the B operand: k-slots (2c, 2c+1) = keys 2c, 2c+1; (2c+8, 2c+9) = keys 2c+8, 2c+9
+            const uint32_t pb0 = pack_bf16x2(p[0][0], p[0][1]);
+            const uint32_t pb1 = pack_bf16x2(p[1][0], p[1][1]);
+#pragma unroll
+            for (int hb = 0; hb < NHB; ++hb) {
+                // interleave two V rows: word w of a row holds dims 2w, 2w+1 -> (row_a[d], row_b[d]) pairs
+                const uint32_t va[4] = {vr[0][hb].x, vr[0][hb].y, vr[0][hb].z, vr[0][hb].w};
+                const uint32_t vb[4] = {vr[1][hb].x, vr[1][hb].y, vr[1][hb].z, vr[1][hb].w};
+                const uint32_t vc_[4] = {vr[2][hb].x, vr[2][hb].y, vr[2][hb].z, vr[2][hb].w};
+                const uint32_t vd[4] = {vr[3][hb].x, vr[3][hb].y, vr[3][hb].z, vr[3][hb].w};
+                uint32_t ab[8], cd[8];
+#pragma unroll
+                for (int w = 0; w < 4; ++w) {
+                    ab[2 * w] = __byte_perm(va[w], vb[w], 0x5410);
+                    ab[2 * w + 1] = __byte_perm(va[w], vb[w], 0x7632);
+                    cd[2 * w] = __byte_perm(vc_[w], vd[w], 0x5410);
+                    cd[2 * w + 1] = __byte_perm(vc_[w], vd[w], 0x7632);
+                }
+                // MMA t: row g = dim hb*64 + g*8 + t, row g+8 = dim hb*64 + g*8 + 4 + t
+#pragma unroll
+                for (int t = 0; t < 4; ++t) mma16816(acc[hb][t], ab[t], ab[4 + t], cd[t], cd[4 + t], pb0, pb1);
             }
         }
-        float mt = -INFINITY;
-#pragma unroll
-        for (int u = 0; u < 2; ++u)
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-                const bool ok = (j0 + u * 8 + 2 * c + i) < s1;
-                s[u][i] = ok ? s[u][i] * scale_log2 : -INFINITY;
-                mt = fmaxf(mt, s[u][i]);
-            }
-        mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 1));
-        mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 2));
-        const float m_new = fmaxf(m_run, mt);
-        const float m_ref = (m_new == -INFINITY) ? 0.f : m_new;
-        float alpha = exp2f(m_run - m_ref);  // 0 on the first block (m_run = -inf)
-        m_run = m_new;
-        float p[2][2];
-#pragma unroll
-        for (int u = 0; u < 2; ++u)
-#pragma unroll
-            for (int i = 0; i < 2; ++i) p[u][i] = exp2f(s[u][i] - m_ref);  // masked key: exactly 0
-        if (g >= G) { alpha = 1.f; p[0][0] = p[0][1] = p[1][0] = p[1][1] = 0.f; }
-        l_run = l_run * alpha + (p[0][0] + p[0][1]) + (p[1][0] + p[1][1]);
 
-        // rescale the accumulators: this lane holds output columns (heads) 2c and 2c+1
-        const float a_even = __shfl_sync(0xffffffffu, alpha, (2 * c) * 4);
-        const float a_odd = __shfl_sync(0xffffffffu, alpha, (2 * c + 1) * 4);
-        if (__any_sync(0xffffffffu, alpha != 1.f)) {
+        // ---- this warp's partial is the item's partial: write it out from the fragments
+        l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+        l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+        const size_t slot0 = ((size_t)it.b * Hq + it.kvh * G) * num_splits + it.split;  // head 0 of the group
+        if (g < G && c == 0) {
+            ws_ml[(slot0 + (size_t)g * num_splits) * 2] = m_run;
+            ws_ml[(slot0 + (size_t)g * num_splits) * 2 + 1] = l_run;
+        }
+        if (it.s1 > it.s0) {  // an empty split has m = -inf and its output slot is never read
 #pragma unroll
             for (int hb = 0; hb < NHB; ++hb)
 #pragma unroll
                 for (int t = 0; t < 4; ++t) {
-                    acc[hb][t][0] *= a_even; acc[hb][t][1] *= a_odd;
-                    acc[hb][t][2] *= a_even; acc[hb][t][3] *= a_odd;
+                    const int d0 = hb * 64 + g * 8 + t;
+                    if (2 * c < G) {
+                        float* o = ws_o + (slot0 + (size_t)(2 * c) * num_splits) * D;
+                        o[d0] = acc[hb][t][0];
+                        o[d0 + 4] = acc[hb][t][2];
+                    }
+                    if (2 * c + 1 < G) {
+                        float* o = ws_o + (slot0 + (size_t)(2 * c + 1) * num_splits) * D;
+                        o[d0] = acc[hb][t][1];
+                        o[d0 + 4] = acc[hb][t][3];
+                    }
                 }
         }
-
-        // P^T as the B operand: k-slots (2c, 2c+1) = keys 2c, 2c+1; k-slots (2c+8, 2c+9) = keys 2c+8, 2c+9
-        const uint32_t pb0 = pack_bf16x2(p[0][0], p[0][1]);
-        const uint32_t pb1 = pack_bf16x2(p[1][0], p[1][1]);
-#pragma unroll
-        for (int hb = 0; hb < NHB; ++hb) {
-            // interleave two V rows: word w of a row holds dims 2w, 2w+1 -> (row_a[d], row_b[d]) pairs
-            const uint32_t va[4] = {vr[0][hb].x, vr[0][hb].y, vr[0][hb].z, vr[0][hb].w};
-            const uint32_t vb[4] = {vr[1][hb].x, vr[1][hb].y, vr[1][hb].z, vr[1][hb].w};
-            const uint32_t vc_[4] = {vr[2][hb].x, vr[2][hb].y, vr[2][hb].z, vr[2][hb].w};
-            const uint32_t vd[4] = {vr[3][hb].x, vr[3][hb].y, vr[3][hb].z, vr[3][hb].w};
-            uint32_t ab[8], cd[8];
-#pragma unroll
-            for (int w = 0; w < 4; ++w) {
-                ab[2 * w] = __byte_perm(va[w], vb[w], 0x5410);
-                ab[2 * w + 1] = __byte_perm(va[w], vb[w], 0x7632);
-                cd[2 * w] = __byte_perm(vc_[w], vd[w], 0x5410);
-                cd[2 * w + 1] = __byte_perm(vc_[w], vd[w], 0x7632);
-            }
-            // MMA t: row g = dim hb*64 + g*8 + t, row g+8 = dim hb*64 + g*8 + 4 + t
-#pragma unroll
-            for (int t = 0; t < 4; ++t) mma16816(acc[hb][t], ab[t], ab[4 + t], cd[t], cd[4 + t], pb0, pb1);
-        }
     }
+    cp_async_wait<0>();
 
-    // the 4 lanes of a head hold partial sums over their own keys
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
-    l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-    if (g < G && c == 0) { sm_m[warp][g] = m_run; sm_l[warp][g] = l_run; }
-#pragma unroll
-    for (int hb = 0; hb < NHB; ++hb)
-#pragma unroll
-        for (int t = 0; t < 4; ++t) {
-            const int d0 = hb * 64 + g * 8 + t;
-            if (2 * c < G) { sm_acc[warp][2 * c][d0] = acc[hb][t][0]; sm_acc[warp][2 * c][d0 + 4] = acc[hb][t][2]; }
-            if (2 * c + 1 < G) { sm_acc[warp][2 * c + 1][d0] = acc[hb][t][1]; sm_acc[warp][2 * c + 1][d0 + 4] = acc[hb][t][3]; }
-        }
-    __syncthreads();
-    for (int idx = tid; idx < G * D; idx += kThreads) {
-        const int hg = idx / D, d = idx % D;
-        float M = -INFINITY;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) M = fmaxf(M, sm_m[w][hg]);
-        const float Mref = (M == -INFINITY) ? 0.f : M;
-        float L = 0.f, O = 0.f;
-#pragma unroll
-        for (int w = 0; w < kWarps; ++w) {
-            const float wgt = exp2f(sm_m[w][hg] - Mref);
-            L = fmaf(wgt, sm_l[w][hg], L);
-            O = fmaf(wgt, sm_acc[w][hg][d], O);
-        }
-        const size_t slot = ((size_t)b * Hq + kvh * G + hg) * num_splits + split;
-        ws_o[slot * D + d] = O;
-        if (d == 0) { ws_ml[slot * 2] = M; ws_ml[slot * 2 + 1] = L; }
-    }
+    // Let the combine kernel (launched with programmatic stream serialisation) be scheduled once every
+    // CTA of this grid got here; it still waits for this grid's completion before it reads.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
 // grid = B * Hq, block = D threads: merges the num_splits partials of one (batch, head).
@@ -229,40 +333,54 @@ decode_combine_kernel(const float* __restrict__ ws_o, const float* __restrict__ 
     const size_t bh = blockIdx.x;
     const int d = threadIdx.x;
     const float* ml = ws_ml + bh * num_splits * 2;
+    // the split kernel's writes are visible only after this returns
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     float M = -INFINITY;
+#pragma unroll 8
     for (int s = 0; s < num_splits; ++s) M = fmaxf(M, ml[2 * s]);
     float L = 0.f, O = 0.f;
     if (M != -INFINITY) {
+#pragma unroll 8
         for (int s = 0; s < num_splits; ++s) {
             const float ms = ml[2 * s];
-            if (ms == -INFINITY) continue;  // empty split: its output slot was never written
+            // empty split: m = -inf gives weight 0; its output slot was never written, so do not read it
             const float wgt = exp2f(ms - M);
+            const float o = (ms == -INFINITY) ? 0.f : ws_o[(bh * num_splits + s) * D + d];
             L = fmaf(wgt, ml[2 * s + 1], L);
-            O = fmaf(wgt, ws_o[(bh * num_splits + s) * D + d], O);
+            O = fmaf(wgt, o, O);
         }
     }
     out[bh * D + d] = __float2bfloat16_rn(L > 0.f ? O / L : 0.f);
 }
 
 template <int D, int G>
-void launch_split(const void* q, const void* kc, const void* vc, const int32_t* lens, float* ws_o, float* ws_ml,
-                  int B, int Hq, int Hkv, int Smax, int num_splits, float scale_log2, cudaStream_t s) {
-    decode_split_kernel<D, G><<<dim3(num_splits, Hkv, B), kThreads, 0, s>>>(
+int launch_split(const void* q, const void* kc, const void* vc, const int32_t* lens, float* ws_o, float* ws_ml,
+                 int B, int Hq, int Hkv, int Smax, int num_splits, float scale_log2, cudaStream_t s) {
+    constexpr int kSmem = kWarps * kWarpRingBytes;
+    auto kernel = decode_split_kernel<D, G>;
+    FORGE_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem));
+    int dev = 0, sms = 0;
+    FORGE_CUDA_TRY(cudaGetDevice(&dev));
+    FORGE_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const long long items = (long long)B * Hkv * num_splits;
+    const long long ctas = (items + kWarps - 1) / kWarps;
+    const int grid = ctas < sms ? (int)ctas : sms;
+    kernel<<<grid, kThreads, kSmem, s>>>(
         static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(kc),
-        static_cast<const __nv_bfloat16*>(vc), lens, ws_o, ws_ml, Hq, Hkv, Smax, num_splits, scale_log2);
+        static_cast<const __nv_bfloat16*>(vc), lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2);
+    return FORGE_OK;
 }
 
 template <int D>
 int dispatch_g(int G, const void* q, const void* kc, const void* vc, const int32_t* lens, float* ws_o,
                float* ws_ml, int B, int Hq, int Hkv, int Smax, int num_splits, float scale_log2, cudaStream_t s) {
     switch (G) {
-        case 1: launch_split<D, 1>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s); break;
-        case 2: launch_split<D, 2>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s); break;
-        case 4: launch_split<D, 4>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s); break;
-        case 8: launch_split<D, 8>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s); break;
+        case 1: return launch_split<D, 1>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
+        case 2: return launch_split<D, 2>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
+        case 4: return launch_split<D, 4>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
+        case 8: return launch_split<D, 8>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
         default: return FORGE_ERR_UNSUPPORTED;
     }
-    return FORGE_OK;
 }
 
 }  // namespace
@@ -298,10 +416,24 @@ extern "C" int forge_attn_decode_splitkv(const void* q, const void* k_cache, con
     if (st != FORGE_OK) return st;
     st = finish_launch(1);
     if (st != FORGE_OK) return st;
+    // The combine kernel is launched with programmatic stream serialisation: its CTAs may be placed
+    // while the split kernel drains, and block in griddepcontrol.wait until that grid has completed.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(B * Hq, 1, 1);
+    cfg.blockDim = dim3(D, 1, 1);
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const float* cws_o = ws_o;
+    const float* cws_ml = ws_ml;
+    __nv_bfloat16* ob = static_cast<__nv_bfloat16*>(out);
     if (D == 64)
-        decode_combine_kernel<64><<<B * Hq, 64, 0, s>>>(ws_o, ws_ml, static_cast<__nv_bfloat16*>(out), num_splits);
+        FORGE_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_combine_kernel<64>, cws_o, cws_ml, ob, num_splits));
     else
-        decode_combine_kernel<128><<<B * Hq, 128, 0, s>>>(ws_o, ws_ml, static_cast<__nv_bfloat16*>(out), num_splits);
+        FORGE_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_combine_kernel<128>, cws_o, cws_ml, ob, num_splits));
     return finish_launch(1);
 }
 

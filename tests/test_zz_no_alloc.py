@@ -31,8 +31,10 @@ def test_matches_the_workspace_entry_point_on_two_calls_in_a_row():
     lib = binding.load()
     stream = torch.cuda.current_stream().cuda_stream
     cases = [
-        wl.decode_workload("first", 61, 16, 32, 8, 1024, 128, 16, 128 ** -0.5, (300, 1024)),  # 4.1 MiB of partials
-        wl.decode_workload("second", 62, 3, 8, 2, 700, 64, 5, 0.125, (1, 700)),               # smaller, other shape
+        # 24 and 20 splits: more than a thread-block cluster holds, so the partials really go through
+        # the fixed array (6.1 MiB of it in the first call, a small corner of it in the second)
+        wl.decode_workload("first", 61, 16, 32, 8, 1024, 128, 24, 128 ** -0.5, (300, 1024)),
+        wl.decode_workload("second", 62, 3, 8, 2, 700, 64, 20, 0.125, (1, 700)),
     ]
     for w in cases:
         q, k, v = to_device(w.q), to_device(w.k_cache), to_device(w.v_cache)

@@ -1,20 +1,23 @@
 // Fused attention, bf16 in / fp32 accumulate / bf16 out (Eq. 8 / Eq. 9): scores, mask, online
 // softmax and the product with V in one kernel; S and P never reach global memory.
 //
-// One CTA = one (batch, query head, 128-query-row tile).  Warp roles:
-//   warp 0    : TMA producer: Q tile once, then K and V tiles (128 keys) through 2-stage rings
-//   warp 1    : tcgen05.mma issuer (one elected lane), owns the TMEM allocation
-//   warps 2-5 : softmax / rescale / epilogue; thread = one query row (TMEM lane), so row
-//               maxima and sums need no cross-thread reduction
-// Tensor memory: S (128 x 128 fp32) double-buffered in columns [0,256), O (128 x D fp32) at 256.
-// Per KV tile j:   S_j = Q K_j^T  ->  softmax warps read S_j, update the running max m and sum l,
-// write P_j (bf16) to shared memory  ->  O += P_j V_j.  S_{j+1} is issued before P_j is waited
-// for, so the tensor core computes the next scores while the softmax of the current tile runs.
+// One CTA = one (batch, query head, pair of 128-row query tiles).  The two tiles run in ping-pong so
+// that the tensor core works on one tile while the softmax of the other is computed.  Warp roles:
+//   warps 0-3 : softmax / rescale / epilogue of tile 0; thread = one query row (TMEM lane), so row
+//   warps 4-7 : the same for tile 1                    maxima and sums need no cross-thread reduction
+//   warp 8    : TMA producer: both Q tiles once, then K and V tiles (128 keys) through rings
+//   warp 9    : tcgen05.mma issuer (one elected lane), owns the TMEM allocation
+//   warps 10-11 only complete the third warpgroup, which hands most of its registers to the other two
+//   (setmaxnreg: 224 per softmax thread, 56 for the rest; 256*224 + 128*56 = 384*168 as launched).
+// Tensor memory (512 columns): S_0 at 0, S_1 at 128 (128 x 128 fp32 each), O_0 at 256, O_1 at 256 + D.
+// P_t (bf16, two per column) is written over the first 64 columns of S_t and is the A operand of
+// the P V product straight from tensor memory.  MMAs execute in issue order, so the issue sequence
+//   S_0(0) S_1(0) | P_0 ready: O_0 += P_0 V_0, S_0(1) | P_1 ready: O_1 += P_1 V_0, S_1(1) | ...
+// keeps every hazard (P_t read before S_t is overwritten, O_t complete before it is rescaled) safe:
+// the barrier that announces S_t(j+1) also covers the completion of every earlier MMA.
 // O is rescaled in TMEM only when a row's maximum grows by more than 2^8 (the stale maximum is
 // kept otherwise; the final division by l uses the same reference, so the result is unchanged).
-//
-// Q and K are K-major operands, V [keys, D] is the MN-major B operand of P V, P is written in the
-// K-major 128-byte-swizzled layout the MMA expects.
+// Q and K are K-major operands, V [keys, D] is the MN-major B operand of P V.
 #include <cuda_bf16.h>
 
 #include "forge_common.cuh"
@@ -26,27 +29,27 @@ namespace {
 
 using namespace ptx;
 
-constexpr int kBM = 128;          // query rows per CTA
+constexpr int kBM = 128;          // query rows per tile
+constexpr int kTilesPerCta = 2;
 constexpr int kBN = 128;          // keys per tile
-constexpr int kThreads = 192;
-constexpr int kSoftmaxThreads = 128;
-constexpr int kKVStages = 2;
+constexpr int kThreads = 384;
+constexpr int kSoftmaxThreads = 128;  // per query tile
 constexpr int kTmemCols = 512;
-constexpr int kColS = 0;          // S buffers at columns 0 and 128
-constexpr int kColO = 256;
+constexpr int kColS = 0;          // S_t at t * 128
+constexpr int kColO = 256;        // O_t at 256 + t * D
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 
 template <int D>
 struct AttnSmem {
-    static constexpr int kChunkBytes = 128 * 128;            // 128 rows x 64 bf16 (one swizzle span wide)
-    static constexpr int kTileBytes = (D / 64) * kChunkBytes;  // Q, K or V tile
-    static constexpr int kPBytes = 2 * kChunkBytes;          // 128 x 128 bf16
+    static constexpr int kChunkBytes = 128 * 128;              // 128 rows x 64 bf16 (one swizzle span wide)
+    static constexpr int kTileBytes = (D / 64) * kChunkBytes;  // a Q, K or V tile
+    static constexpr int kKVStages = (D == 64) ? 4 : 2;
     static constexpr int kQOff = 0;
-    static constexpr int kKOff = kQOff + kTileBytes;
+    static constexpr int kKOff = kQOff + kTilesPerCta * kTileBytes;
     static constexpr int kVOff = kKOff + kKVStages * kTileBytes;
-    static constexpr int kPOff = kVOff + kKVStages * kTileBytes;
-    static constexpr int kBarOff = kPOff + kPBytes;
-    static constexpr int kNumBars = 1 + 4 * kKVStages + 2 + 2;  // q_full, k/v full+empty, s_full[2], p_ready, pv_done
+    static constexpr int kBarOff = kVOff + kKVStages * kTileBytes;
+    // q_full, k/v full+empty per stage, s_full[2], p_ready[2], pv_done[2]
+    static constexpr int kNumBars = 1 + 4 * kKVStages + 6;
     static constexpr int kTotal = kBarOff + kNumBars * 8 + 16;
     static constexpr int kAlloc = kTotal + 1024;
 };
@@ -55,6 +58,33 @@ __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+
+// 3-input maximum and packed two-wide fp32 arithmetic (one instruction for two elements)
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c) {
+    float2 d;
+    asm("{\n\t.reg .b64 ra, rb, rc, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\tmov.b64 rc, {%6, %7};\n\t"
+        "fma.rn.f32x2 rd, ra, rb, rc;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d.x), "=f"(d.y)
+        : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y));
+    return d;
+}
+__device__ __forceinline__ float2 fadd2(float2 a, float2 b) {
+    float2 d;
+    asm("{\n\t.reg .b64 ra, rb, rd;\n\t"
+        "mov.b64 ra, {%2, %3};\n\tmov.b64 rb, {%4, %5};\n\t"
+        "add.rn.f32x2 rd, ra, rb;\n\t"
+        "mov.b64 {%0, %1}, rd;\n\t}"
+        : "=f"(d.x), "=f"(d.y)
+        : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+    return d;
 }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
@@ -76,38 +106,46 @@ __global__ void __launch_bounds__(kThreads, 1)
 attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                  const __grid_constant__ CUtensorMap tmap_v, const AttnParams p) {
     using L = AttnSmem<D>;
+    constexpr int kKVStages = L::kKVStages;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* sQ = smem + L::kQOff;
     uint8_t* sK = smem + L::kKOff;
     uint8_t* sV = smem + L::kVOff;
-    uint8_t* sP = smem + L::kPOff;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBarOff);
     uint64_t* q_full = bars;
     uint64_t* k_full = bars + 1;
     uint64_t* k_empty = k_full + kKVStages;
     uint64_t* v_full = k_empty + kKVStages;
     uint64_t* v_empty = v_full + kKVStages;
-    uint64_t* s_full = v_empty + kKVStages;  // [2]
-    uint64_t* p_ready = s_full + 2;
-    uint64_t* pv_done = p_ready + 1;
-    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(pv_done + 1);
+    uint64_t* s_full = v_empty + kKVStages;  // [2] per query tile
+    uint64_t* p_ready = s_full + 2;          // [2]
+    uint64_t* pv_done = p_ready + 2;         // [2]
+    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(pv_done + 2);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int num_q_tiles = (p.Sq + kBM - 1) / kBM;
-    const int q_tile = num_q_tiles - 1 - blockIdx.x;  // longest (causal) tiles first
+    const int num_q_pairs = (p.Sq + kTilesPerCta * kBM - 1) / (kTilesPerCta * kBM);
+    const int q_pair = num_q_pairs - 1 - blockIdx.x;  // longest (causal) tiles first
     const int h = blockIdx.y, b = blockIdx.z;
     const int kvh = h / (p.Hq / p.Hkv);
-    const int q0 = q_tile * kBM;
     const int causal_off = p.Skv - p.Sq;
     const bool causal = (p.mask_kind & FORGE_MASK_CAUSAL) != 0;
 
     int kvlen = p.Skv;
     if (p.mask_kind & FORGE_MASK_PADDING) kvlen = min(max(p.lens[b], 0), p.Skv);
-    int kv_end = kvlen;  // keys visible to at least one row of this tile
-    if (causal) kv_end = min(kv_end, min(q0 + kBM, p.Sq) + causal_off);
-    kv_end = max(kv_end, 0);
-    const int n_tiles = (kv_end + kBN - 1) / kBN;
+    // KV tiles that are visible to at least one row of each query tile (0 for a tile beyond Sq)
+    int n_tiles[kTilesPerCta];
+    int n_max = 0;
+#pragma unroll
+    for (int t = 0; t < kTilesPerCta; ++t) {
+        const int q0 = (q_pair * kTilesPerCta + t) * kBM;
+        int kv_end = kvlen;
+        if (causal) kv_end = min(kv_end, min(q0 + kBM, p.Sq) + causal_off);
+        if (q0 >= p.Sq) kv_end = 0;
+        kv_end = max(kv_end, 0);
+        n_tiles[t] = (kv_end + kBN - 1) / kBN;
+        n_max = max(n_max, n_tiles[t]);
+    }
 
     if (threadIdx.x == 0) {
         mbar_init(q_full, 1);
@@ -115,13 +153,13 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1);
             mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1);
         }
-        mbar_init(&s_full[0], 1); mbar_init(&s_full[1], 1);
-        mbar_init(p_ready, kSoftmaxThreads);
-        mbar_init(pv_done, 1);
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(&s_full[t], 1); mbar_init(&p_ready[t], kSoftmaxThreads); mbar_init(&pv_done[t], 1);
+        }
         fence_mbar_init();
         prefetch_tmap(&tmap_q); prefetch_tmap(&tmap_k); prefetch_tmap(&tmap_v);
     }
-    if (warp == 1) {
+    if (warp == 9) {
         tmem_alloc(tmem_base_slot, kTmemCols);
         tmem_relinquish();
     }
@@ -131,12 +169,18 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     const uint32_t tmem_base = *tmem_base_slot;
     bool failed = false;
 
-    if (warp == 0) {
-        if (n_tiles > 0 && elect_one()) {
-            mbar_expect_tx(q_full, L::kTileBytes);
+    if (warp >= 8) {
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+      if (warp == 8) {
+        if (n_max > 0 && elect_one()) {
+            mbar_expect_tx(q_full, kTilesPerCta * L::kTileBytes);
 #pragma unroll
-            for (int c = 0; c < D / 64; ++c) tma_load_3d(sQ + c * L::kChunkBytes, &tmap_q, q_full, c * 64, q0, b * p.Hq + h);
-            for (int j = 0; j < n_tiles; ++j) {
+            for (int t = 0; t < kTilesPerCta; ++t)
+#pragma unroll
+                for (int c = 0; c < D / 64; ++c)  // rows beyond Sq are zero-filled by the TMA unit
+                    tma_load_3d(sQ + t * L::kTileBytes + c * L::kChunkBytes, &tmap_q, q_full, c * 64,
+                                (q_pair * kTilesPerCta + t) * kBM, b * p.Hq + h);
+            for (int j = 0; j < n_max; ++j) {
                 const int st = j % kKVStages;
                 const uint32_t ph = (j / kKVStages) & 1;
                 if (!mbar_wait(&k_empty[st], ph ^ 1)) { failed = true; break; }
@@ -153,58 +197,84 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                                 b * p.Hkv + kvh);
             }
         }
-    } else if (warp == 1) {
-        if (n_tiles > 0 && elect_one()) {
+      } else if (warp == 9) {
+        if (n_max > 0 && elect_one()) {
             constexpr uint32_t idesc_s = make_idesc_bf16(kBM, kBN, false, false);
             constexpr uint32_t idesc_o = make_idesc_bf16(kBM, D, false, true);
-            const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV), p_addr = smem_u32(sP);
+            const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
+            int k_waited = -1, v_waited = -1;  // highest KV tile whose arrival has been observed
 
-            auto issue_qk = [&](int j) -> bool {
+            // S_t(j) = Q_t K_j^T; the last tile that uses K_j releases its stage
+            auto issue_qk = [&](int t, int j) -> bool {
                 const int st = j % kKVStages;
-                if (!mbar_wait(&k_full[st], (j / kKVStages) & 1)) return false;
+                if (j > k_waited) {
+                    if (!mbar_wait(&k_full[st], (j / kKVStages) & 1)) return false;
+                    k_waited = j;
+                }
                 tc_fence_after_sync();
-                const uint32_t kb = k_addr + st * L::kTileBytes;
+                const uint32_t kb = k_addr + st * L::kTileBytes, qb = q_addr + t * L::kTileBytes;
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint32_t off = (kk / 4) * L::kChunkBytes + (kk % 4) * 32;
-                    mma_ss(tmem_base + kColS + (j & 1) * kBN, make_smem_desc(q_addr + off, 16, 1024),
+                    mma_ss(tmem_base + kColS + t * kBN, make_smem_desc(qb + off, 16, 1024),
                            make_smem_desc(kb + off, 16, 1024), idesc_s, kk != 0);
                 }
-                mma_commit(&k_empty[st]);
-                mma_commit(&s_full[j & 1]);
+                bool last = true;
+                for (int u = t + 1; u < kTilesPerCta; ++u) last = last && !(j < n_tiles[u]);
+                if (last) mma_commit(&k_empty[st]);
+                mma_commit(&s_full[t]);
                 return true;
             };
-
-            if (!mbar_wait(q_full, 0)) failed = true;
-            if (!failed && !issue_qk(0)) failed = true;
-            for (int j = 0; j < n_tiles && !failed; ++j) {
-                if (j + 1 < n_tiles && !issue_qk(j + 1)) { failed = true; break; }
+            // O_t += P_t(j) V_j with P_t read from tensor memory
+            auto issue_pv = [&](int t, int j) -> bool {
                 const int st = j % kKVStages;
-                if (!mbar_wait(p_ready, j & 1)) { failed = true; break; }
-                if (!mbar_wait(&v_full[st], (j / kKVStages) & 1)) { failed = true; break; }
+                if (!mbar_wait(&p_ready[t], j & 1)) return false;
+                if (j > v_waited) {
+                    if (!mbar_wait(&v_full[st], (j / kKVStages) & 1)) return false;
+                    v_waited = j;
+                }
                 tc_fence_after_sync();
                 const uint32_t vb = v_addr + st * L::kTileBytes;
 #pragma unroll
                 for (int kk = 0; kk < kBN / 16; ++kk) {
-                    // P: K-major, 16 keys = 32 bytes along the swizzled row, 64-key chunks 16 KB apart.
-                    // V: MN-major, 16 keys = two 1024-byte groups; 64-wide chunks of D are 16 KB apart.
-                    mma_ss(tmem_base + kColO,
-                           make_smem_desc(p_addr + (kk / 4) * L::kChunkBytes + (kk % 4) * 32, 16, 1024),
+                    // P: 16 keys = 8 columns of packed bf16 pairs.  V: MN-major, 16 keys = two 1024-byte
+                    // groups; the 64-wide chunks of D are 16 KB apart.
+                    mma_ts(tmem_base + kColO + t * D, tmem_base + kColS + t * kBN + kk * 8,
                            make_smem_desc(vb + kk * 2048, L::kChunkBytes, 1024), idesc_o, (j | kk) != 0);
                 }
-                mma_commit(&v_empty[st]);
-                mma_commit(pv_done);
+                bool last = true;
+                for (int u = t + 1; u < kTilesPerCta; ++u) last = last && !(j < n_tiles[u]);
+                if (last) mma_commit(&v_empty[st]);
+                mma_commit(&pv_done[t]);
+                return true;
+            };
+
+            if (!mbar_wait(q_full, 0)) failed = true;
+            for (int t = 0; t < kTilesPerCta && !failed; ++t)
+                if (n_tiles[t] > 0 && !issue_qk(t, 0)) failed = true;
+            for (int j = 0; j < n_max && !failed; ++j) {
+                for (int t = 0; t < kTilesPerCta && !failed; ++t) {
+                    if (j >= n_tiles[t]) continue;
+                    if (!issue_pv(t, j)) { failed = true; break; }
+                    if (j + 1 < n_tiles[t] && !issue_qk(t, j + 1)) { failed = true; break; }
+                }
             }
         }
+      }
     } else {
-        const int quarter = warp & 3;
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+        const int t = warp >> 2;  // query tile of this warp group
+        const int quarter = warp & 3;   // TMEM lane quarter this warp may access
         const int row = quarter * 32 + lane;
+        const int q0 = (q_pair * kTilesPerCta + t) * kBM;
         const int qi = q0 + row;
+        const int nt = n_tiles[t];
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+        const uint32_t col_s = kColS + t * kBN, col_o = kColO + t * D;
         const float sl2 = p.scale_log2;
         __nv_bfloat16* orow = p.out + ((size_t)(b * p.Hq + h) * p.Sq + qi) * D;
 
-        if (n_tiles == 0) {
+        if (nt == 0) {
             if (qi < p.Sq) {
 #pragma unroll
                 for (int c = 0; c < D / 8; ++c) reinterpret_cast<uint4*>(orow)[c] = make_uint4(0, 0, 0, 0);
@@ -213,14 +283,16 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             float m_run = -INFINITY;  // running maximum of the raw scores (reference of the exponentials)
             float l_run = 0.f;
             const int row_limit = causal ? qi + causal_off : 0x7fffffff;  // last visible key of this row
-            for (int j = 0; j < n_tiles; ++j) {
-                if (!warp_wait(&s_full[j & 1], (j >> 1) & 1)) { failed = true; break; }
+            for (int j = 0; j < nt; ++j) {
+                // S_t(j) is complete, and so is every MMA issued before it: O_t holds all earlier P V
+                // products and P_t(j-1) has been consumed.
+                if (!warp_wait(&s_full[t], j & 1)) { failed = true; break; }
                 tc_fence_after_sync();
                 float s[kBN];
 #pragma unroll
                 for (int c = 0; c < kBN / 32; ++c) {
                     uint32_t r[32];
-                    tmem_ld_x32(lane_base + kColS + (j & 1) * kBN + c * 32, r);
+                    tmem_ld_x32(lane_base + col_s + c * 32, r);
 #pragma unroll
                     for (int i = 0; i < 32; ++i) s[c * 32 + i] = __uint_as_float(r[i]);
                 }
@@ -233,9 +305,18 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
 #pragma unroll
                     for (int i = 0; i < kBN; ++i) s[i] = (i <= lim) ? s[i] : -INFINITY;
                 }
-                float m_tile = s[0];
+                // row maximum: four independent chains of 3-input maxima
+                float mx[4] = {s[0], s[1], s[2], s[3]};
 #pragma unroll
-                for (int i = 1; i < kBN; ++i) m_tile = fmaxf(m_tile, s[i]);
+                for (int i = 4; i + 7 < kBN; i += 8) {
+                    mx[0] = max3(mx[0], s[i], s[i + 1]);
+                    mx[1] = max3(mx[1], s[i + 2], s[i + 3]);
+                    mx[2] = max3(mx[2], s[i + 4], s[i + 5]);
+                    mx[3] = max3(mx[3], s[i + 6], s[i + 7]);
+                }
+                mx[0] = max3(mx[0], s[kBN - 4], s[kBN - 3]);
+                mx[1] = max3(mx[1], s[kBN - 2], s[kBN - 1]);
+                const float m_tile = max3(fmaxf(mx[0], mx[1]), mx[2], mx[3]);
 
                 // Keep the old reference unless this tile's maximum exceeds it by more than the
                 // threshold (in log2 units of the scaled scores); then every later exponent is <= 8.
@@ -247,62 +328,56 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     alpha = (m_run == -INFINITY) ? 1.f : ex2((m_run - m_tile) * sl2);
                     m_run = m_tile;
                 }
+                if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t r[32];
+                        tmem_ld_x32(lane_base + col_o + c * 32, r);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+                        tmem_st_x32(lane_base + col_o + c * 32, r);
+                    }
+                }
                 const float m_ref = (m_run == -INFINITY) ? 0.f : m_run;
-                const float neg_m = -m_ref * sl2;
-                float l_tile = 0.f;
-                uint32_t packed[kBN / 2];
+                const float2 sl2v = make_float2(sl2, sl2);
+                const float2 neg_m = make_float2(-m_ref * sl2, -m_ref * sl2);
+                const bool fix_zero_scale = need_mask && sl2 == 0.f;  // -inf * 0 would be NaN
+                float2 lsum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+                // P as packed bf16 pairs, written over the first 64 columns of S_t in two halves
 #pragma unroll
-                for (int i = 0; i < kBN / 2; ++i) {
-                    // masked: s = -inf.  With sl2 > 0 the fma gives -inf and ex2 gives exactly 0.
-                    float p0 = ex2(fmaf(s[2 * i], sl2, neg_m));
-                    float p1 = ex2(fmaf(s[2 * i + 1], sl2, neg_m));
-                    if (need_mask) {  // also covers sl2 == 0, where -inf * 0 would be NaN
-                        p0 = (s[2 * i] == -INFINITY) ? 0.f : p0;
-                        p1 = (s[2 * i + 1] == -INFINITY) ? 0.f : p1;
-                    }
-                    l_tile += p0 + p1;
-                    packed[i] = pack_bf16(p0, p1);
-                }
-                l_run = l_run * alpha + l_tile;
-
-                // P buffer and O are free once the previous P V has completed.
-                if (j > 0) {
-                    if (!warp_wait(pv_done, (j - 1) & 1)) { failed = true; break; }
-                    tc_fence_after_sync();
-                    if (__any_sync(0xffffffffu, alpha != 1.f)) {
+                for (int half = 0; half < 2; ++half) {
+                    uint32_t packed[32];
 #pragma unroll
-                        for (int c = 0; c < D / 32; ++c) {
-                            uint32_t r[32];
-                            tmem_ld_x32(lane_base + kColO + c * 32, r);
-                            tmem_ld_wait();
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-                            tmem_st_x32(lane_base + kColO + c * 32, r);
+                    for (int i = 0; i < 32; ++i) {
+                        const float s0 = s[half * 64 + 2 * i], s1 = s[half * 64 + 2 * i + 1];
+                        // masked: s = -inf; with sl2 > 0 the fma gives -inf and ex2 gives exactly 0
+                        const float2 x = ffma2(make_float2(s0, s1), sl2v, neg_m);
+                        float2 pr = make_float2(ex2(x.x), ex2(x.y));
+                        if (fix_zero_scale) {
+                            pr.x = (s0 == -INFINITY) ? 0.f : 1.f;
+                            pr.y = (s1 == -INFINITY) ? 0.f : 1.f;
                         }
-                        tmem_st_wait();
+                        lsum[i & 1] = fadd2(lsum[i & 1], pr);
+                        packed[i] = pack_bf16(pr.x, pr.y);
                     }
+                    tmem_st_x32(lane_base + col_s + half * 32, packed);
                 }
-                // P[row, 0..127] as bf16 into the K-major swizzled layout: 16-byte chunk c of the row
-                // goes to chunk (c % 8) ^ (row % 8) of its 128-byte line; keys 64..127 sit 16 KB further.
-#pragma unroll
-                for (int c = 0; c < 16; ++c) {
-                    uint8_t* dst = sP + (c / 8) * L::kChunkBytes + row * 128 + (((c % 8) ^ (row & 7)) << 4);
-                    *reinterpret_cast<uint4*>(dst) =
-                        make_uint4(packed[4 * c], packed[4 * c + 1], packed[4 * c + 2], packed[4 * c + 3]);
-                }
-                fence_proxy_async_smem();
+                const float l_tile = (lsum[0].x + lsum[0].y) + (lsum[1].x + lsum[1].y);
+                l_run = l_run * alpha + l_tile;
+                tmem_st_wait();
                 tc_fence_before_sync();
-                mbar_arrive(p_ready);
+                mbar_arrive(&p_ready[t]);
             }
 
-            if (!failed && !warp_wait(pv_done, (n_tiles - 1) & 1)) failed = true;
+            if (!failed && !warp_wait(&pv_done[t], (nt - 1) & 1)) failed = true;
             if (!failed) {
                 tc_fence_after_sync();
                 const float inv = l_run > 0.f ? 1.f / l_run : 0.f;  // no visible key: zeros
 #pragma unroll
                 for (int c = 0; c < D / 32; ++c) {
                     uint32_t r[32];
-                    tmem_ld_x32(lane_base + kColO + c * 32, r);
+                    tmem_ld_x32(lane_base + col_o + c * 32, r);
                     tmem_ld_wait();
                     if (qi < p.Sq) {
 #pragma unroll
@@ -326,7 +401,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     }
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == 9) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, kTmemCols);
     }
@@ -359,7 +434,7 @@ int launch_attn(const void* q, const void* k, const void* v, void* out, int B, i
     if (!p.status) return FORGE_ERR_CUDA;
     auto kernel = attn_bf16_kernel<D>;
     FORGE_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kAlloc));
-    const dim3 grid((Sq + kBM - 1) / kBM, Hq, B);
+    const dim3 grid((Sq + kTilesPerCta * kBM - 1) / (kTilesPerCta * kBM), Hq, B);
     kernel<<<grid, kThreads, L::kAlloc, s>>>(tq, tk, tv, p);
     return finish_launch(1);
 }

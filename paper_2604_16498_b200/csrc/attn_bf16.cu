@@ -20,6 +20,8 @@
 // Q and K are K-major operands, V [keys, D] is the MN-major B operand of P V.
 #include <cuda_bf16.h>
 
+#include <type_traits>
+
 #include "forge_common.cuh"
 #include "sm100_ptx.cuh"
 #include "tmap.cuh"
@@ -125,8 +127,10 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_q_pairs = (p.Sq + kTilesPerCta * kBM - 1) / (kTilesPerCta * kBM);
-    const int q_pair = num_q_pairs - 1 - blockIdx.x;  // longest (causal) tiles first
-    const int h = blockIdx.y, b = blockIdx.z;
+    // blockIdx.x runs over (batch, head), blockIdx.y over the tile pairs with the longest (causal) pair
+    // first: CTAs are dispatched in that order, so the long ones start first everywhere (LPT).
+    const int q_pair = num_q_pairs - 1 - blockIdx.y;
+    const int h = blockIdx.x % p.Hq, b = blockIdx.x / p.Hq;
     const int kvh = h / (p.Hq / p.Hkv);
     const int causal_off = p.Skv - p.Sq;
     const bool causal = (p.mask_kind & FORGE_MASK_CAUSAL) != 0;
@@ -342,27 +346,32 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 const float m_ref = (m_run == -INFINITY) ? 0.f : m_run;
                 const float2 sl2v = make_float2(sl2, sl2);
                 const float2 neg_m = make_float2(-m_ref * sl2, -m_ref * sl2);
-                const bool fix_zero_scale = need_mask && sl2 == 0.f;  // -inf * 0 would be NaN
                 float2 lsum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-                // P as packed bf16 pairs, written over the first 64 columns of S_t in two halves
+                // P = 2^(s * sl2 - m * sl2) as packed bf16 pairs, written over the first 64 columns of S_t
+                // in two halves.  In masked tiles the probability of a masked key is forced to exactly 0
+                // (that also covers sl2 == 0, where -inf * 0 would be NaN); full tiles skip the selects.
+                auto exp_and_store = [&](auto masked_tag) {
+                    constexpr bool kMasked = decltype(masked_tag)::value;
 #pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    uint32_t packed[32];
+                    for (int half = 0; half < 2; ++half) {
+                        uint32_t packed[32];
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const float s0 = s[half * 64 + 2 * i], s1 = s[half * 64 + 2 * i + 1];
-                        // masked: s = -inf; with sl2 > 0 the fma gives -inf and ex2 gives exactly 0
-                        const float2 x = ffma2(make_float2(s0, s1), sl2v, neg_m);
-                        float2 pr = make_float2(ex2(x.x), ex2(x.y));
-                        if (fix_zero_scale) {
-                            pr.x = (s0 == -INFINITY) ? 0.f : 1.f;
-                            pr.y = (s1 == -INFINITY) ? 0.f : 1.f;
+                        for (int i = 0; i < 32; ++i) {
+                            const float s0 = s[half * 64 + 2 * i], s1 = s[half * 64 + 2 * i + 1];
+                            const float2 x = ffma2(make_float2(s0, s1), sl2v, neg_m);
+                            float2 pr = make_float2(ex2(x.x), ex2(x.y));
+                            if constexpr (kMasked) {
+                                pr.x = (s0 == -INFINITY) ? 0.f : pr.x;
+                                pr.y = (s1 == -INFINITY) ? 0.f : pr.y;
+                            }
+                            lsum[i & 1] = fadd2(lsum[i & 1], pr);
+                            packed[i] = pack_bf16(pr.x, pr.y);
                         }
-                        lsum[i & 1] = fadd2(lsum[i & 1], pr);
-                        packed[i] = pack_bf16(pr.x, pr.y);
+                        tmem_st_x32(lane_base + col_s + half * 32, packed);
                     }
-                    tmem_st_x32(lane_base + col_s + half * 32, packed);
-                }
+                };
+                if (need_mask) exp_and_store(std::true_type{});
+                else exp_and_store(std::false_type{});
                 const float l_tile = (lsum[0].x + lsum[0].y) + (lsum[1].x + lsum[1].y);
                 l_run = l_run * alpha + l_tile;
                 tmem_st_wait();
@@ -434,7 +443,7 @@ int launch_attn(const void* q, const void* k, const void* v, void* out, int B, i
     if (!p.status) return FORGE_ERR_CUDA;
     auto kernel = attn_bf16_kernel<D>;
     FORGE_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kAlloc));
-    const dim3 grid((Sq + kTilesPerCta * kBM - 1) / (kTilesPerCta * kBM), Hq, B);
+    const dim3 grid(Hq * B, (Sq + kTilesPerCta * kBM - 1) / (kTilesPerCta * kBM), 1);
     kernel<<<grid, kThreads, L::kAlloc, s>>>(tq, tk, tv, p);
     return finish_launch(1);
 }
@@ -448,7 +457,7 @@ extern "C" int forge_attn_fused(const void* q, const void* k, const void* v, voi
     using namespace forge;
     int st = check_attn_args(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens);
     if (st != FORGE_OK) return st;
-    if (Hq > 65535 || B > 65535) return FORGE_ERR_UNSUPPORTED;
+    if ((long long)Hq * B > 2147483647LL || (Sq + 255) / 256 > 65535) return FORGE_ERR_UNSUPPORTED;
     if (!(scale >= 0.f)) return FORGE_ERR_UNSUPPORTED;  // the running maximum is taken on unscaled scores
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     return D == 64 ? launch_attn<64>(q, k, v, out, B, Hq, Hkv, Sq, Skv, mask_kind, lens, scale, s)

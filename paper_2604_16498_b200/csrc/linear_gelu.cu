@@ -5,7 +5,7 @@
 // Persistent, warp-specialised kernel, one CTA per SM:
 //   warp 0    : TMA producer  (X tile 128 x 64, W tile 64 x BN per stage, 128-byte swizzle)
 //   warp 1    : tcgen05.mma issuer (one elected lane), owns the TMEM allocation
-//   warps 2-5 : epilogue (TMEM -> registers -> +bias -> GELU -> bf16 -> global)
+//   warps 2-5 : epilogue (TMEM -> registers -> +bias -> GELU -> bf16 -> swizzled shared memory -> TMA store)
 // Two TMEM accumulators: the epilogue of tile i overlaps the main loop of tile i+1.
 // X [M,K] is the K-major A operand; W [K,N] (N contiguous) is the MN-major B operand, so no
 // transposed copy of the weights is needed.
@@ -32,7 +32,9 @@ struct LinearSmem {
     static constexpr int kABytes = kBM * kBK * 2;        // 16 KB
     static constexpr int kBBytes = kBK * BN * 2;         // 64 rows of K x BN
     static constexpr int kStageBytes = kABytes + kBBytes;
-    static constexpr int kBarOffset = STAGES * kStageBytes;
+    static constexpr int kOutBytes = kBM * 128;          // output staging: 128 rows x 64 bf16, two buffers
+    static constexpr int kOutOffset = STAGES * kStageBytes;
+    static constexpr int kBarOffset = kOutOffset + 2 * kOutBytes;
     // barriers: full[S], empty[S], tmem_full[2], tmem_empty[2]; then the TMEM base, then bias[2][BN]
     static constexpr int kBiasOffset = kBarOffset + (2 * STAGES + 4) * 8 + 16;
     static constexpr int kTotal = kBiasOffset + 2 * BN * 4;
@@ -56,7 +58,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 template <int BN, int STAGES>
 __global__ void __launch_bounds__(kThreads, 1)
 linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
-                        const __nv_bfloat16* __restrict__ bias, __nv_bfloat16* __restrict__ y,
+                        const __grid_constant__ CUtensorMap tmap_y, const __nv_bfloat16* __restrict__ bias,
                         int M, int N, int K, int* __restrict__ status) {
     using L = LinearSmem<BN, STAGES>;
     extern __shared__ uint8_t smem_raw[];
@@ -79,6 +81,7 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
         fence_mbar_init();
         prefetch_tmap(&tmap_x);
         prefetch_tmap(&tmap_w);
+        prefetch_tmap(&tmap_y);
     }
     if (warp == 1) {
         tmem_alloc(tmem_base_slot, kTmemCols);
@@ -145,6 +148,7 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
         const int quarter = warp & 3;            // TMEM lane quarter this warp may access
         const int etid = (warp - 2) * 32 + lane; // 0..127
         int it = 0;
+        int out_blocks = 0;  // 64-column blocks stored so far (selects the staging buffer)
         for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
             const int m0 = (tile / tiles_n) * kBM, n0 = (tile % tiles_n) * BN;
             const int acc = it & 1;
@@ -158,34 +162,51 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
             if (!failed && !warp_wait(&tmem_full[acc], acc_phase)) failed = true;
             if (failed) continue;
             tc_fence_after_sync();
-            const int row = m0 + quarter * 32 + lane;
+            const int row = quarter * 32 + lane;  // row of the tile = TMEM lane
             const uint32_t taddr = tmem_base + acc * kAccStride + (static_cast<uint32_t>(quarter * 32) << 16);
-            __nv_bfloat16* yrow = y + (size_t)row * N + n0;
+            // 64 output columns at a time: registers -> bf16 -> swizzled staging buffer -> one TMA store.
+            // Two staging buffers: the store of one block drains while the next block is computed.
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t r[32];
-                tmem_ld_x32(taddr + c * 32, r);
-                tmem_ld_wait();
-                uint32_t packed[16];
+            for (int blk = 0; blk < BN / 64; ++blk, ++out_blocks) {
+                uint8_t* stage_out = smem + L::kOutOffset + (out_blocks & 1) * L::kOutBytes;
+                uint32_t r[64];
+                {
+                    uint32_t lo[32], hi[32];
+                    tmem_ld_x32(taddr + blk * 64, lo);
+                    tmem_ld_x32(taddr + blk * 64 + 32, hi);
+                    tmem_ld_wait();
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const float z0 = __uint_as_float(r[2 * i]) + bias_s[c * 32 + 2 * i];
-                    const float z1 = __uint_as_float(r[2 * i + 1]) + bias_s[c * 32 + 2 * i + 1];
-                    packed[i] = pack_bf16(gelu_tanh_f32(z0), gelu_tanh_f32(z1));
+                    for (int i = 0; i < 32; ++i) { r[i] = lo[i]; r[32 + i] = hi[i]; }
                 }
-                if (row < M) {
+                // the store issued two blocks ago has finished reading this buffer
+                if (etid == 0) tma_store_wait_read<1>();
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        if (n0 + c * 32 + v * 8 < N)  // N is a multiple of 8: an 8-column group is all in or all out
-                            *reinterpret_cast<uint4*>(yrow + c * 32 + v * 8) =
-                                make_uint4(packed[4 * v], packed[4 * v + 1], packed[4 * v + 2], packed[4 * v + 3]);
+                for (int c = 0; c < 8; ++c) {  // 16-byte chunk c of the row's 128-byte line
+                    uint32_t w[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int col = c * 8 + 2 * i;
+                        const float z0 = __uint_as_float(r[col]) + bias_s[blk * 64 + col];
+                        const float z1 = __uint_as_float(r[col + 1]) + bias_s[blk * 64 + col + 1];
+                        w[i] = pack_bf16(gelu_tanh_f32(z0), gelu_tanh_f32(z1));
                     }
+                    *reinterpret_cast<uint4*>(stage_out + row * 128 + ((c ^ (row & 7)) << 4)) =
+                        make_uint4(w[0], w[1], w[2], w[3]);
+                }
+                fence_proxy_async_smem();
+                asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+                if (etid == 0) {
+                    // rows >= M and columns >= N are clipped by the TMA unit
+                    tma_store_2d(&tmap_y, stage_out, n0 + blk * 64, m0);
+                    tma_store_commit();
                 }
             }
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&tmem_empty[acc]);
         }
+        if (etid == 0) tma_store_wait_all<0>();  // every output tile has left shared memory and is written
     }
 
     if (failed) {
@@ -217,6 +238,13 @@ int launch_linear(const void* x, const void* w, const void* b, void* y, int M, i
         const uint32_t box[2] = {64, kBK};
         if (!encode_tmap_bf16_sw128(&tmap_w, w, 2, dims, strides, box)) return FORGE_ERR_CUDA;
     }
+    CUtensorMap tmap_y;
+    {
+        const uint64_t dims[2] = {(uint64_t)N, (uint64_t)M};
+        const uint64_t strides[1] = {(uint64_t)N * 2};
+        const uint32_t box[2] = {64, kBM};
+        if (!encode_tmap_bf16_sw128(&tmap_y, y, 2, dims, strides, box)) return FORGE_ERR_CUDA;
+    }
     int* status = device_status_word();
     if (!status) return FORGE_ERR_CUDA;
     int dev = 0, sms = 0;
@@ -226,8 +254,8 @@ int launch_linear(const void* x, const void* w, const void* b, void* y, int M, i
     FORGE_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kAlloc));
     const int tiles = ((M + kBM - 1) / kBM) * ((N + BN - 1) / BN);
     const int grid = tiles < sms ? tiles : sms;
-    kernel<<<grid, kThreads, L::kAlloc, s>>>(tmap_x, tmap_w, static_cast<const __nv_bfloat16*>(b),
-                                             static_cast<__nv_bfloat16*>(y), M, N, K, status);
+    kernel<<<grid, kThreads, L::kAlloc, s>>>(tmap_x, tmap_w, tmap_y, static_cast<const __nv_bfloat16*>(b), M, N, K,
+                                             status);
     return finish_launch(1);
 }
 
@@ -241,5 +269,5 @@ extern "C" int forge_linear_bias_gelu(const void* x, const void* w, const void* 
     if (M <= 0 || N <= 0 || K <= 0) return FORGE_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(w) || !aligned16(b) || !aligned16(y)) return FORGE_ERR_INVALID_ARG;
     if ((K % 8) != 0 || (N % 8) != 0) return FORGE_ERR_UNSUPPORTED;
-    return launch_linear<192, 5>(x, w, b, y, M, N, K, static_cast<cudaStream_t>(stream));
+    return launch_linear<192, 4>(x, w, b, y, M, N, K, static_cast<cudaStream_t>(stream));
 }

@@ -5,7 +5,7 @@
 // Persistent, warp-specialised kernel, one CTA per SM:
 //   warp 0    : TMA producer  (X tile 128 x 64, W tile 64 x BN per stage, 128-byte swizzle)
 //   warp 1    : tcgen05.mma issuer (one elected lane), owns the TMEM allocation
-//   warps 2-5 : epilogue (TMEM -> registers -> +bias -> GELU -> bf16 -> swizzled shared memory -> TMA store)
+//   warps 2-9 : epilogue, two warps per TMEM lane quarter, each half of the 64 columns of a block (TMEM -> registers -> +bias -> GELU -> bf16 -> swizzled shared memory -> TMA store)
 // Two TMEM accumulators: the epilogue of tile i overlaps the main loop of tile i+1.
 // X [M,K] is the K-major A operand; W [K,N] (N contiguous) is the MN-major B operand, so no
 // transposed copy of the weights is needed.
@@ -22,8 +22,8 @@ using namespace ptx;
 
 constexpr int kBM = 128;
 constexpr int kBK = 64;
-constexpr int kThreads = 192;
-constexpr int kEpiThreads = 128;
+constexpr int kThreads = 320;
+constexpr int kEpiThreads = 256;
 constexpr int kAccStride = 256;   // TMEM columns between the two accumulators
 constexpr int kTmemCols = 512;
 
@@ -146,7 +146,8 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
         }
     } else {
         const int quarter = warp & 3;            // TMEM lane quarter this warp may access
-        const int etid = (warp - 2) * 32 + lane; // 0..127
+        const int etid = (warp - 2) * 32 + lane; // 0..255
+        const int chalf = (warp - 2) >> 2;       // which 32 of a block's 64 columns this warp handles
         int it = 0;
         int out_blocks = 0;  // 64-column blocks stored so far (selects the staging buffer)
         for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
@@ -169,29 +170,23 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
 #pragma unroll 1
             for (int blk = 0; blk < BN / 64; ++blk, ++out_blocks) {
                 uint8_t* stage_out = smem + L::kOutOffset + (out_blocks & 1) * L::kOutBytes;
-                uint32_t r[64];
-                {
-                    uint32_t lo[32], hi[32];
-                    tmem_ld_x32(taddr + blk * 64, lo);
-                    tmem_ld_x32(taddr + blk * 64 + 32, hi);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) { r[i] = lo[i]; r[32 + i] = hi[i]; }
-                }
+                uint32_t r[32];
+                tmem_ld_x32(taddr + blk * 64 + chalf * 32, r);
+                tmem_ld_wait();
                 // the store issued two blocks ago has finished reading this buffer
                 if (etid == 0) tma_store_wait_read<1>();
                 asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {  // 16-byte chunk c of the row's 128-byte line
+                for (int c = 0; c < 4; ++c) {  // 16-byte chunk chalf*4 + c of the row's 128-byte line
                     uint32_t w[4];
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const int col = c * 8 + 2 * i;
-                        const float z0 = __uint_as_float(r[col]) + bias_s[blk * 64 + col];
-                        const float z1 = __uint_as_float(r[col + 1]) + bias_s[blk * 64 + col + 1];
+                        const float z0 = __uint_as_float(r[col]) + bias_s[blk * 64 + chalf * 32 + col];
+                        const float z1 = __uint_as_float(r[col + 1]) + bias_s[blk * 64 + chalf * 32 + col + 1];
                         w[i] = pack_bf16(gelu_tanh_f32(z0), gelu_tanh_f32(z1));
                     }
-                    *reinterpret_cast<uint4*>(stage_out + row * 128 + ((c ^ (row & 7)) << 4)) =
+                    *reinterpret_cast<uint4*>(stage_out + row * 128 + (((chalf * 4 + c) ^ (row & 7)) << 4)) =
                         make_uint4(w[0], w[1], w[2], w[3]);
                 }
                 fence_proxy_async_smem();

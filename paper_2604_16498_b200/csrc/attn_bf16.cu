@@ -158,7 +158,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1);
         }
         for (int t = 0; t < 2; ++t) {
-            mbar_init(&s_full[t], 1); mbar_init(&p_ready[t], kSoftmaxThreads); mbar_init(&pv_done[t], 1);
+            mbar_init(&s_full[t], 1); mbar_init(&p_ready[t], kSoftmaxThreads / 32); mbar_init(&pv_done[t], 1);
         }
         fence_mbar_init();
         prefetch_tmap(&tmap_q); prefetch_tmap(&tmap_k); prefetch_tmap(&tmap_v);
@@ -309,74 +309,107 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
 #pragma unroll
                     for (int i = 0; i < kBN; ++i) s[i] = (i <= lim) ? s[i] : -INFINITY;
                 }
-                // row maximum: four independent chains of 3-input maxima
-                float mx[4] = {s[0], s[1], s[2], s[3]};
-#pragma unroll
-                for (int i = 4; i + 7 < kBN; i += 8) {
-                    mx[0] = max3(mx[0], s[i], s[i + 1]);
-                    mx[1] = max3(mx[1], s[i + 2], s[i + 3]);
-                    mx[2] = max3(mx[2], s[i + 4], s[i + 5]);
-                    mx[3] = max3(mx[3], s[i + 6], s[i + 7]);
-                }
-                mx[0] = max3(mx[0], s[kBN - 4], s[kBN - 3]);
-                mx[1] = max3(mx[1], s[kBN - 2], s[kBN - 1]);
-                const float m_tile = max3(fmaxf(mx[0], mx[1]), mx[2], mx[3]);
-
-                // Keep the old reference unless this tile's maximum exceeds it by more than the
-                // threshold (in log2 units of the scaled scores); then every later exponent is <= 8.
-                float alpha = 1.f;
-                bool grow = (m_tile - m_run) * sl2 > kRescaleThreshold || m_run == -INFINITY;
-                if (m_tile == -INFINITY) grow = false;
-                if (grow) {
-                    // first visible keys of this row: nothing accumulated yet, nothing to rescale
-                    alpha = (m_run == -INFINITY) ? 1.f : ex2((m_run - m_tile) * sl2);
-                    m_run = m_tile;
-                }
-                if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-#pragma unroll
-                    for (int c = 0; c < D / 32; ++c) {
-                        uint32_t r[32];
-                        tmem_ld_x32(lane_base + col_o + c * 32, r);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-                        tmem_st_x32(lane_base + col_o + c * 32, r);
-                    }
-                }
-                const float m_ref = (m_run == -INFINITY) ? 0.f : m_run;
                 const float2 sl2v = make_float2(sl2, sl2);
-                const float2 neg_m = make_float2(-m_ref * sl2, -m_ref * sl2);
-                float2 lsum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-                // P = 2^(s * sl2 - m * sl2) as packed bf16 pairs, written over the first 64 columns of S_t
-                // in two halves.  In masked tiles the probability of a masked key is forced to exactly 0
-                // (that also covers sl2 == 0, where -inf * 0 would be NaN); full tiles skip the selects.
-                auto exp_and_store = [&](auto masked_tag) {
-                    constexpr bool kMasked = decltype(masked_tag)::value;
+                // Fast path (full tiles once every row has a finite reference): exponentials against the
+                // current reference in the same pass that finds the tile maximum.  Valid as long as no row's
+                // maximum exceeds its reference by more than the threshold, which is what the lazy rescale
+                // tolerates anyway; otherwise the tile is redone below with a new reference.
+                bool done = false;
+                if (!need_mask && __all_sync(0xffffffffu, m_run != -INFINITY)) {
+                    const float2 neg_m = make_float2(-m_run * sl2, -m_run * sl2);
+                    float2 lsum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+                    float mx[4] = {s[0], s[1], s[2], s[3]};
 #pragma unroll
                     for (int half = 0; half < 2; ++half) {
                         uint32_t packed[32];
 #pragma unroll
                         for (int i = 0; i < 32; ++i) {
                             const float s0 = s[half * 64 + 2 * i], s1 = s[half * 64 + 2 * i + 1];
+                            mx[i & 3] = max3(mx[i & 3], s0, s1);
                             const float2 x = ffma2(make_float2(s0, s1), sl2v, neg_m);
-                            float2 pr = make_float2(ex2(x.x), ex2(x.y));
-                            if constexpr (kMasked) {
-                                pr.x = (s0 == -INFINITY) ? 0.f : pr.x;
-                                pr.y = (s1 == -INFINITY) ? 0.f : pr.y;
-                            }
+                            const float2 pr = make_float2(ex2(x.x), ex2(x.y));
                             lsum[i & 1] = fadd2(lsum[i & 1], pr);
                             packed[i] = pack_bf16(pr.x, pr.y);
                         }
                         tmem_st_x32(lane_base + col_s + half * 32, packed);
                     }
-                };
-                if (need_mask) exp_and_store(std::true_type{});
-                else exp_and_store(std::false_type{});
-                const float l_tile = (lsum[0].x + lsum[0].y) + (lsum[1].x + lsum[1].y);
-                l_run = l_run * alpha + l_tile;
+                    const float m_tile = max3(fmaxf(mx[0], mx[1]), mx[2], mx[3]);
+                    if (!__any_sync(0xffffffffu, (m_tile - m_run) * sl2 > kRescaleThreshold)) {
+                        l_run += (lsum[0].x + lsum[0].y) + (lsum[1].x + lsum[1].y);
+                        done = true;
+                    }
+                }
+                if (!done) {
+                    // row maximum: four independent chains of 3-input maxima
+                    float mx[4] = {s[0], s[1], s[2], s[3]};
+    #pragma unroll
+                    for (int i = 4; i + 7 < kBN; i += 8) {
+                        mx[0] = max3(mx[0], s[i], s[i + 1]);
+                        mx[1] = max3(mx[1], s[i + 2], s[i + 3]);
+                        mx[2] = max3(mx[2], s[i + 4], s[i + 5]);
+                        mx[3] = max3(mx[3], s[i + 6], s[i + 7]);
+                    }
+                    mx[0] = max3(mx[0], s[kBN - 4], s[kBN - 3]);
+                    mx[1] = max3(mx[1], s[kBN - 2], s[kBN - 1]);
+                    const float m_tile = max3(fmaxf(mx[0], mx[1]), mx[2], mx[3]);
+
+                    // Keep the old reference unless this tile's maximum exceeds it by more than the
+                    // threshold (in log2 units of the scaled scores); then every later exponent is <= 8.
+                    float alpha = 1.f;
+                    bool grow = (m_tile - m_run) * sl2 > kRescaleThreshold || m_run == -INFINITY;
+                    if (m_tile == -INFINITY) grow = false;
+                    if (grow) {
+                        // first visible keys of this row: nothing accumulated yet, nothing to rescale
+                        alpha = (m_run == -INFINITY) ? 1.f : ex2((m_run - m_tile) * sl2);
+                        m_run = m_tile;
+                    }
+                    if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+                        // rare after the first tiles: small chunks, not unrolled, to keep register pressure low
+    #pragma unroll 1
+                        for (int c = 0; c < D / 16; ++c) {
+                            uint32_t r[16];
+                            tmem_ld_x16(lane_base + col_o + c * 16, r);
+                            tmem_ld_wait();
+    #pragma unroll
+                            for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+                            tmem_st_x16(lane_base + col_o + c * 16, r);
+                        }
+                    }
+                    const float m_ref = (m_run == -INFINITY) ? 0.f : m_run;
+                    const float2 neg_m = make_float2(-m_ref * sl2, -m_ref * sl2);
+                    float2 lsum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+                    // P = 2^(s * sl2 - m * sl2) as packed bf16 pairs, written over the first 64 columns of S_t
+                    // in two halves.  In masked tiles the probability of a masked key is forced to exactly 0
+                    // (that also covers sl2 == 0, where -inf * 0 would be NaN); full tiles skip the selects.
+                    auto exp_and_store = [&](auto masked_tag) {
+                        constexpr bool kMasked = decltype(masked_tag)::value;
+    #pragma unroll
+                        for (int half = 0; half < 2; ++half) {
+                            uint32_t packed[32];
+    #pragma unroll
+                            for (int i = 0; i < 32; ++i) {
+                                const float s0 = s[half * 64 + 2 * i], s1 = s[half * 64 + 2 * i + 1];
+                                const float2 x = ffma2(make_float2(s0, s1), sl2v, neg_m);
+                                float2 pr = make_float2(ex2(x.x), ex2(x.y));
+                                if constexpr (kMasked) {
+                                    pr.x = (s0 == -INFINITY) ? 0.f : pr.x;
+                                    pr.y = (s1 == -INFINITY) ? 0.f : pr.y;
+                                }
+                                lsum[i & 1] = fadd2(lsum[i & 1], pr);
+                                packed[i] = pack_bf16(pr.x, pr.y);
+                            }
+                            tmem_st_x32(lane_base + col_s + half * 32, packed);
+                        }
+                    };
+                    if (need_mask) exp_and_store(std::true_type{});
+                    else exp_and_store(std::false_type{});
+                    const float l_tile = (lsum[0].x + lsum[0].y) + (lsum[1].x + lsum[1].y);
+                    l_run = l_run * alpha + l_tile;
+                }
                 tmem_st_wait();
                 tc_fence_before_sync();
-                mbar_arrive(&p_ready[t]);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&p_ready[t]);  // one arrival per warp
             }
 
             if (!failed && !warp_wait(&pv_done[t], (nt - 1) & 1)) failed = true;

@@ -51,7 +51,7 @@ struct AttnSmem {
     static constexpr int kVOff = kKOff + kKVStages * kTileBytes;
     static constexpr int kBarOff = kVOff + kKVStages * kTileBytes;
     // q_full, k/v full+empty per stage, s_full[2], p_ready[2], pv_done[2]
-    static constexpr int kNumBars = 1 + 4 * kKVStages + 6;
+    static constexpr int kNumBars = 2 + 4 * kKVStages + 8;
     static constexpr int kTotal = kBarOff + kNumBars * 8 + 16;
     static constexpr int kAlloc = kTotal + 1024;
 };
@@ -97,10 +97,17 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 struct AttnParams {
     __nv_bfloat16* out;
     const int32_t* lens;
-    int Hq, Hkv, Sq, Skv;
+    int B, Hq, Hkv, Sq, Skv;
     int mask_kind;
     float scale_log2;
     int* status;
+};
+
+// What one CTA needs to know about a work item (a pair of query tiles of one head).
+struct ItemInfo {
+    int q_pair, h, b, kvh, kvlen;
+    int n_tiles[kTilesPerCta];  // KV tiles visible to at least one row of each query tile (0: tile beyond Sq)
+    int n_max;
 };
 
 template <int D>
@@ -116,49 +123,64 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     uint8_t* sV = smem + L::kVOff;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBarOff);
     uint64_t* q_full = bars;
-    uint64_t* k_full = bars + 1;
+    uint64_t* q_empty = bars + 1;
+    uint64_t* k_full = bars + 2;
     uint64_t* k_empty = k_full + kKVStages;
     uint64_t* v_full = k_empty + kKVStages;
     uint64_t* v_empty = v_full + kKVStages;
     uint64_t* s_full = v_empty + kKVStages;  // [2] per query tile
     uint64_t* p_ready = s_full + 2;          // [2]
     uint64_t* pv_done = p_ready + 2;         // [2]
-    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(pv_done + 2);
+    uint64_t* o_free = pv_done + 2;          // [2]
+    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(o_free + 2);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_q_pairs = (p.Sq + kTilesPerCta * kBM - 1) / (kTilesPerCta * kBM);
-    // blockIdx.x runs over (batch, head), blockIdx.y over the tile pairs with the longest (causal) pair
-    // first: CTAs are dispatched in that order, so the long ones start first everywhere (LPT).
-    const int q_pair = num_q_pairs - 1 - blockIdx.y;
-    const int h = blockIdx.x % p.Hq, b = blockIdx.x / p.Hq;
-    const int kvh = h / (p.Hq / p.Hkv);
+    const int heads = p.Hq * p.B;
+    const int num_items = num_q_pairs * heads;
     const int causal_off = p.Skv - p.Sq;
     const bool causal = (p.mask_kind & FORGE_MASK_CAUSAL) != 0;
 
-    int kvlen = p.Skv;
-    if (p.mask_kind & FORGE_MASK_PADDING) kvlen = min(max(p.lens[b], 0), p.Skv);
-    // KV tiles that are visible to at least one row of each query tile (0 for a tile beyond Sq)
-    int n_tiles[kTilesPerCta];
-    int n_max = 0;
+    // Persistent schedule.  Items are ordered longest first (the last query-tile pair of every head, then
+    // the one before, ...); CTA c takes item c of every round of gridDim.x items, in alternating direction
+    // from round to round, which keeps the per-CTA sums of causal work close together.
+    auto item_of_round = [&](int r) {
+        const int c = (r & 1) ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)blockIdx.x;
+        return r * (int)gridDim.x + c;
+    };
+    auto decode = [&](int i) {
+        ItemInfo it;
+        it.q_pair = num_q_pairs - 1 - i / heads;
+        const int hb = i % heads;
+        it.h = hb % p.Hq;
+        it.b = hb / p.Hq;
+        it.kvh = it.h / (p.Hq / p.Hkv);
+        it.kvlen = p.Skv;
+        if (p.mask_kind & FORGE_MASK_PADDING) it.kvlen = min(max(p.lens[it.b], 0), p.Skv);
+        it.n_max = 0;
 #pragma unroll
-    for (int t = 0; t < kTilesPerCta; ++t) {
-        const int q0 = (q_pair * kTilesPerCta + t) * kBM;
-        int kv_end = kvlen;
-        if (causal) kv_end = min(kv_end, min(q0 + kBM, p.Sq) + causal_off);
-        if (q0 >= p.Sq) kv_end = 0;
-        kv_end = max(kv_end, 0);
-        n_tiles[t] = (kv_end + kBN - 1) / kBN;
-        n_max = max(n_max, n_tiles[t]);
-    }
+        for (int t = 0; t < kTilesPerCta; ++t) {
+            const int q0 = (it.q_pair * kTilesPerCta + t) * kBM;
+            int kv_end = it.kvlen;
+            if (causal) kv_end = min(kv_end, min(q0 + kBM, p.Sq) + causal_off);
+            if (q0 >= p.Sq) kv_end = 0;
+            kv_end = max(kv_end, 0);
+            it.n_tiles[t] = (kv_end + kBN - 1) / kBN;
+            it.n_max = max(it.n_max, it.n_tiles[t]);
+        }
+        return it;
+    };
 
     if (threadIdx.x == 0) {
         mbar_init(q_full, 1);
+        mbar_init(q_empty, 1);
         for (int i = 0; i < kKVStages; ++i) {
             mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1);
             mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1);
         }
         for (int t = 0; t < 2; ++t) {
-            mbar_init(&s_full[t], 1); mbar_init(&p_ready[t], kSoftmaxThreads / 32); mbar_init(&pv_done[t], 1);
+            mbar_init(&s_full[t], 1); mbar_init(&p_ready[t], kSoftmaxThreads / 32);
+            mbar_init(&pv_done[t], 1); mbar_init(&o_free[t], kSoftmaxThreads / 32);
         }
         fence_mbar_init();
         prefetch_tmap(&tmap_q); prefetch_tmap(&tmap_k); prefetch_tmap(&tmap_v);
@@ -176,121 +198,162 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     if (warp >= 8) {
       asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
       if (warp == 8) {
-        if (n_max > 0 && elect_one()) {
-            mbar_expect_tx(q_full, kTilesPerCta * L::kTileBytes);
+        // ------------------------------------------------------------------ TMA producer
+        if (elect_one()) {
+            int kvn = 0;     // KV tiles loaded so far (ring position), across items
+            int items = 0;   // items with work so far
+            for (int r = 0; !failed; ++r) {
+                const int i = item_of_round(r);
+                if (i >= num_items) break;
+                const ItemInfo it = decode(i);
+                if (it.n_max == 0) continue;
+                // the previous item's last S = Q K^T has been issued and completed: Q may be replaced
+                if (!mbar_wait(q_empty, (items & 1) ^ 1)) { failed = true; break; }
+                mbar_expect_tx(q_full, kTilesPerCta * L::kTileBytes);
 #pragma unroll
-            for (int t = 0; t < kTilesPerCta; ++t)
+                for (int t = 0; t < kTilesPerCta; ++t)
 #pragma unroll
-                for (int c = 0; c < D / 64; ++c)  // rows beyond Sq are zero-filled by the TMA unit
-                    tma_load_3d(sQ + t * L::kTileBytes + c * L::kChunkBytes, &tmap_q, q_full, c * 64,
-                                (q_pair * kTilesPerCta + t) * kBM, b * p.Hq + h);
-            for (int j = 0; j < n_max; ++j) {
-                const int st = j % kKVStages;
-                const uint32_t ph = (j / kKVStages) & 1;
-                if (!mbar_wait(&k_empty[st], ph ^ 1)) { failed = true; break; }
-                mbar_expect_tx(&k_full[st], L::kTileBytes);
+                    for (int c = 0; c < D / 64; ++c)  // rows beyond Sq are zero-filled by the TMA unit
+                        tma_load_3d(sQ + t * L::kTileBytes + c * L::kChunkBytes, &tmap_q, q_full, c * 64,
+                                    (it.q_pair * kTilesPerCta + t) * kBM, it.b * p.Hq + it.h);
+                for (int j = 0; j < it.n_max; ++j, ++kvn) {
+                    const int st = kvn % kKVStages;
+                    const uint32_t ph = (kvn / kKVStages) & 1;
+                    if (!mbar_wait(&k_empty[st], ph ^ 1)) { failed = true; break; }
+                    mbar_expect_tx(&k_full[st], L::kTileBytes);
 #pragma unroll
-                for (int c = 0; c < D / 64; ++c)
-                    tma_load_3d(sK + st * L::kTileBytes + c * L::kChunkBytes, &tmap_k, &k_full[st], c * 64, j * kBN,
-                                b * p.Hkv + kvh);
-                if (!mbar_wait(&v_empty[st], ph ^ 1)) { failed = true; break; }
-                mbar_expect_tx(&v_full[st], L::kTileBytes);
+                    for (int c = 0; c < D / 64; ++c)
+                        tma_load_3d(sK + st * L::kTileBytes + c * L::kChunkBytes, &tmap_k, &k_full[st], c * 64,
+                                    j * kBN, it.b * p.Hkv + it.kvh);
+                    if (!mbar_wait(&v_empty[st], ph ^ 1)) { failed = true; break; }
+                    mbar_expect_tx(&v_full[st], L::kTileBytes);
 #pragma unroll
-                for (int c = 0; c < D / 64; ++c)
-                    tma_load_3d(sV + st * L::kTileBytes + c * L::kChunkBytes, &tmap_v, &v_full[st], c * 64, j * kBN,
-                                b * p.Hkv + kvh);
+                    for (int c = 0; c < D / 64; ++c)
+                        tma_load_3d(sV + st * L::kTileBytes + c * L::kChunkBytes, &tmap_v, &v_full[st], c * 64,
+                                    j * kBN, it.b * p.Hkv + it.kvh);
+                }
+                ++items;
             }
         }
       } else if (warp == 9) {
-        if (n_max > 0 && elect_one()) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (elect_one()) {
             constexpr uint32_t idesc_s = make_idesc_bf16(kBM, kBN, false, false);
             constexpr uint32_t idesc_o = make_idesc_bf16(kBM, D, false, true);
             const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
-            int k_waited = -1, v_waited = -1;  // highest KV tile whose arrival has been observed
+            int kvbase = 0;                 // ring position of the item's first KV tile
+            int k_waited = -1, v_waited = -1;  // highest ring position whose arrival has been observed
+            int items = 0;                  // items with work so far
+            int its[kTilesPerCta] = {0, 0};     // tile iterations issued so far per query tile (barrier phases)
+            int used[kTilesPerCta] = {0, 0};    // items in which each query tile had work (phase of o_free)
 
-            // S_t(j) = Q_t K_j^T; the last tile that uses K_j releases its stage
-            auto issue_qk = [&](int t, int j) -> bool {
-                const int st = j % kKVStages;
-                if (j > k_waited) {
-                    if (!mbar_wait(&k_full[st], (j / kKVStages) & 1)) return false;
-                    k_waited = j;
-                }
-                tc_fence_after_sync();
-                const uint32_t kb = k_addr + st * L::kTileBytes, qb = q_addr + t * L::kTileBytes;
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = (kk / 4) * L::kChunkBytes + (kk % 4) * 32;
-                    mma_ss(tmem_base + kColS + t * kBN, make_smem_desc(qb + off, 16, 1024),
-                           make_smem_desc(kb + off, 16, 1024), idesc_s, kk != 0);
-                }
-                bool last = true;
-                for (int u = t + 1; u < kTilesPerCta; ++u) last = last && !(j < n_tiles[u]);
-                if (last) mma_commit(&k_empty[st]);
-                mma_commit(&s_full[t]);
-                return true;
-            };
-            // O_t += P_t(j) V_j with P_t read from tensor memory
-            auto issue_pv = [&](int t, int j) -> bool {
-                const int st = j % kKVStages;
-                if (!mbar_wait(&p_ready[t], j & 1)) return false;
-                if (j > v_waited) {
-                    if (!mbar_wait(&v_full[st], (j / kKVStages) & 1)) return false;
-                    v_waited = j;
-                }
-                tc_fence_after_sync();
-                const uint32_t vb = v_addr + st * L::kTileBytes;
-#pragma unroll
-                for (int kk = 0; kk < kBN / 16; ++kk) {
-                    // P: 16 keys = 8 columns of packed bf16 pairs.  V: MN-major, 16 keys = two 1024-byte
-                    // groups; the 64-wide chunks of D are 16 KB apart.
-                    mma_ts(tmem_base + kColO + t * D, tmem_base + kColS + t * kBN + kk * 8,
-                           make_smem_desc(vb + kk * 2048, L::kChunkBytes, 1024), idesc_o, (j | kk) != 0);
-                }
-                bool last = true;
-                for (int u = t + 1; u < kTilesPerCta; ++u) last = last && !(j < n_tiles[u]);
-                if (last) mma_commit(&v_empty[st]);
-                mma_commit(&pv_done[t]);
-                return true;
-            };
+            for (int r = 0; !failed; ++r) {
+                const int i = item_of_round(r);
+                if (i >= num_items) break;
+                const ItemInfo it = decode(i);
+                if (it.n_max == 0) continue;
 
-            if (!mbar_wait(q_full, 0)) failed = true;
-            for (int t = 0; t < kTilesPerCta && !failed; ++t)
-                if (n_tiles[t] > 0 && !issue_qk(t, 0)) failed = true;
-            for (int j = 0; j < n_max && !failed; ++j) {
-                for (int t = 0; t < kTilesPerCta && !failed; ++t) {
-                    if (j >= n_tiles[t]) continue;
-                    if (!issue_pv(t, j)) { failed = true; break; }
-                    if (j + 1 < n_tiles[t] && !issue_qk(t, j + 1)) { failed = true; break; }
+                int qk_issued = 0;
+                const int qk_total = it.n_tiles[0] + it.n_tiles[1];
+                // S_t(j) = Q_t K_j^T; the last tile that uses K_j releases its stage
+                auto issue_qk = [&](int t, int j) -> bool {
+                    const int g = kvbase + j, st = g % kKVStages;
+                    if (g > k_waited) {
+                        if (!mbar_wait(&k_full[st], (g / kKVStages) & 1)) return false;
+                        k_waited = g;
+                    }
+                    tc_fence_after_sync();
+                    const uint32_t kb = k_addr + st * L::kTileBytes, qb = q_addr + t * L::kTileBytes;
+#pragma unroll
+                    for (int kk = 0; kk < D / 16; ++kk) {
+                        const uint32_t off = (kk / 4) * L::kChunkBytes + (kk % 4) * 32;
+                        mma_ss(tmem_base + kColS + t * kBN, make_smem_desc(qb + off, 16, 1024),
+                               make_smem_desc(kb + off, 16, 1024), idesc_s, kk != 0);
+                    }
+                    bool last = true;
+                    for (int u = t + 1; u < kTilesPerCta; ++u) last = last && !(j < it.n_tiles[u]);
+                    if (last) mma_commit(&k_empty[st]);
+                    mma_commit(&s_full[t]);
+                    // the item's last S = Q K^T: once it completes, the next item's Q tiles may be loaded
+                    if (++qk_issued == qk_total) mma_commit(q_empty);
+                    return true;
+                };
+                // O_t += P_t(j) V_j with P_t read from tensor memory
+                auto issue_pv = [&](int t, int j) -> bool {
+                    const int g = kvbase + j, st = g % kKVStages;
+                    if (!mbar_wait(&p_ready[t], its[t] & 1)) return false;
+                    if (g > v_waited) {
+                        if (!mbar_wait(&v_full[st], (g / kKVStages) & 1)) return false;
+                        v_waited = g;
+                    }
+                    // the first product of an item overwrites O_t: the previous item's epilogue must have read it
+                    if (j == 0 && !mbar_wait(&o_free[t], (used[t] & 1) ^ 1)) return false;
+                    tc_fence_after_sync();
+                    const uint32_t vb = v_addr + st * L::kTileBytes;
+#pragma unroll
+                    for (int kk = 0; kk < kBN / 16; ++kk) {
+                        // P: 16 keys = 8 columns of packed bf16 pairs.  V: MN-major, 16 keys = two 1024-byte
+                        // groups; the 64-wide chunks of D are 16 KB apart.
+                        mma_ts(tmem_base + kColO + t * D, tmem_base + kColS + t * kBN + kk * 8,
+                               make_smem_desc(vb + kk * 2048, L::kChunkBytes, 1024), idesc_o, (j | kk) != 0);
+                    }
+                    bool last = true;
+                    for (int u = t + 1; u < kTilesPerCta; ++u) last = last && !(j < it.n_tiles[u]);
+                    if (last) mma_commit(&v_empty[st]);
+                    mma_commit(&pv_done[t]);
+                    ++its[t];
+                    return true;
+                };
+
+                if (!mbar_wait(q_full, items & 1)) { failed = true; break; }
+                for (int t = 0; t < kTilesPerCta && !failed; ++t)
+                    if (it.n_tiles[t] > 0 && !issue_qk(t, 0)) failed = true;
+                for (int j = 0; j < it.n_max && !failed; ++j) {
+                    for (int t = 0; t < kTilesPerCta && !failed; ++t) {
+                        if (j >= it.n_tiles[t]) continue;
+                        if (!issue_pv(t, j)) { failed = true; break; }
+                        if (j + 1 < it.n_tiles[t] && !issue_qk(t, j + 1)) { failed = true; break; }
+                    }
                 }
+                for (int t = 0; t < kTilesPerCta; ++t) used[t] += it.n_tiles[t] > 0;
+                kvbase += it.n_max;
+                ++items;
             }
         }
       }
     } else {
+        // ------------------------------------------------------------------ softmax / rescale / epilogue
         asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
-        const int t = warp >> 2;  // query tile of this warp group
-        const int quarter = warp & 3;   // TMEM lane quarter this warp may access
+        const int t = warp >> 2;       // query tile of this warp group
+        const int quarter = warp & 3;  // TMEM lane quarter this warp may access
         const int row = quarter * 32 + lane;
-        const int q0 = (q_pair * kTilesPerCta + t) * kBM;
-        const int qi = q0 + row;
-        const int nt = n_tiles[t];
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
         const uint32_t col_s = kColS + t * kBN, col_o = kColO + t * D;
         const float sl2 = p.scale_log2;
-        __nv_bfloat16* orow = p.out + ((size_t)(b * p.Hq + h) * p.Sq + qi) * D;
+        int its = 0;  // tile iterations done so far (barrier phases run across items)
 
-        if (nt == 0) {
-            if (qi < p.Sq) {
+        for (int r = 0; !failed; ++r) {
+            const int i = item_of_round(r);
+            if (i >= num_items) break;
+            const ItemInfo it = decode(i);
+            const int q0 = (it.q_pair * kTilesPerCta + t) * kBM;
+            const int qi = q0 + row;
+            const int nt = it.n_tiles[t];
+            __nv_bfloat16* orow = p.out + ((size_t)(it.b * p.Hq + it.h) * p.Sq + qi) * D;
+            if (nt == 0) {  // no visible key for any row of this tile (or the tile lies beyond Sq)
+                if (qi < p.Sq) {
 #pragma unroll
-                for (int c = 0; c < D / 8; ++c) reinterpret_cast<uint4*>(orow)[c] = make_uint4(0, 0, 0, 0);
+                    for (int c = 0; c < D / 8; ++c) reinterpret_cast<uint4*>(orow)[c] = make_uint4(0, 0, 0, 0);
+                }
+                continue;
             }
-        } else {
             float m_run = -INFINITY;  // running maximum of the raw scores (reference of the exponentials)
             float l_run = 0.f;
             const int row_limit = causal ? qi + causal_off : 0x7fffffff;  // last visible key of this row
-            for (int j = 0; j < nt; ++j) {
+            for (int j = 0; j < nt; ++j, ++its) {
                 // S_t(j) is complete, and so is every MMA issued before it: O_t holds all earlier P V
                 // products and P_t(j-1) has been consumed.
-                if (!warp_wait(&s_full[t], j & 1)) { failed = true; break; }
+                if (!warp_wait(&s_full[t], its & 1)) { failed = true; break; }
                 tc_fence_after_sync();
                 float s[kBN];
 #pragma unroll
@@ -303,9 +366,9 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 tmem_ld_wait();
 
                 const int j0 = j * kBN;
-                const bool need_mask = (j0 + kBN > kvlen) || (causal && (j0 + kBN - 1 > q0 + causal_off));
+                const bool need_mask = (j0 + kBN > it.kvlen) || (causal && (j0 + kBN - 1 > q0 + causal_off));
                 if (need_mask) {
-                    const int lim = min(kvlen - 1, row_limit) - j0;  // last visible column of this tile
+                    const int lim = min(it.kvlen - 1, row_limit) - j0;  // last visible column of this tile
 #pragma unroll
                     for (int i = 0; i < kBN; ++i) s[i] = (i <= lim) ? s[i] : -INFINITY;
                 }
@@ -411,27 +474,31 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&p_ready[t]);  // one arrival per warp
             }
-
-            if (!failed && !warp_wait(&pv_done[t], (nt - 1) & 1)) failed = true;
-            if (!failed) {
-                tc_fence_after_sync();
+            if (failed) break;
+            if (!warp_wait(&pv_done[t], (its - 1) & 1)) { failed = true; break; }
+            tc_fence_after_sync();
+            // O_t -> registers, then hand O_t back to the MMA warp before the stores go out
+            uint32_t o[D];
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t rr[32];
+                tmem_ld_x32(lane_base + col_o + c * 32, rr);
+#pragma unroll
+                for (int k = 0; k < 32; ++k) o[c * 32 + k] = rr[k];
+            }
+            tmem_ld_wait();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&o_free[t]);
+            if (qi < p.Sq) {
                 const float inv = l_run > 0.f ? 1.f / l_run : 0.f;  // no visible key: zeros
 #pragma unroll
-                for (int c = 0; c < D / 32; ++c) {
-                    uint32_t r[32];
-                    tmem_ld_x32(lane_base + col_o + c * 32, r);
-                    tmem_ld_wait();
-                    if (qi < p.Sq) {
+                for (int c = 0; c < D / 8; ++c) {
+                    uint32_t w[4];
 #pragma unroll
-                        for (int v4 = 0; v4 < 4; ++v4) {
-                            uint32_t w[4];
-#pragma unroll
-                            for (int i = 0; i < 4; ++i)
-                                w[i] = pack_bf16(__uint_as_float(r[v4 * 8 + 2 * i]) * inv,
-                                                 __uint_as_float(r[v4 * 8 + 2 * i + 1]) * inv);
-                            reinterpret_cast<uint4*>(orow + c * 32)[v4] = make_uint4(w[0], w[1], w[2], w[3]);
-                        }
-                    }
+                    for (int k = 0; k < 4; ++k)
+                        w[k] = pack_bf16(__uint_as_float(o[c * 8 + 2 * k]) * inv, __uint_as_float(o[c * 8 + 2 * k + 1]) * inv);
+                    reinterpret_cast<uint4*>(orow)[c] = make_uint4(w[0], w[1], w[2], w[3]);
                 }
             }
         }
@@ -469,14 +536,18 @@ int launch_attn(const void* q, const void* k, const void* v, void* out, int B, i
     AttnParams p;
     p.out = static_cast<__nv_bfloat16*>(out);
     p.lens = lens;
-    p.Hq = Hq; p.Hkv = Hkv; p.Sq = Sq; p.Skv = Skv;
+    p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.Sq = Sq; p.Skv = Skv;
     p.mask_kind = mask_kind;
     p.scale_log2 = scale * 1.4426950408889634f;
     p.status = device_status_word();
     if (!p.status) return FORGE_ERR_CUDA;
     auto kernel = attn_bf16_kernel<D>;
     FORGE_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kAlloc));
-    const dim3 grid(Hq * B, (Sq + kTilesPerCta * kBM - 1) / (kTilesPerCta * kBM), 1);
+    int dev = 0, sms = 0;
+    FORGE_CUDA_TRY(cudaGetDevice(&dev));
+    FORGE_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const long long items = (long long)Hq * B * ((Sq + kTilesPerCta * kBM - 1) / (kTilesPerCta * kBM));
+    const int grid = items < sms ? (int)items : sms;
     kernel<<<grid, kThreads, L::kAlloc, s>>>(tq, tk, tv, p);
     return finish_launch(1);
 }
@@ -490,7 +561,7 @@ extern "C" int forge_attn_fused(const void* q, const void* k, const void* v, voi
     using namespace forge;
     int st = check_attn_args(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens);
     if (st != FORGE_OK) return st;
-    if ((long long)Hq * B > 2147483647LL || (Sq + 255) / 256 > 65535) return FORGE_ERR_UNSUPPORTED;
+    if ((long long)Hq * B * ((Sq + 255) / 256) > 2147483647LL) return FORGE_ERR_UNSUPPORTED;
     if (!(scale >= 0.f)) return FORGE_ERR_UNSUPPORTED;  // the running maximum is taken on unscaled scores
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     return D == 64 ? launch_attn<64>(q, k, v, out, B, Hq, Hkv, Sq, Skv, mask_kind, lens, scale, s)

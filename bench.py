@@ -37,7 +37,7 @@ WORKLOAD = ("GPT-2-small layer (causal attention B8 H12 S1024 D64 + c_fc GEMM 81
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (None once the kernel has changed since the capture).
-NCU_TRAFFIC_BYTES = {"attention": None, "linear": None, "decode": None}
+NCU_TRAFFIC_BYTES = {"attention": 38003968, "linear": 18797824, "decode": 147300000}
 
 
 def load_peaks():
@@ -321,6 +321,48 @@ def run_gpu(args):
         "peak_source": f"{peak_src} ({'sustained' if sustained and d['bound'] == 'tensor' else 'burst'})",
     }
 
+    # ---- the other configurations, each timed on its own after the step loop (not part of `value`):
+    # 8B-class GQA prefill (the shape where the tensor-core target applies), the padded encoder batch and
+    # the fp32 GPT-2-small case (latency).  Device-drawn inputs of the workloads' shapes and distributions.
+    other = None
+    if rank == 0 and not args.no_other_configs:
+        def timed(fn, iters):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(iters):
+                fn()
+            b_.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b_) / iters
+
+        other = {}
+        B4, Hq4, Hkv4, S4, D4 = 4, 32, 8, 2048, 128
+        q4, k4, v4 = randn((B4, Hq4, S4, D4)), randn((B4, Hkv4, S4, D4)), randn((B4, Hkv4, S4, D4))
+        o4 = torch.empty_like(q4)
+        ms = timed(lambda: binding.attn_fused(q4, k4, v4, wl.MASK_CAUSAL, None, D4 ** -0.5, out=o4), 20)
+        fl = 4 * D4 * B4 * Hq4 * (S4 * (S4 + 1) // 2)
+        other["cfg4_gqa_prefill_B4_32/8_S2048_D128"] = {
+            "ms": ms, "tflops": fl / ms / 1e9, "frac_of_bf16_peak": fl / ms / 1e9 / peaks["bf16_tflops"],
+            "flops": fl, "l2": "warm (inputs 101 MB, reused across calls)"}
+        del q4, k4, v4, o4
+        B3, H3, S3, D3 = 32, 12, 128, 64
+        lens3 = torch.from_numpy(wl.cfg3_encoder().lens).to(dev)
+        q3, k3, v3 = randn((B3, H3, S3, D3)), randn((B3, H3, S3, D3)), randn((B3, H3, S3, D3))
+        o3 = torch.empty_like(q3)
+        ms = timed(lambda: binding.attn_fused(q3, k3, v3, wl.MASK_PADDING, lens3, 0.125, out=o3), 50)
+        sl = int(lens3.sum().item())
+        other["cfg3_encoder_padding_B32_H12_S128_D64"] = {
+            "ms": ms, "tflops": 393216 * sl / ms / 1e9, "gbs": (12582912 + 3072 * sl) / ms / 1e6, "sum_lens": sl,
+            "l2": "warm"}
+        q1 = torch.randn((1, 12, 128, 64), generator=gen, device=dev)
+        k1, v1 = torch.randn_like(q1), torch.randn_like(q1)
+        o1 = torch.empty_like(q1)
+        ms = timed(lambda: binding.attn_fused_f32(q1, k1, v1, wl.MASK_CAUSAL, None, 0.125, out=o1), 50)
+        other["cfg1_gpt2_fp32_B1_H12_S128_D64"] = {"latency_us": ms * 1e3, "l2": "warm"}
+
     # ---- spot check of set 0 against values the oracle computes one by one (not timed)
     spot = None
     if rank == 0 and base is not None:
@@ -391,7 +433,7 @@ def run_gpu(args):
                              f"more than the 126 MB L2 between two uses of any buffer)",
                        "sum_lens": int(dec.lens.sum())},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-            "roofline": roofline, "cpu_baseline": base, "kernels": kern,
+            "roofline": roofline, "cpu_baseline": base, "kernels": kern, "other_configs": other,
             "decode_hbm": {"value": kern["decode"]["gbs"], "unit": "GB/s", "frac_of_measured_peak": kern["decode"]["frac"]},
             "wall_ms_per_step": wall / args.steps * 1e3, "spot_check": spot,
         }
@@ -409,6 +451,7 @@ def main():
     ap.add_argument("--impl", default="forge", choices=["forge", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-other-configs", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

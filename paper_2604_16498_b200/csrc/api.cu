@@ -17,6 +17,18 @@ __device__ int g_device_status = 0;
 void set_last_cuda_error(cudaError_t e) { tl_last_cuda_error = static_cast<int>(e); }
 void count_launch(int n) { g_launches.fetch_add(static_cast<unsigned long long>(n), std::memory_order_relaxed); }
 
+int sm_count() {
+    static int cache[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    if (!cache[dev]) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+        cache[dev] = n;
+    }
+    return cache[dev];
+}
+
 int* device_status_word() {
     // Resolved per device: the symbol has one instance per device that loads the module.
     int dev = 0;

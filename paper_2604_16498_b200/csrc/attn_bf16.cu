@@ -542,10 +542,9 @@ int launch_attn(const void* q, const void* k, const void* v, void* out, int B, i
     p.status = device_status_word();
     if (!p.status) return FORGE_ERR_CUDA;
     auto kernel = attn_bf16_kernel<D>;
-    FORGE_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kAlloc));
-    int dev = 0, sms = 0;
-    FORGE_CUDA_TRY(cudaGetDevice(&dev));
-    FORGE_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    FORGE_SET_SMEM_ONCE(kernel, L::kAlloc);
+    const int sms = sm_count();
+    if (sms <= 0) return FORGE_ERR_CUDA;
     const long long items = (long long)Hq * B * ((Sq + kTilesPerCta * kBM - 1) / (kTilesPerCta * kBM));
     const int grid = items < sms ? (int)items : sms;
     kernel<<<grid, kThreads, L::kAlloc, s>>>(tq, tk, tv, p);

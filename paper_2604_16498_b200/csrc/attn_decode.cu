@@ -358,10 +358,9 @@ int launch_split(const void* q, const void* kc, const void* vc, const int32_t* l
                  int B, int Hq, int Hkv, int Smax, int num_splits, float scale_log2, cudaStream_t s) {
     constexpr int kSmem = kWarps * kWarpRingBytes;
     auto kernel = decode_split_kernel<D, G>;
-    FORGE_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem));
-    int dev = 0, sms = 0;
-    FORGE_CUDA_TRY(cudaGetDevice(&dev));
-    FORGE_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    FORGE_SET_SMEM_ONCE(kernel, kSmem);
+    const int sms = sm_count();
+    if (sms <= 0) return FORGE_ERR_CUDA;
     const long long items = (long long)B * Hkv * num_splits;
     const long long ctas = (items + kWarps - 1) / kWarps;
     const int grid = ctas < sms ? (int)ctas : sms;

@@ -27,6 +27,23 @@ inline int finish_launch(int nkernels) {
     return FORGE_OK;
 }
 
+// Number of SMs of the current device (looked up once per device).
+int sm_count();
+
+// Opts a kernel in to `bytes` of dynamic shared memory once per device and call site (the attribute
+// call costs microseconds, which matters for the latency-bound shapes).
+#define FORGE_SET_SMEM_ONCE(kernel, bytes)                                                          \
+    do {                                                                                            \
+        static bool done__[64] = {};                                                                \
+        int dev__ = 0;                                                                              \
+        FORGE_CUDA_TRY(cudaGetDevice(&dev__));                                                      \
+        if (dev__ < 0 || dev__ >= 64 || !done__[dev__]) {                                           \
+            FORGE_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                                                (int)(bytes)));                                     \
+            if (dev__ >= 0 && dev__ < 64) done__[dev__] = true;                                     \
+        }                                                                                           \
+    } while (0)
+
 #define FORGE_CUDA_TRY(expr)                                         \
     do {                                                             \
         cudaError_t e__ = (expr);                                    \

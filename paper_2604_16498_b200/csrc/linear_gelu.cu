@@ -242,11 +242,10 @@ int launch_linear(const void* x, const void* w, const void* b, void* y, int M, i
     }
     int* status = device_status_word();
     if (!status) return FORGE_ERR_CUDA;
-    int dev = 0, sms = 0;
-    FORGE_CUDA_TRY(cudaGetDevice(&dev));
-    FORGE_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const int sms = sm_count();
+    if (sms <= 0) return FORGE_ERR_CUDA;
     auto kernel = linear_bias_gelu_kernel<BN, STAGES>;
-    FORGE_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kAlloc));
+    FORGE_SET_SMEM_ONCE(kernel, L::kAlloc);
     const int tiles = ((M + kBM - 1) / kBM) * ((N + BN - 1) / BN);
     const int grid = tiles < sms ? tiles : sms;
     kernel<<<grid, kThreads, L::kAlloc, s>>>(tmap_x, tmap_w, tmap_y, static_cast<const __nv_bfloat16*>(b), M, N, K,

@@ -192,6 +192,23 @@ def run_reference(args):
     return 0
 
 
+# ----------------------------------------------------------------------------- multi-rank helpers
+def max_over_ranks(ms: float, device=None, distributed: bool = False) -> float:
+    """The slowest rank's time: every rank passes its own device time, all get the maximum."""
+    if not distributed:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_rate(world: int, units_per_rank: float, ms: float) -> float:
+    """Units all ranks processed per second (every rank does `units_per_rank`; weak scaling)."""
+    return world * units_per_rank / (ms * 1e-3)
+
+
 # ----------------------------------------------------------------------------- GPU arm
 def run_gpu(args):
     import torch
@@ -288,14 +305,11 @@ def run_gpu(args):
     dev_ms = evs[0][0].elapsed_time(evs[-1][3])          # first kernel start to last kernel end
     k_ms = [float(np.mean([e[i].elapsed_time(e[i + 1]) for e in evs])) for i in range(3)]
 
-    t = torch.tensor([dev_ms], device=dev, dtype=torch.float64)
-    if distributed:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    dev_ms = float(t.item())
+    dev_ms = max_over_ranks(dev_ms, dev, distributed)
     ms_per_step = dev_ms / args.steps
 
     step_flops = att.flops() + lin.flops() + dec.flops()
-    value = world * step_flops / (ms_per_step * 1e-3) / 1e12
+    value = whole_job_rate(world, step_flops, ms_per_step) / 1e12
 
     # ---- per-kernel numbers and the roofline of the dominant one
     sustained = dev_ms >= 1000.0
@@ -414,14 +428,12 @@ def run_gpu(args):
             host_step()
         e1.record()
         barrier()
-        te = torch.tensor([e0.elapsed_time(e1)], device=dev, dtype=torch.float64)
-        if distributed:
-            dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        e2e_ms = max_over_ranks(e0.elapsed_time(e1), dev, distributed)
         h2d = sum(pin[k].numel() * 2 for k in pin) + dec.B * 4
         d2h = sum(outs[k].numel() * 2 for k in outs)
-        e2e = {"value": world * step_flops / (float(te.item()) / e_steps * 1e-3) / 1e12, "unit": "TFLOP/s",
+        e2e = {"value": world * step_flops / (e2e_ms / e_steps * 1e-3) / 1e12, "unit": "TFLOP/s",
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e_steps,
-               "ms_per_step": float(te.item()) / e_steps}
+               "ms_per_step": e2e_ms / e_steps}
 
     if rank == 0:
         line = {

@@ -30,20 +30,30 @@ def build(force: bool = False) -> str:
     return _LIB
 
 
+def _configure(lib):
+    i = ctypes.c_int
+    lib.forge_ref_attn.argtypes = [_dp, _dp, _dp, _dp, i, i, i, i, i, i, i, _ip, ctypes.c_double]
+    lib.forge_ref_attn_probs.argtypes = [_dp, _dp, _dp, _dp, _dp, i, i, i, i, i, i, i, _ip, ctypes.c_double]
+    lib.forge_ref_attn_decode.argtypes = [_dp, _dp, _dp, _dp, i, i, i, i, i, _ip, ctypes.c_double]
+    lib.forge_ref_linear_bias_gelu.argtypes = [_dp, _dp, _dp, _dp, i, i, i]
+    lib.forge_ref_gelu_tanh.argtypes = [ctypes.c_double]
+    lib.forge_ref_gelu_tanh.restype = ctypes.c_double
+    lib.forge_ref_num_threads.restype = i
+    return lib
+
+
 def _load():
     global _lib
     if _lib is None:
-        lib = ctypes.CDLL(build())
-        i = ctypes.c_int
-        lib.forge_ref_attn.argtypes = [_dp, _dp, _dp, _dp, i, i, i, i, i, i, i, _ip, ctypes.c_double]
-        lib.forge_ref_attn_probs.argtypes = [_dp, _dp, _dp, _dp, _dp, i, i, i, i, i, i, i, _ip, ctypes.c_double]
-        lib.forge_ref_attn_decode.argtypes = [_dp, _dp, _dp, _dp, i, i, i, i, i, _ip, ctypes.c_double]
-        lib.forge_ref_linear_bias_gelu.argtypes = [_dp, _dp, _dp, _dp, i, i, i]
-        lib.forge_ref_gelu_tanh.argtypes = [ctypes.c_double]
-        lib.forge_ref_gelu_tanh.restype = ctypes.c_double
-        lib.forge_ref_num_threads.restype = i
-        _lib = lib
+        _lib = _configure(ctypes.CDLL(build()))
     return _lib
+
+
+def use_library(path):
+    """Points the binding at another build of the oracle (used by the tests that plant mistakes in a
+    copy of the C source to see that the pins catch them).  ``None`` restores the real one."""
+    global _lib
+    _lib = None if path is None else _configure(ctypes.CDLL(path))
 
 
 def _f64(a):

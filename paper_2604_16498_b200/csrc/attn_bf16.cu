@@ -49,9 +49,10 @@ struct AttnSmem {
     static constexpr int kQOff = 0;
     static constexpr int kKOff = kQOff + kTilesPerCta * kTileBytes;
     static constexpr int kVOff = kKOff + kKVStages * kTileBytes;
-    static constexpr int kBarOff = kVOff + kKVStages * kTileBytes;
+    static constexpr int kOutOff = kVOff + kKVStages * kTileBytes;  // output staging: 128 rows x 64 bf16 per query tile
+    static constexpr int kBarOff = kOutOff + kTilesPerCta * kChunkBytes;
     // q_full, k/v full+empty per stage, s_full[2], p_ready[2], pv_done[2]
-    static constexpr int kNumBars = 2 + 4 * kKVStages + 8;
+    static constexpr int kNumBars = 2 + 4 * kKVStages + 10;
     static constexpr int kTotal = kBarOff + kNumBars * 8 + 16;
     static constexpr int kAlloc = kTotal + 1024;
 };
@@ -113,7 +114,8 @@ struct ItemInfo {
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
-                 const __grid_constant__ CUtensorMap tmap_v, const AttnParams p) {
+                 const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_o,
+                 const AttnParams p) {
     using L = AttnSmem<D>;
     constexpr int kKVStages = L::kKVStages;
     extern __shared__ uint8_t smem_raw[];
@@ -132,7 +134,8 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     uint64_t* p_ready = s_full + 2;          // [2]
     uint64_t* pv_done = p_ready + 2;         // [2]
     uint64_t* o_free = pv_done + 2;          // [2]
-    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(o_free + 2);
+    uint64_t* wg_bar = o_free + 2;           // [2] meeting point of a tile's four softmax warps
+    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(wg_bar + 2);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int num_q_pairs = (p.Sq + kTilesPerCta * kBM - 1) / (kTilesPerCta * kBM);
@@ -181,9 +184,10 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
         for (int t = 0; t < 2; ++t) {
             mbar_init(&s_full[t], 1); mbar_init(&p_ready[t], kSoftmaxThreads / 32);
             mbar_init(&pv_done[t], 1); mbar_init(&o_free[t], kSoftmaxThreads / 32);
+            mbar_init(&wg_bar[t], kSoftmaxThreads / 32);
         }
         fence_mbar_init();
-        prefetch_tmap(&tmap_q); prefetch_tmap(&tmap_k); prefetch_tmap(&tmap_v);
+        prefetch_tmap(&tmap_q); prefetch_tmap(&tmap_k); prefetch_tmap(&tmap_v); prefetch_tmap(&tmap_o);
     }
     if (warp == 9) {
         tmem_alloc(tmem_base_slot, kTmemCols);
@@ -327,10 +331,20 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
         const int t = warp >> 2;       // query tile of this warp group
         const int quarter = warp & 3;  // TMEM lane quarter this warp may access
         const int row = quarter * 32 + lane;
+        const int wg_tid = threadIdx.x & 127;  // index inside the warp group of this tile
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
         const uint32_t col_s = kColS + t * kBN, col_o = kColO + t * D;
         const float sl2 = p.scale_log2;
         int its = 0;  // tile iterations done so far (barrier phases run across items)
+        uint32_t wg_phase = 0;
+        // the four warps of this tile meet on an mbarrier: unlike bar.sync, the wait is bounded
+        auto wg_sync = [&]() -> bool {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&wg_bar[t]);
+            const bool ok = warp_wait(&wg_bar[t], wg_phase);
+            wg_phase ^= 1;
+            return ok;
+        };
 
         for (int r = 0; !failed; ++r) {
             const int i = item_of_round(r);
@@ -490,18 +504,35 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&o_free[t]);
-            if (qi < p.Sq) {
+            // O / l as bf16 through a 128-byte-swizzled staging buffer and one TMA store per 64 columns
+            // (rows beyond Sq are clipped by the TMA unit).  The store drains while the next item starts.
+            {
                 const float inv = l_run > 0.f ? 1.f / l_run : 0.f;  // no visible key: zeros
+                uint8_t* stage_out = smem + L::kOutOff + t * L::kChunkBytes;
 #pragma unroll
-                for (int c = 0; c < D / 8; ++c) {
-                    uint32_t w[4];
+                for (int cb = 0; cb < D / 64; ++cb) {
+                    if (wg_tid == 0) tma_store_wait_read<0>();  // the previous store has read the buffer
+                    if (!wg_sync()) { failed = true; break; }
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        w[k] = pack_bf16(__uint_as_float(o[c * 8 + 2 * k]) * inv, __uint_as_float(o[c * 8 + 2 * k + 1]) * inv);
-                    reinterpret_cast<uint4*>(orow)[c] = make_uint4(w[0], w[1], w[2], w[3]);
+                    for (int c = 0; c < 8; ++c) {
+                        uint32_t w[4];
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            w[k] = pack_bf16(__uint_as_float(o[cb * 64 + c * 8 + 2 * k]) * inv,
+                                             __uint_as_float(o[cb * 64 + c * 8 + 2 * k + 1]) * inv);
+                        *reinterpret_cast<uint4*>(stage_out + row * 128 + ((c ^ (row & 7)) << 4)) =
+                            make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                    fence_proxy_async_smem();
+                    if (!wg_sync()) { failed = true; break; }
+                    if (wg_tid == 0) {
+                        tma_store_3d(&tmap_o, stage_out, cb * 64, q0, it.b * p.Hq + it.h);
+                        tma_store_commit();
+                    }
                 }
             }
         }
+        if (wg_tid == 0) tma_store_wait_all<0>();  // every output tile has left shared memory and is written
     }
 
     if (failed) {
@@ -533,6 +564,12 @@ int launch_attn(const void* q, const void* k, const void* v, void* out, int B, i
         if (!encode_tmap_bf16_sw128(&tk, k, 3, dims, strides, box)) return FORGE_ERR_CUDA;
         if (!encode_tmap_bf16_sw128(&tv, v, 3, dims, strides, box)) return FORGE_ERR_CUDA;
     }
+    CUtensorMap to;
+    {
+        const uint64_t dims[3] = {(uint64_t)D, (uint64_t)Sq, (uint64_t)B * Hq};
+        const uint64_t strides[2] = {(uint64_t)D * 2, (uint64_t)Sq * D * 2};
+        if (!encode_tmap_bf16_sw128(&to, out, 3, dims, strides, box)) return FORGE_ERR_CUDA;
+    }
     AttnParams p;
     p.out = static_cast<__nv_bfloat16*>(out);
     p.lens = lens;
@@ -547,7 +584,7 @@ int launch_attn(const void* q, const void* k, const void* v, void* out, int B, i
     if (sms <= 0) return FORGE_ERR_CUDA;
     const long long items = (long long)Hq * B * ((Sq + kTilesPerCta * kBM - 1) / (kTilesPerCta * kBM));
     const int grid = items < sms ? (int)items : sms;
-    kernel<<<grid, kThreads, L::kAlloc, s>>>(tq, tk, tv, p);
+    kernel<<<grid, kThreads, L::kAlloc, s>>>(tq, tk, tv, to, p);
     return finish_launch(1);
 }
 

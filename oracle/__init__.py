@@ -8,6 +8,12 @@ from .ref import (  # noqa: F401
     attn_probs,
     attn_decode,
     linear_bias_gelu,
+    linear_act,
+    ACT_GELU_TANH,
+    ACT_GELU_ERF,
+    ACT_RELU,
+    ACT_SILU,
+    ACT_NONE,
     gelu_tanh,
     num_threads,
     build,

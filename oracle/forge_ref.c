@@ -185,6 +185,43 @@ int forge_ref_linear_bias_gelu(const double *x, const double *w, const double *b
     return 0;
 }
 
+/*
+ * The other patterns the operator-fusion pass produces (Section 4.3 "Pass 5": linear+relu, linear+gelu,
+ * linear+silu, and mm+add, a residual addition after a raw matrix multiply):
+ *     y[m, n] = act(b[n] + sum_k x[m, k] W(k, n)) + r[m, n]
+ * act: 0 tanh-GELU, 1 erf-GELU (0.5 z (1 + erf(z / sqrt 2))), 2 ReLU, 3 SiLU (z / (1 + e^-z)), 4 identity.
+ * w_layout: 0 = w stored [K, N]; 1 = w stored [N, K], the [out, in] layout of the listing's Linear.
+ * b (length N) and r ([M, N]) may be NULL and then contribute nothing.
+ */
+int forge_ref_linear_act(const double *x, const double *w, const double *b, const double *r, double *y,
+                         int M, int N, int K, int act, int w_layout)
+{
+    if (!x || !w || !y || M <= 0 || N <= 0 || K <= 0) return 1;
+    if (act < 0 || act > 4 || w_layout < 0 || w_layout > 1) return 1;
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        for (int n = 0; n < N; ++n) {
+            double z = 0.0;
+            for (int kk = 0; kk < K; ++kk) {
+                const double wkn = w_layout == 0 ? w[(size_t)kk * N + n] : w[(size_t)n * K + kk];
+                z += x[(size_t)m * K + kk] * wkn;
+            }
+            if (b) z += b[n];
+            double a;
+            switch (act) {
+            case 0: a = forge_ref_gelu_tanh(z); break;
+            case 1: a = 0.5 * z * (1.0 + erf(z / sqrt(2.0))); break;
+            case 2: a = z > 0.0 ? z : 0.0; break;
+            case 3: a = z / (1.0 + exp(-z)); break;
+            default: a = z; break;
+            }
+            if (r) a += r[(size_t)m * N + n];
+            y[(size_t)m * N + n] = a;
+        }
+    }
+    return 0;
+}
+
 /* Number of OpenMP threads the loops above will use (1 when built without OpenMP). */
 #ifdef _OPENMP
 #include <omp.h>

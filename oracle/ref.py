@@ -36,6 +36,7 @@ def _configure(lib):
     lib.forge_ref_attn_probs.argtypes = [_dp, _dp, _dp, _dp, _dp, i, i, i, i, i, i, i, _ip, ctypes.c_double]
     lib.forge_ref_attn_decode.argtypes = [_dp, _dp, _dp, _dp, i, i, i, i, i, _ip, ctypes.c_double]
     lib.forge_ref_linear_bias_gelu.argtypes = [_dp, _dp, _dp, _dp, i, i, i]
+    lib.forge_ref_linear_act.argtypes = [_dp, _dp, _dp, _dp, _dp, i, i, i, i, i]
     lib.forge_ref_gelu_tanh.argtypes = [ctypes.c_double]
     lib.forge_ref_gelu_tanh.restype = ctypes.c_double
     lib.forge_ref_num_threads.restype = i
@@ -121,6 +122,26 @@ def linear_bias_gelu(x, w, b):
     y = np.empty((M, N), dtype=np.float64)
     _check(_load().forge_ref_linear_bias_gelu(_ptr(x), _ptr(w), _ptr(b), _ptr(y), M, N, K),
            "forge_ref_linear_bias_gelu")
+    return y
+
+
+ACT_GELU_TANH, ACT_GELU_ERF, ACT_RELU, ACT_SILU, ACT_NONE = range(5)
+
+
+def linear_act(x, w, b=None, residual=None, act=ACT_GELU_TANH, w_layout=0):
+    """act(x W + b) + residual; w is [K,N] (w_layout 0) or [N,K] (w_layout 1); b, residual optional."""
+    x, w = _f64(x), _f64(w)
+    M, K = x.shape
+    N = w.shape[1] if w_layout == 0 else w.shape[0]
+    assert w.shape == ((K, N) if w_layout == 0 else (N, K))
+    b = None if b is None else _f64(b)
+    residual = None if residual is None else _f64(residual)
+    assert b is None or b.shape == (N,)
+    assert residual is None or residual.shape == (M, N)
+    y = np.empty((M, N), dtype=np.float64)
+    _check(_load().forge_ref_linear_act(_ptr(x), _ptr(w), None if b is None else _ptr(b),
+                                        None if residual is None else _ptr(residual), _ptr(y), M, N, K,
+                                        int(act), int(w_layout)), "forge_ref_linear_act")
     return y
 
 

@@ -85,3 +85,50 @@ def test_linear_against_torch_library():
 def test_linear_invalid_arguments():
     with pytest.raises((ValueError, AssertionError)):
         oracle.linear_bias_gelu(np.zeros((2, 3)), np.zeros((4, 2)), np.zeros(2))
+
+
+# ---- the other operator-fusion patterns: linear+relu, linear+silu, erf-GELU, mm+add, [N,K] weights
+ACTS = {
+    oracle.ACT_GELU_TANH: lambda t: torch.nn.functional.gelu(t, approximate="tanh"),
+    oracle.ACT_GELU_ERF: lambda t: torch.nn.functional.gelu(t),
+    oracle.ACT_RELU: torch.relu,
+    oracle.ACT_SILU: torch.nn.functional.silu,
+    oracle.ACT_NONE: lambda t: t,
+}
+
+
+@pytest.mark.parametrize("act", sorted(ACTS))
+@pytest.mark.parametrize("w_layout", [0, 1])
+def test_linear_act_against_torch_library(act, w_layout):
+    M, N, K = 9, 7, 11
+    x = RNG.standard_normal((M, K)); w = RNG.standard_normal((K, N)) * 0.5
+    b = RNG.standard_normal(N); r = RNG.standard_normal((M, N))
+    ws = w if w_layout == 0 else np.ascontiguousarray(w.T)
+    want = ACTS[act](torch.from_numpy(x @ w + b)).numpy() + r
+    np.testing.assert_allclose(oracle.linear_act(x, ws, b, r, act, w_layout), want, rtol=0, atol=1e-13)
+    # optional operands really are optional
+    np.testing.assert_allclose(oracle.linear_act(x, ws, None, None, act, w_layout),
+                               ACTS[act](torch.from_numpy(x @ w)).numpy(), rtol=0, atol=1e-13)
+
+
+def test_linear_act_closed_forms():
+    one = np.ones((1, 1))
+    f = lambda z, act: oracle.linear_act(np.array([[z]]), one, None, None, act)[0, 0]
+    assert f(-2.0, oracle.ACT_RELU) == 0.0 and f(2.5, oracle.ACT_RELU) == 2.5
+    assert f(0.0, oracle.ACT_SILU) == 0.0
+    for z in (0.3, 1.0, 4.0):   # z sigma(z) + z sigma(-z) = z
+        assert abs(f(z, oracle.ACT_SILU) - f(-z, oracle.ACT_SILU) - z) < 1e-15 * max(1, z)
+        assert abs(f(z, oracle.ACT_GELU_ERF) - f(-z, oracle.ACT_GELU_ERF) - z) < 1e-15 * max(1, z)
+    assert abs(f(1.0, oracle.ACT_SILU) - 1.0 / (1.0 + math.exp(-1.0))) < 1e-16
+    assert abs(f(1.0, oracle.ACT_GELU_ERF) - 0.8413447460685429) < 1e-15     # Phi(1)
+    assert abs(f(1.0, oracle.ACT_GELU_ERF) - f(1.0, oracle.ACT_GELU_TANH)) > 1e-4
+
+
+def test_linear_act_matches_the_gelu_entry_and_mm_add():
+    M, N, K = 6, 5, 4
+    x = RNG.standard_normal((M, K)); w = RNG.standard_normal((K, N)); b = RNG.standard_normal(N)
+    r = RNG.standard_normal((M, N))
+    np.testing.assert_array_equal(oracle.linear_act(x, w, b), oracle.linear_bias_gelu(x, w, b))
+    np.testing.assert_allclose(oracle.linear_act(x, w, None, r, oracle.ACT_NONE), x @ w + r, rtol=0, atol=1e-14)
+    with pytest.raises(ValueError):
+        oracle.linear_act(x, w, b, None, 9)

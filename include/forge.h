@@ -141,6 +141,20 @@ int forge_linear_bias_gelu(const void* x, const void* w, const void* b, void* y,
                            int M, int N, int K, void* stream);
 
 /*
+ * The other patterns of the operator-fusion pass (Section 4.3 "Pass 5": linear+relu, linear+gelu,
+ * linear+silu, and mm+add, a residual addition after a raw matrix multiply), on the same kernel:
+ *     y[m,n] = act(b[n] + sum_k x[m,k] * W(k,n)) + residual[m,n]
+ * act: FORGE_ACT_GELU_TANH, FORGE_ACT_GELU_ERF (0.5 z (1 + erf(z / sqrt 2))), FORGE_ACT_RELU,
+ * FORGE_ACT_SILU (z / (1 + exp(-z))) or FORGE_ACT_NONE.  w_layout: FORGE_W_KN = w stored [K,N] (as in
+ * forge_linear_bias_gelu), FORGE_W_NK = w stored [N,K], the [out,in] layout of the listing's Linear.
+ * b ([N]) and residual ([M,N], bf16) may be NULL.  Same shape limits as forge_linear_bias_gelu.
+ */
+enum { FORGE_ACT_GELU_TANH = 0, FORGE_ACT_GELU_ERF = 1, FORGE_ACT_RELU = 2, FORGE_ACT_SILU = 3, FORGE_ACT_NONE = 4 };
+enum { FORGE_W_KN = 0, FORGE_W_NK = 1 };
+int forge_linear_act(const void* x, const void* w, const void* b, const void* residual, void* y,
+                     int M, int N, int K, int act, int w_layout, void* stream);
+
+/*
  * Host-buffer variants: the same operators for callers whose tensors live in
  * HOST memory (pinned memory makes the copies asynchronous).  Inputs are copied
  * to `dev_scratch`, the operator runs there, and the result is copied back to the

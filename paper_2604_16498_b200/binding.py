@@ -29,6 +29,7 @@ SIGNATURES = {
     "forge_attn_decode_workspace_bytes": (_sz, [_i, _i, _i, _i]),
     "forge_attn_decode_splitkv_static": (_i, _DEC + [_vp]),
     "forge_linear_bias_gelu": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
+    "forge_linear_act": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]),
     "forge_attn_host_scratch_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _i]),
     "forge_attn_fused_host": (_i, _ATTN + [_vp, _sz, _vp]),
     "forge_attn_fused_f32_host": (_i, _ATTN + [_vp, _sz, _vp]),
@@ -176,6 +177,29 @@ def linear_bias_gelu(x, w, b, out=None):
     _check("forge_linear_bias_gelu", load().forge_linear_bias_gelu(
         _dev(x, torch.bfloat16, "x"), _dev(w, torch.bfloat16, "w"), _dev(b, torch.bfloat16, "b"),
         _dev(out, torch.bfloat16, "out"), M, N, K, _stream()))
+    return out
+
+
+ACT_GELU_TANH, ACT_GELU_ERF, ACT_RELU, ACT_SILU, ACT_NONE = range(5)
+W_KN, W_NK = 0, 1
+
+
+def linear_act(x, w, b=None, residual=None, act=ACT_GELU_TANH, w_layout=W_KN, out=None):
+    """forge_linear_act: act(x @ W + b) + residual with W given as [K,N] (W_KN) or [N,K] (W_NK)."""
+    M, K = x.shape
+    N = w.shape[1] if w_layout == W_KN else w.shape[0]
+    if tuple(w.shape) != ((K, N) if w_layout == W_KN else (N, K)):
+        raise ValueError("w must be [K,N] for W_KN and [N,K] for W_NK")
+    if b is not None and tuple(b.shape) != (N,):
+        raise ValueError("b [N] expected")
+    if residual is not None and tuple(residual.shape) != (M, N):
+        raise ValueError("residual [M,N] expected")
+    out = torch.empty((M, N), dtype=torch.bfloat16, device=x.device) if out is None else out
+    bf = torch.bfloat16
+    _check("forge_linear_act", load().forge_linear_act(
+        _dev(x, bf, "x"), _dev(w, bf, "w"), None if b is None else _dev(b, bf, "b"),
+        None if residual is None else _dev(residual, bf, "residual"), _dev(out, bf, "out"),
+        M, N, K, int(act), int(w_layout), _stream()))
     return out
 
 

@@ -50,16 +50,28 @@ __device__ __forceinline__ float gelu_tanh_f32(float z) {
     return fmaf(hz, t, hz);
 }
 
+// Epilogue activations of the operator-fusion patterns (linear+gelu, linear+relu, linear+silu, mm+add).
+template <int ACT>
+__device__ __forceinline__ float activate(float z) {
+    if constexpr (ACT == FORGE_ACT_GELU_TANH) return gelu_tanh_f32(z);
+    if constexpr (ACT == FORGE_ACT_GELU_ERF) return 0.5f * z * (1.0f + erff(z * 0.70710678118654752f));
+    if constexpr (ACT == FORGE_ACT_RELU) return fmaxf(z, 0.f);
+    if constexpr (ACT == FORGE_ACT_SILU) return z / (1.0f + __expf(-z));
+    return z;
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int BN, int STAGES>
+// ACT: activation; W_NK: W is stored [N, K] (K-major B operand) instead of [K, N] (MN-major B operand).
+// bias and residual may be null.
+template <int BN, int STAGES, int ACT, bool W_NK>
 __global__ void __launch_bounds__(kThreads, 1)
 linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                         const __grid_constant__ CUtensorMap tmap_y, const __nv_bfloat16* __restrict__ bias,
-                        int M, int N, int K, int* __restrict__ status) {
+                        const __nv_bfloat16* __restrict__ residual, int M, int N, int K, int* __restrict__ status) {
     using L = LinearSmem<BN, STAGES>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -105,16 +117,20 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
                     uint8_t* sb = sa + L::kABytes;
                     mbar_expect_tx(&full[stage], L::kStageBytes);
                     tma_load_2d(sa, &tmap_x, &full[stage], kb * kBK, m0);
+                    if constexpr (W_NK) {  // BN rows of W, 64 K-elements (one swizzle span) each
+                        tma_load_2d(sb, &tmap_w, &full[stage], kb * kBK, n0);
+                    } else {
 #pragma unroll
-                    for (int c = 0; c < BN / 64; ++c)
-                        tma_load_2d(sb + c * (kBK * 128), &tmap_w, &full[stage], n0 + c * 64, kb * kBK);
+                        for (int c = 0; c < BN / 64; ++c)
+                            tma_load_2d(sb + c * (kBK * 128), &tmap_w, &full[stage], n0 + c * 64, kb * kBK);
+                    }
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
             }
         }
     } else if (warp == 1) {
         if (elect_one()) {
-            constexpr uint32_t idesc = make_idesc_bf16(kBM, BN, /*a_mn_major=*/false, /*b_mn_major=*/true);
+            constexpr uint32_t idesc = make_idesc_bf16(kBM, BN, /*a_mn_major=*/false, /*b_mn_major=*/!W_NK);
             int stage = 0;
             uint32_t phase = 0;
             int it = 0;
@@ -134,7 +150,9 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
                         // A: 16 K-elements = 32 bytes further along the 128-byte swizzled row
                         const uint64_t a_desc = make_smem_desc(sa + k * 32, 16, 1024);
                         // B: 16 K-rows = two 1024-byte groups further; 64-column chunks are kBK*128 bytes apart
-                        const uint64_t b_desc = make_smem_desc(sb + k * 2048, kBK * 128, 1024);
+                        // [N,K] weights: K-major like A (32 bytes per k-step inside the swizzled row)
+                        const uint64_t b_desc = W_NK ? make_smem_desc(sb + k * 32, 16, 1024)
+                                                     : make_smem_desc(sb + k * 2048, kBK * 128, 1024);
                         mma_ss(d_tmem, a_desc, b_desc, idesc, (kb | k) != 0);
                     }
                     mma_commit(&empty[stage]);  // the stage is free once these MMAs have read it
@@ -156,7 +174,7 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
             const uint32_t acc_phase = (it >> 1) & 1;
             float* bias_s = s_bias + acc * BN;
             for (int i = etid; i < BN; i += kEpiThreads)
-                bias_s[i] = (n0 + i < N) ? __bfloat162float(bias[n0 + i]) : 0.f;
+                bias_s[i] = (bias != nullptr && n0 + i < N) ? __bfloat162float(bias[n0 + i]) : 0.f;
             asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
             // A warp that gave up keeps taking part in the named barrier above (so the others never
             // wait for it there) but skips the work.
@@ -179,12 +197,19 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {  // 16-byte chunk chalf*4 + c of the row's 128-byte line
                     uint32_t w[4];
+                    // residual[m, n .. n+7] (mm+add pattern): 16 bytes of this thread's output row
+                    uint4 res = make_uint4(0, 0, 0, 0);
+                    const int gcol = n0 + blk * 64 + chalf * 32 + c * 8;
+                    if (residual != nullptr && m0 + row < M && gcol < N)
+                        res = *reinterpret_cast<const uint4*>(residual + (size_t)(m0 + row) * N + gcol);
+                    const uint32_t rw[4] = {res.x, res.y, res.z, res.w};
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const int col = c * 8 + 2 * i;
                         const float z0 = __uint_as_float(r[col]) + bias_s[blk * 64 + chalf * 32 + col];
                         const float z1 = __uint_as_float(r[col + 1]) + bias_s[blk * 64 + chalf * 32 + col + 1];
-                        w[i] = pack_bf16(gelu_tanh_f32(z0), gelu_tanh_f32(z1));
+                        w[i] = pack_bf16(activate<ACT>(z0) + __uint_as_float(rw[i] << 16),
+                                         activate<ACT>(z1) + __uint_as_float(rw[i] & 0xffff0000u));
                     }
                     *reinterpret_cast<uint4*>(stage_out + row * 128 + (((chalf * 4 + c) ^ (row & 7)) << 4)) =
                         make_uint4(w[0], w[1], w[2], w[3]);
@@ -217,23 +242,28 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
     }
 }
 
-template <int BN, int STAGES>
-int launch_linear(const void* x, const void* w, const void* b, void* y, int M, int N, int K, cudaStream_t s) {
+template <int BN, int STAGES, int ACT, bool W_NK>
+int launch_linear(const void* x, const void* w, const void* b, const void* residual, void* y, int M, int N, int K,
+                  cudaStream_t s) {
     using L = LinearSmem<BN, STAGES>;
-    CUtensorMap tmap_x, tmap_w;
+    CUtensorMap tmap_x, tmap_w, tmap_y;
     {
         const uint64_t dims[2] = {(uint64_t)K, (uint64_t)M};
         const uint64_t strides[1] = {(uint64_t)K * 2};
         const uint32_t box[2] = {kBK, kBM};
         if (!encode_tmap_bf16_sw128(&tmap_x, x, 2, dims, strides, box)) return FORGE_ERR_CUDA;
     }
-    {
+    if (W_NK) {  // w[N, K]: rows of 64 K-elements
+        const uint64_t dims[2] = {(uint64_t)K, (uint64_t)N};
+        const uint64_t strides[1] = {(uint64_t)K * 2};
+        const uint32_t box[2] = {kBK, BN};
+        if (!encode_tmap_bf16_sw128(&tmap_w, w, 2, dims, strides, box)) return FORGE_ERR_CUDA;
+    } else {     // w[K, N]: 64 K-rows of 64 N-elements per box
         const uint64_t dims[2] = {(uint64_t)N, (uint64_t)K};
         const uint64_t strides[1] = {(uint64_t)N * 2};
         const uint32_t box[2] = {64, kBK};
         if (!encode_tmap_bf16_sw128(&tmap_w, w, 2, dims, strides, box)) return FORGE_ERR_CUDA;
     }
-    CUtensorMap tmap_y;
     {
         const uint64_t dims[2] = {(uint64_t)N, (uint64_t)M};
         const uint64_t strides[1] = {(uint64_t)N * 2};
@@ -244,24 +274,47 @@ int launch_linear(const void* x, const void* w, const void* b, void* y, int M, i
     if (!status) return FORGE_ERR_CUDA;
     const int sms = sm_count();
     if (sms <= 0) return FORGE_ERR_CUDA;
-    auto kernel = linear_bias_gelu_kernel<BN, STAGES>;
+    auto kernel = linear_bias_gelu_kernel<BN, STAGES, ACT, W_NK>;
     FORGE_SET_SMEM_ONCE(kernel, L::kAlloc);
     const int tiles = ((M + kBM - 1) / kBM) * ((N + BN - 1) / BN);
     const int grid = tiles < sms ? tiles : sms;
-    kernel<<<grid, kThreads, L::kAlloc, s>>>(tmap_x, tmap_w, tmap_y, static_cast<const __nv_bfloat16*>(b), M, N, K,
-                                             status);
+    kernel<<<grid, kThreads, L::kAlloc, s>>>(tmap_x, tmap_w, tmap_y, static_cast<const __nv_bfloat16*>(b),
+                                             static_cast<const __nv_bfloat16*>(residual), M, N, K, status);
     return finish_launch(1);
+}
+
+template <int ACT>
+int launch_layout(int w_layout, const void* x, const void* w, const void* b, const void* r, void* y, int M, int N,
+                  int K, cudaStream_t s) {
+    return w_layout == FORGE_W_NK ? launch_linear<192, 4, ACT, true>(x, w, b, r, y, M, N, K, s)
+                                  : launch_linear<192, 4, ACT, false>(x, w, b, r, y, M, N, K, s);
 }
 
 }  // namespace
 }  // namespace forge
 
+extern "C" int forge_linear_act(const void* x, const void* w, const void* b, const void* residual, void* y,
+                                int M, int N, int K, int act, int w_layout, void* stream) {
+    using namespace forge;
+    if (!x || !w || !y) return FORGE_ERR_INVALID_ARG;
+    if (M <= 0 || N <= 0 || K <= 0) return FORGE_ERR_INVALID_ARG;
+    if (act < FORGE_ACT_GELU_TANH || act > FORGE_ACT_NONE) return FORGE_ERR_INVALID_ARG;
+    if (w_layout != FORGE_W_KN && w_layout != FORGE_W_NK) return FORGE_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(w) || !aligned16(y) || (b && !aligned16(b)) || (residual && !aligned16(residual)))
+        return FORGE_ERR_INVALID_ARG;
+    if ((K % 8) != 0 || (N % 8) != 0) return FORGE_ERR_UNSUPPORTED;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    switch (act) {
+        case FORGE_ACT_GELU_TANH: return launch_layout<FORGE_ACT_GELU_TANH>(w_layout, x, w, b, residual, y, M, N, K, s);
+        case FORGE_ACT_GELU_ERF: return launch_layout<FORGE_ACT_GELU_ERF>(w_layout, x, w, b, residual, y, M, N, K, s);
+        case FORGE_ACT_RELU: return launch_layout<FORGE_ACT_RELU>(w_layout, x, w, b, residual, y, M, N, K, s);
+        case FORGE_ACT_SILU: return launch_layout<FORGE_ACT_SILU>(w_layout, x, w, b, residual, y, M, N, K, s);
+        default: return launch_layout<FORGE_ACT_NONE>(w_layout, x, w, b, residual, y, M, N, K, s);
+    }
+}
+
 extern "C" int forge_linear_bias_gelu(const void* x, const void* w, const void* b, void* y,
                                       int M, int N, int K, void* stream) {
-    using namespace forge;
-    if (!x || !w || !b || !y) return FORGE_ERR_INVALID_ARG;
-    if (M <= 0 || N <= 0 || K <= 0) return FORGE_ERR_INVALID_ARG;
-    if (!aligned16(x) || !aligned16(w) || !aligned16(b) || !aligned16(y)) return FORGE_ERR_INVALID_ARG;
-    if ((K % 8) != 0 || (N % 8) != 0) return FORGE_ERR_UNSUPPORTED;
-    return launch_linear<192, 4>(x, w, b, y, M, N, K, static_cast<cudaStream_t>(stream));
+    if (!b) return FORGE_ERR_INVALID_ARG;
+    return forge_linear_act(x, w, b, nullptr, y, M, N, K, FORGE_ACT_GELU_TANH, FORGE_W_KN, stream);
 }

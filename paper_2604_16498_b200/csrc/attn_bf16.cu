@@ -1,7 +1,7 @@
 // Fused attention, bf16 in / fp32 accumulate / bf16 out (Eq. 8 / Eq. 9): scores, mask, online
 // softmax and the product with V in one kernel; S and P never reach global memory.
 //
-// One CTA = one (batch, query head, pair of 128-row query tiles).  The two tiles run in ping-pong so
+// One work item = two 128-row query tiles that share K and V (see the item decoding below).  The two tiles run in ping-pong so
 // that the tensor core works on one tile while the softmax of the other is computed.  Warp roles:
 //   warps 0-3 : softmax / rescale / epilogue of tile 0; thread = one query row (TMEM lane), so row
 //   warps 4-7 : the same for tile 1                    maxima and sums need no cross-thread reduction
@@ -106,7 +106,9 @@ struct AttnParams {
 
 // What one CTA needs to know about a work item (a pair of query tiles of one head).
 struct ItemInfo {
-    int q_pair, h, b, kvh, kvlen;
+    int b, kvh, kvlen;
+    int q0[kTilesPerCta];       // first query row of each of the two tiles
+    int h[kTilesPerCta];        // query head of each tile
     int n_tiles[kTilesPerCta];  // KV tiles visible to at least one row of each query tile (0: tile beyond Sq)
     int n_max;
 };
@@ -138,9 +140,15 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(wg_bar + 2);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int num_q_pairs = (p.Sq + kTilesPerCta * kBM - 1) / (kTilesPerCta * kBM);
-    const int heads = p.Hq * p.B;
-    const int num_items = num_q_pairs * heads;
+    // The two tiles of an item: with an even number of query heads per KV head, the same 128 query rows of
+    // two heads that share K and V (equal causal lengths, so neither tile waits for the other); otherwise
+    // two consecutive 128-row tiles of one head.
+    const int G = p.Hq / p.Hkv;
+    const bool pair_heads = (G % 2) == 0;
+    const int num_q_tiles = (p.Sq + kBM - 1) / kBM;
+    const int rows_of_items = pair_heads ? num_q_tiles : (num_q_tiles + 1) / 2;  // steps along the query axis
+    const int heads = pair_heads ? (p.Hq / 2) * p.B : p.Hq * p.B;               // items per such step
+    const int num_items = rows_of_items * heads;
     const int causal_off = p.Skv - p.Sq;
     const bool causal = (p.mask_kind & FORGE_MASK_CAUSAL) != 0;
 
@@ -153,17 +161,25 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     };
     auto decode = [&](int i) {
         ItemInfo it;
-        it.q_pair = num_q_pairs - 1 - i / heads;
+        const int qstep = rows_of_items - 1 - i / heads;  // longest (causal) first
         const int hb = i % heads;
-        it.h = hb % p.Hq;
-        it.b = hb / p.Hq;
-        it.kvh = it.h / (p.Hq / p.Hkv);
+        if (pair_heads) {
+            const int hp = hb % (p.Hq / 2);
+            it.b = hb / (p.Hq / 2);
+            it.h[0] = 2 * hp; it.h[1] = 2 * hp + 1;
+            it.q0[0] = it.q0[1] = qstep * kBM;
+        } else {
+            it.b = hb / p.Hq;
+            it.h[0] = it.h[1] = hb % p.Hq;
+            it.q0[0] = 2 * qstep * kBM; it.q0[1] = (2 * qstep + 1) * kBM;
+        }
+        it.kvh = it.h[0] / G;
         it.kvlen = p.Skv;
         if (p.mask_kind & FORGE_MASK_PADDING) it.kvlen = min(max(p.lens[it.b], 0), p.Skv);
         it.n_max = 0;
 #pragma unroll
         for (int t = 0; t < kTilesPerCta; ++t) {
-            const int q0 = (it.q_pair * kTilesPerCta + t) * kBM;
+            const int q0 = it.q0[t];
             int kv_end = it.kvlen;
             if (causal) kv_end = min(kv_end, min(q0 + kBM, p.Sq) + causal_off);
             if (q0 >= p.Sq) kv_end = 0;
@@ -219,7 +235,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
 #pragma unroll
                     for (int c = 0; c < D / 64; ++c)  // rows beyond Sq are zero-filled by the TMA unit
                         tma_load_3d(sQ + t * L::kTileBytes + c * L::kChunkBytes, &tmap_q, q_full, c * 64,
-                                    (it.q_pair * kTilesPerCta + t) * kBM, it.b * p.Hq + it.h);
+                                    it.q0[t], it.b * p.Hq + it.h[t]);
                 for (int j = 0; j < it.n_max; ++j, ++kvn) {
                     const int st = kvn % kKVStages;
                     const uint32_t ph = (kvn / kKVStages) & 1;
@@ -350,10 +366,10 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             const int i = item_of_round(r);
             if (i >= num_items) break;
             const ItemInfo it = decode(i);
-            const int q0 = (it.q_pair * kTilesPerCta + t) * kBM;
+            const int q0 = it.q0[t];
             const int qi = q0 + row;
             const int nt = it.n_tiles[t];
-            __nv_bfloat16* orow = p.out + ((size_t)(it.b * p.Hq + it.h) * p.Sq + qi) * D;
+            __nv_bfloat16* orow = p.out + ((size_t)(it.b * p.Hq + it.h[t]) * p.Sq + qi) * D;
             if (nt == 0) {  // no visible key for any row of this tile (or the tile lies beyond Sq)
                 if (qi < p.Sq) {
 #pragma unroll
@@ -526,7 +542,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     fence_proxy_async_smem();
                     if (!wg_sync()) { failed = true; break; }
                     if (wg_tid == 0) {
-                        tma_store_3d(&tmap_o, stage_out, cb * 64, q0, it.b * p.Hq + it.h);
+                        tma_store_3d(&tmap_o, stage_out, cb * 64, q0, it.b * p.Hq + it.h[t]);
                         tma_store_commit();
                     }
                 }
@@ -582,7 +598,9 @@ int launch_attn(const void* q, const void* k, const void* v, void* out, int B, i
     FORGE_SET_SMEM_ONCE(kernel, L::kAlloc);
     const int sms = sm_count();
     if (sms <= 0) return FORGE_ERR_CUDA;
-    const long long items = (long long)Hq * B * ((Sq + kTilesPerCta * kBM - 1) / (kTilesPerCta * kBM));
+    const int q_tiles = (Sq + kBM - 1) / kBM;
+    const long long items = ((Hq / Hkv) % 2 == 0) ? (long long)(Hq / 2) * B * q_tiles
+                                                  : (long long)Hq * B * ((q_tiles + 1) / 2);
     const int grid = items < sms ? (int)items : sms;
     kernel<<<grid, kThreads, L::kAlloc, s>>>(tq, tk, tv, to, p);
     return finish_launch(1);

@@ -106,7 +106,8 @@ struct AttnParams {
 
 // What one CTA needs to know about a work item (a pair of query tiles of one head).
 struct ItemInfo {
-    int b, kvh, kvlen;
+    int b, kvlen;
+    int kvh[kTilesPerCta];      // KV head of each tile (equal unless the tiles read separate K/V streams)
     int q0[kTilesPerCta];       // first query row of each of the two tiles
     int h[kTilesPerCta];        // query head of each tile
     int n_tiles[kTilesPerCta];  // KV tiles visible to at least one row of each query tile (0: tile beyond Sq)
@@ -145,10 +146,18 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     // two consecutive 128-row tiles of one head.
     const int G = p.Hq / p.Hkv;
     const bool pair_heads = (G % 2) == 0;
+    // With an odd group size and D = 64 (where shared memory has room for it) the two tiles are still two
+    // heads on the same query rows, each with its own K/V stream through half of the stage ring.
+    const bool two_streams = !pair_heads && kKVStages >= 4;
+    const int ring_len = two_streams ? kKVStages / 2 : kKVStages;
     const int num_q_tiles = (p.Sq + kBM - 1) / kBM;
-    const int rows_of_items = pair_heads ? num_q_tiles : (num_q_tiles + 1) / 2;  // steps along the query axis
-    const int heads = pair_heads ? (p.Hq / 2) * p.B : p.Hq * p.B;               // items per such step
+    const int head_pairs = (p.Hq + 1) / 2;
+    const int rows_of_items = (pair_heads || two_streams) ? num_q_tiles : (num_q_tiles + 1) / 2;
+    const int heads = (pair_heads || two_streams) ? head_pairs * p.B : p.Hq * p.B;  // items per query step
     const int num_items = rows_of_items * heads;
+    // ring slot and phase of the g-th KV tile of stream u
+    auto kv_slot = [&](int u, int g) { return (two_streams ? u * ring_len : 0) + g % ring_len; };
+    auto kv_phase = [&](int g) { return (uint32_t)((g / ring_len) & 1); };
     const int causal_off = p.Skv - p.Sq;
     const bool causal = (p.mask_kind & FORGE_MASK_CAUSAL) != 0;
 
@@ -163,17 +172,20 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
         ItemInfo it;
         const int qstep = rows_of_items - 1 - i / heads;  // longest (causal) first
         const int hb = i % heads;
-        if (pair_heads) {
-            const int hp = hb % (p.Hq / 2);
-            it.b = hb / (p.Hq / 2);
-            it.h[0] = 2 * hp; it.h[1] = 2 * hp + 1;
+        if (pair_heads || two_streams) {
+            const int hp = hb % head_pairs;
+            it.b = hb / head_pairs;
+            it.h[0] = 2 * hp;
+            it.h[1] = min(2 * hp + 1, p.Hq - 1);
             it.q0[0] = it.q0[1] = qstep * kBM;
+            if (2 * hp + 1 >= p.Hq) it.q0[1] = num_q_tiles * kBM;  // odd head count: no second tile
         } else {
             it.b = hb / p.Hq;
             it.h[0] = it.h[1] = hb % p.Hq;
             it.q0[0] = 2 * qstep * kBM; it.q0[1] = (2 * qstep + 1) * kBM;
         }
-        it.kvh = it.h[0] / G;
+        it.kvh[0] = it.h[0] / G;
+        it.kvh[1] = it.h[1] / G;
         it.kvlen = p.Skv;
         if (p.mask_kind & FORGE_MASK_PADDING) it.kvlen = min(max(p.lens[it.b], 0), p.Skv);
         it.n_max = 0;
@@ -220,8 +232,8 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
       if (warp == 8) {
         // ------------------------------------------------------------------ TMA producer
         if (elect_one()) {
-            int kvn = 0;     // KV tiles loaded so far (ring position), across items
-            int items = 0;   // items with work so far
+            int kvn[2] = {0, 0};  // KV tiles loaded so far per stream (ring position), across items
+            int items = 0;        // items with work so far
             for (int r = 0; !failed; ++r) {
                 const int i = item_of_round(r);
                 if (i >= num_items) break;
@@ -236,21 +248,25 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     for (int c = 0; c < D / 64; ++c)  // rows beyond Sq are zero-filled by the TMA unit
                         tma_load_3d(sQ + t * L::kTileBytes + c * L::kChunkBytes, &tmap_q, q_full, c * 64,
                                     it.q0[t], it.b * p.Hq + it.h[t]);
-                for (int j = 0; j < it.n_max; ++j, ++kvn) {
-                    const int st = kvn % kKVStages;
-                    const uint32_t ph = (kvn / kKVStages) & 1;
-                    if (!mbar_wait(&k_empty[st], ph ^ 1)) { failed = true; break; }
-                    mbar_expect_tx(&k_full[st], L::kTileBytes);
+                for (int j = 0; j < it.n_max && !failed; ++j) {
+                    for (int u = 0; u < (two_streams ? 2 : 1); ++u) {
+                        if (two_streams && j >= it.n_tiles[u]) continue;
+                        const int g = kvn[u]++, st = kv_slot(u, g);
+                        const uint32_t ph = kv_phase(g);
+                        const int kv_row = it.b * p.Hkv + it.kvh[u];
+                        if (!mbar_wait(&k_empty[st], ph ^ 1)) { failed = true; break; }
+                        mbar_expect_tx(&k_full[st], L::kTileBytes);
 #pragma unroll
-                    for (int c = 0; c < D / 64; ++c)
-                        tma_load_3d(sK + st * L::kTileBytes + c * L::kChunkBytes, &tmap_k, &k_full[st], c * 64,
-                                    j * kBN, it.b * p.Hkv + it.kvh);
-                    if (!mbar_wait(&v_empty[st], ph ^ 1)) { failed = true; break; }
-                    mbar_expect_tx(&v_full[st], L::kTileBytes);
+                        for (int c = 0; c < D / 64; ++c)
+                            tma_load_3d(sK + st * L::kTileBytes + c * L::kChunkBytes, &tmap_k, &k_full[st], c * 64,
+                                        j * kBN, kv_row);
+                        if (!mbar_wait(&v_empty[st], ph ^ 1)) { failed = true; break; }
+                        mbar_expect_tx(&v_full[st], L::kTileBytes);
 #pragma unroll
-                    for (int c = 0; c < D / 64; ++c)
-                        tma_load_3d(sV + st * L::kTileBytes + c * L::kChunkBytes, &tmap_v, &v_full[st], c * 64,
-                                    j * kBN, it.b * p.Hkv + it.kvh);
+                        for (int c = 0; c < D / 64; ++c)
+                            tma_load_3d(sV + st * L::kTileBytes + c * L::kChunkBytes, &tmap_v, &v_full[st], c * 64,
+                                        j * kBN, kv_row);
+                    }
                 }
                 ++items;
             }
@@ -261,8 +277,8 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             constexpr uint32_t idesc_s = make_idesc_bf16(kBM, kBN, false, false);
             constexpr uint32_t idesc_o = make_idesc_bf16(kBM, D, false, true);
             const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
-            int kvbase = 0;                 // ring position of the item's first KV tile
-            int k_waited = -1, v_waited = -1;  // highest ring position whose arrival has been observed
+            int kvbase[2] = {0, 0};          // per stream: ring position of the item's first KV tile
+            int k_waited[2] = {-1, -1}, v_waited[2] = {-1, -1};  // highest ring position seen to have arrived
             int items = 0;                  // items with work so far
             int its[kTilesPerCta] = {0, 0};     // tile iterations issued so far per query tile (barrier phases)
             int used[kTilesPerCta] = {0, 0};    // items in which each query tile had work (phase of o_free)
@@ -277,10 +293,10 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 const int qk_total = it.n_tiles[0] + it.n_tiles[1];
                 // S_t(j) = Q_t K_j^T; the last tile that uses K_j releases its stage
                 auto issue_qk = [&](int t, int j) -> bool {
-                    const int g = kvbase + j, st = g % kKVStages;
-                    if (g > k_waited) {
-                        if (!mbar_wait(&k_full[st], (g / kKVStages) & 1)) return false;
-                        k_waited = g;
+                    const int u = two_streams ? t : 0, g = kvbase[u] + j, st = kv_slot(u, g);
+                    if (g > k_waited[u]) {
+                        if (!mbar_wait(&k_full[st], kv_phase(g))) return false;
+                        k_waited[u] = g;
                     }
                     tc_fence_after_sync();
                     const uint32_t kb = k_addr + st * L::kTileBytes, qb = q_addr + t * L::kTileBytes;
@@ -290,8 +306,8 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                         mma_ss(tmem_base + kColS + t * kBN, make_smem_desc(qb + off, 16, 1024),
                                make_smem_desc(kb + off, 16, 1024), idesc_s, kk != 0);
                     }
-                    bool last = true;
-                    for (int u = t + 1; u < kTilesPerCta; ++u) last = last && !(j < it.n_tiles[u]);
+                    bool last = true;  // no later tile reads this K tile (always so with separate streams)
+                    for (int t2 = t + 1; t2 < kTilesPerCta && !two_streams; ++t2) last = last && !(j < it.n_tiles[t2]);
                     if (last) mma_commit(&k_empty[st]);
                     mma_commit(&s_full[t]);
                     // the item's last S = Q K^T: once it completes, the next item's Q tiles may be loaded
@@ -300,11 +316,11 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 };
                 // O_t += P_t(j) V_j with P_t read from tensor memory
                 auto issue_pv = [&](int t, int j) -> bool {
-                    const int g = kvbase + j, st = g % kKVStages;
+                    const int u = two_streams ? t : 0, g = kvbase[u] + j, st = kv_slot(u, g);
                     if (!mbar_wait(&p_ready[t], its[t] & 1)) return false;
-                    if (g > v_waited) {
-                        if (!mbar_wait(&v_full[st], (g / kKVStages) & 1)) return false;
-                        v_waited = g;
+                    if (g > v_waited[u]) {
+                        if (!mbar_wait(&v_full[st], kv_phase(g))) return false;
+                        v_waited[u] = g;
                     }
                     // the first product of an item overwrites O_t: the previous item's epilogue must have read it
                     if (j == 0 && !mbar_wait(&o_free[t], (used[t] & 1) ^ 1)) return false;
@@ -318,7 +334,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                                make_smem_desc(vb + kk * 2048, L::kChunkBytes, 1024), idesc_o, (j | kk) != 0);
                     }
                     bool last = true;
-                    for (int u = t + 1; u < kTilesPerCta; ++u) last = last && !(j < it.n_tiles[u]);
+                    for (int t2 = t + 1; t2 < kTilesPerCta && !two_streams; ++t2) last = last && !(j < it.n_tiles[t2]);
                     if (last) mma_commit(&v_empty[st]);
                     mma_commit(&pv_done[t]);
                     ++its[t];
@@ -336,7 +352,8 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     }
                 }
                 for (int t = 0; t < kTilesPerCta; ++t) used[t] += it.n_tiles[t] > 0;
-                kvbase += it.n_max;
+                if (two_streams) { kvbase[0] += it.n_tiles[0]; kvbase[1] += it.n_tiles[1]; }
+                else kvbase[0] += it.n_max;
                 ++items;
             }
         }
@@ -599,8 +616,9 @@ int launch_attn(const void* q, const void* k, const void* v, void* out, int B, i
     const int sms = sm_count();
     if (sms <= 0) return FORGE_ERR_CUDA;
     const int q_tiles = (Sq + kBM - 1) / kBM;
-    const long long items = ((Hq / Hkv) % 2 == 0) ? (long long)(Hq / 2) * B * q_tiles
-                                                  : (long long)Hq * B * ((q_tiles + 1) / 2);
+    const bool head_pairs = ((Hq / Hkv) % 2 == 0) || L::kKVStages >= 4;  // same rule as in the kernel
+    const long long items = head_pairs ? (long long)((Hq + 1) / 2) * B * q_tiles
+                                       : (long long)Hq * B * ((q_tiles + 1) / 2);
     const int grid = items < sms ? (int)items : sms;
     kernel<<<grid, kThreads, L::kAlloc, s>>>(tq, tk, tv, to, p);
     return finish_launch(1);

@@ -299,12 +299,14 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                         k_waited[u] = g;
                     }
                     tc_fence_after_sync();
-                    const uint32_t kb = k_addr + st * L::kTileBytes, qb = q_addr + t * L::kTileBytes;
+                    // descriptors differ only in the start-address field: build one per operand, then add
+                    // (byte offset >> 4) for each 16-wide K step (the field cannot overflow below 256 KB)
+                    const uint64_t qd = make_smem_desc(q_addr + t * L::kTileBytes, 16, 1024);
+                    const uint64_t kd = make_smem_desc(k_addr + st * L::kTileBytes, 16, 1024);
 #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk) {
-                        const uint32_t off = (kk / 4) * L::kChunkBytes + (kk % 4) * 32;
-                        mma_ss(tmem_base + kColS + t * kBN, make_smem_desc(qb + off, 16, 1024),
-                               make_smem_desc(kb + off, 16, 1024), idesc_s, kk != 0);
+                        const uint32_t off = ((kk / 4) * L::kChunkBytes + (kk % 4) * 32) >> 4;
+                        mma_ss(tmem_base + kColS + t * kBN, qd + off, kd + off, idesc_s, kk != 0);
                     }
                     bool last = true;  // no later tile reads this K tile (always so with separate streams)
                     for (int t2 = t + 1; t2 < kTilesPerCta && !two_streams; ++t2) last = last && !(j < it.n_tiles[t2]);
@@ -325,14 +327,14 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     // the first product of an item overwrites O_t: the previous item's epilogue must have read it
                     if (j == 0 && !mbar_wait(&o_free[t], (used[t] & 1) ^ 1)) return false;
                     tc_fence_after_sync();
-                    const uint32_t vb = v_addr + st * L::kTileBytes;
+                    // P: 16 keys = 8 columns of packed bf16 pairs.  V: MN-major, 16 keys = two 1024-byte groups
+                    // (2048 bytes per step); the 64-wide chunks of D are 16 KB apart.
+                    const uint64_t vd = make_smem_desc(v_addr + st * L::kTileBytes, L::kChunkBytes, 1024);
+                    const uint32_t o_tmem = tmem_base + kColO + t * D, p_tmem = tmem_base + kColS + t * kBN;
+                    if (j == 0) mma_ts(o_tmem, p_tmem, vd, idesc_o, 0u);
+                    else mma_ts(o_tmem, p_tmem, vd, idesc_o, 1u);
 #pragma unroll
-                    for (int kk = 0; kk < kBN / 16; ++kk) {
-                        // P: 16 keys = 8 columns of packed bf16 pairs.  V: MN-major, 16 keys = two 1024-byte
-                        // groups; the 64-wide chunks of D are 16 KB apart.
-                        mma_ts(tmem_base + kColO + t * D, tmem_base + kColS + t * kBN + kk * 8,
-                               make_smem_desc(vb + kk * 2048, L::kChunkBytes, 1024), idesc_o, (j | kk) != 0);
-                    }
+                    for (int kk = 1; kk < kBN / 16; ++kk) mma_ts(o_tmem, p_tmem + kk * 8, vd + kk * (2048 >> 4), idesc_o, 1u);
                     bool last = true;
                     for (int t2 = t + 1; t2 < kTilesPerCta && !two_streams; ++t2) last = last && !(j < it.n_tiles[t2]);
                     if (last) mma_commit(&v_empty[st]);

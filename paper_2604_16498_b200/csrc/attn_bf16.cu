@@ -1,26 +1,28 @@
 // Fused attention, bf16 in / fp32 accumulate / bf16 out (Eq. 8 / Eq. 9): scores, mask, online
 // softmax and the product with V in one kernel; S and P never reach global memory.
 //
-// One work item = two 128-row query tiles that share K and V (see the item decoding below).  The two tiles run in ping-pong so
-// that the tensor core works on one tile while the softmax of the other is computed.  Warp roles:
+// One work item = two 128-row query tiles (see the item decoding below).  Every 128-key tile of S is
+// computed, normalised and multiplied with V in two 64-key halves with their own barriers, so each
+// query tile has two independent half-step streams and the CTA has four: while a softmax thread works
+// on one half, the tensor core multiplies the other half's P with V and produces that half's next S.
+// Warp roles:
 //   warps 0-3 : softmax / rescale / epilogue of tile 0; thread = one query row (TMEM lane), so row
 //   warps 4-7 : the same for tile 1                    maxima and sums need no cross-thread reduction
-//   warp 8    : TMA producer: both Q tiles once, then K and V tiles (128 keys) through rings
-//   warp 9    : tcgen05.mma issuer (one elected lane), owns the TMEM allocation
-//   warps 10-11 only complete the third warpgroup, which hands most of its registers to the other two
-//   (setmaxnreg: 224 per softmax thread, 56 for the rest; 256*224 + 128*56 = 384*168 as launched).
-// Tensor memory (512 columns): S_0 at 0, S_1 at 128 (128 x 128 fp32 each), O_0 at 256, O_1 at 256 + D.
-// P_t (bf16, two per column) is written over the first 64 columns of S_t and is the A operand of
-// the P V product straight from tensor memory.  MMAs execute in issue order, so the issue sequence
-//   S_0(0) S_1(0) | P_0 ready: O_0 += P_0 V_0, S_0(1) | P_1 ready: O_1 += P_1 V_0, S_1(1) | ...
-// keeps every hazard (P_t read before S_t is overwritten, O_t complete before it is rescaled) safe:
-// the barrier that announces S_t(j+1) also covers the completion of every earlier MMA.
+//   warp 8    : TMA producer: Q tiles, then K and V tiles (128 keys) through rings
+//   warp 9    : tcgen05.mma issuer of tile 0 (one elected lane), owns the TMEM allocation
+//   warp 10   : tcgen05.mma issuer of tile 1
+//   warp 11 only completes the third warpgroup, which hands registers to the other two
+//   (setmaxnreg: 208 per softmax thread, 88 for the rest; 256*208 + 128*88 = 384*168 as launched).
+// Tensor memory (512 columns): S_t at t*128 (half h at +64h, 64 fp32 columns each), O_0 at 256,
+// O_1 at 256 + D.  P (bf16, two per column) of half h is written over the first 32 columns of that
+// half of S and is the A operand of the P V product straight from tensor memory.  A tile's issuer
+// thread issues, per half-step g (key tile g/2, half g%2):  O += P(g) V(g), then S(g+2) = Q K(g+2)^T.
+// MMAs of one thread execute in issue order, so P(g) is read before S(g+2) overwrites it, and the
+// barrier that announces S(g+2) also covers the completion of the P V products up to g.
 // O is rescaled in TMEM only when a row's maximum grows by more than 2^8 (the stale maximum is
 // kept otherwise; the final division by l uses the same reference, so the result is unchanged).
 // Q and K are K-major operands, V [keys, D] is the MN-major B operand of P V.
 #include <cuda_bf16.h>
-
-#include <type_traits>
 
 #include "forge_common.cuh"
 #include "sm100_ptx.cuh"
@@ -33,9 +35,9 @@ using namespace ptx;
 
 constexpr int kBM = 128;          // query rows per tile
 constexpr int kTilesPerCta = 2;
-constexpr int kBN = 128;          // keys per tile
+constexpr int kBN = 128;          // keys per K/V tile in shared memory
+constexpr int kHalf = 64;         // keys per half-step
 constexpr int kThreads = 384;
-constexpr int kSoftmaxThreads = 128;  // per query tile
 constexpr int kTmemCols = 512;
 constexpr int kColS = 0;          // S_t at t * 128
 constexpr int kColO = 256;        // O_t at 256 + t * D
@@ -49,10 +51,10 @@ struct AttnSmem {
     static constexpr int kQOff = 0;
     static constexpr int kKOff = kQOff + kTilesPerCta * kTileBytes;
     static constexpr int kVOff = kKOff + kKVStages * kTileBytes;
-    static constexpr int kOutOff = kVOff + kKVStages * kTileBytes;  // output staging: 128 rows x 64 bf16 per query tile
-    static constexpr int kBarOff = kOutOff + kTilesPerCta * kChunkBytes;
-    // q_full, k/v full+empty per stage, s_full[2], p_ready[2], pv_done[2]
-    static constexpr int kNumBars = 2 + 4 * kKVStages + 10;
+    static constexpr int kOutOff = kVOff + kKVStages * kTileBytes;  // output staging: 32 rows x 64 bf16 per softmax warp
+    static constexpr int kBarOff = kOutOff + 8 * 4096;
+    // q_full[2], q_empty[2], k/v full+empty per stage, s_full[4], p_ready[4], pv_done[4], o_free[2]
+    static constexpr int kNumBars = 4 + 4 * kKVStages + 14;
     static constexpr int kTotal = kBarOff + kNumBars * 8 + 16;
     static constexpr int kAlloc = kTotal + 1024;
 };
@@ -100,19 +102,23 @@ struct AttnParams {
     const int32_t* lens;
     int B, Hq, Hkv, Sq, Skv;
     int mask_kind;
-    float scale_log2;
+    float scale_log2;  // > 0 (a zero scale is passed as the smallest normal number: every product flushes to 0)
     int* status;
 };
 
-// What one CTA needs to know about a work item (a pair of query tiles of one head).
+// What one CTA needs to know about a work item (a pair of query tiles).
 struct ItemInfo {
     int b, kvlen;
     int kvh[kTilesPerCta];      // KV head of each tile (equal unless the tiles read separate K/V streams)
     int q0[kTilesPerCta];       // first query row of each of the two tiles
     int h[kTilesPerCta];        // query head of each tile
-    int n_tiles[kTilesPerCta];  // KV tiles visible to at least one row of each query tile (0: tile beyond Sq)
+    int nh[kTilesPerCta];       // 64-key half-steps visible to at least one row of each query tile (0: no work)
+    int n_tiles[kTilesPerCta];  // the same in 128-key tiles
     int n_max;
 };
+
+// element t of a two-element array without dynamic indexing (keeps the array in registers)
+__device__ __forceinline__ int pick(const int (&a)[kTilesPerCta], int t) { return t ? a[1] : a[0]; }
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -127,18 +133,17 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     uint8_t* sK = smem + L::kKOff;
     uint8_t* sV = smem + L::kVOff;
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBarOff);
-    uint64_t* q_full = bars;
-    uint64_t* q_empty = bars + 1;
-    uint64_t* k_full = bars + 2;
+    uint64_t* q_full = bars;                 // [2] per query tile
+    uint64_t* q_empty = bars + 2;            // [2]
+    uint64_t* k_full = bars + 4;
     uint64_t* k_empty = k_full + kKVStages;
     uint64_t* v_full = k_empty + kKVStages;
     uint64_t* v_empty = v_full + kKVStages;
-    uint64_t* s_full = v_empty + kKVStages;  // [2] per query tile
-    uint64_t* p_ready = s_full + 2;          // [2]
-    uint64_t* pv_done = p_ready + 2;         // [2]
-    uint64_t* o_free = pv_done + 2;          // [2]
-    uint64_t* wg_bar = o_free + 2;           // [2] meeting point of a tile's four softmax warps
-    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(wg_bar + 2);
+    uint64_t* s_full = v_empty + kKVStages;  // [4] query tile t, half h at t * 2 + h
+    uint64_t* p_ready = s_full + 4;          // [4]
+    uint64_t* pv_done = p_ready + 4;         // [4] one completion per P V product of that tile and half
+    uint64_t* o_free = pv_done + 4;          // [2] per query tile
+    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(o_free + 2);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // The two tiles of an item: with an even number of query heads per KV head, the same 128 query rows of
@@ -196,24 +201,23 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             if (causal) kv_end = min(kv_end, min(q0 + kBM, p.Sq) + causal_off);
             if (q0 >= p.Sq) kv_end = 0;
             kv_end = max(kv_end, 0);
-            it.n_tiles[t] = (kv_end + kBN - 1) / kBN;
+            it.nh[t] = (kv_end + kHalf - 1) / kHalf;
+            it.n_tiles[t] = (it.nh[t] + 1) / 2;
             it.n_max = max(it.n_max, it.n_tiles[t]);
         }
         return it;
     };
 
     if (threadIdx.x == 0) {
-        mbar_init(q_full, 1);
-        mbar_init(q_empty, 1);
+        for (int t = 0; t < 2; ++t) { mbar_init(&q_full[t], 1); mbar_init(&q_empty[t], 1); }
+        // a shared K/V stage is released by both tiles' issuer threads, a private one by its own
+        const uint32_t releases = two_streams ? 1 : 2;
         for (int i = 0; i < kKVStages; ++i) {
-            mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], 1);
-            mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], 1);
+            mbar_init(&k_full[i], 1); mbar_init(&k_empty[i], releases);
+            mbar_init(&v_full[i], 1); mbar_init(&v_empty[i], releases);
         }
-        for (int t = 0; t < 2; ++t) {
-            mbar_init(&s_full[t], 1); mbar_init(&p_ready[t], kSoftmaxThreads / 32);
-            mbar_init(&pv_done[t], 1); mbar_init(&o_free[t], kSoftmaxThreads / 32);
-            mbar_init(&wg_bar[t], kSoftmaxThreads / 32);
-        }
+        for (int i = 0; i < 4; ++i) { mbar_init(&s_full[i], 1); mbar_init(&p_ready[i], 4); mbar_init(&pv_done[i], 1); }
+        for (int t = 0; t < 2; ++t) mbar_init(&o_free[t], 4);
         fence_mbar_init();
         prefetch_tmap(&tmap_q); prefetch_tmap(&tmap_k); prefetch_tmap(&tmap_v); prefetch_tmap(&tmap_o);
     }
@@ -228,28 +232,33 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     bool failed = false;
 
     if (warp >= 8) {
-      asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
       if (warp == 8) {
         // ------------------------------------------------------------------ TMA producer
         if (elect_one()) {
-            int kvn[2] = {0, 0};  // KV tiles loaded so far per stream (ring position), across items
-            int items = 0;        // items with work so far
+            int kvn[2] = {0, 0};     // KV tiles loaded so far per stream (ring position), across items
+            int q_loads[2] = {0, 0}; // Q tiles loaded so far per query tile
             for (int r = 0; !failed; ++r) {
                 const int i = item_of_round(r);
                 if (i >= num_items) break;
                 const ItemInfo it = decode(i);
                 if (it.n_max == 0) continue;
-                // the previous item's last S = Q K^T has been issued and completed: Q may be replaced
-                if (!mbar_wait(q_empty, (items & 1) ^ 1)) { failed = true; break; }
-                mbar_expect_tx(q_full, kTilesPerCta * L::kTileBytes);
 #pragma unroll
-                for (int t = 0; t < kTilesPerCta; ++t)
+                for (int t = 0; t < kTilesPerCta; ++t) {
+                    if (it.nh[t] == 0) continue;
+                    // the tile's last S = Q K^T of its previous item has completed: Q may be replaced
+                    if (!mbar_wait(&q_empty[t], (q_loads[t] & 1) ^ 1)) { failed = true; break; }
+                    ++q_loads[t];
+                    mbar_expect_tx(&q_full[t], L::kTileBytes);
 #pragma unroll
                     for (int c = 0; c < D / 64; ++c)  // rows beyond Sq are zero-filled by the TMA unit
-                        tma_load_3d(sQ + t * L::kTileBytes + c * L::kChunkBytes, &tmap_q, q_full, c * 64,
+                        tma_load_3d(sQ + t * L::kTileBytes + c * L::kChunkBytes, &tmap_q, &q_full[t], c * 64,
                                     it.q0[t], it.b * p.Hq + it.h[t]);
+                }
                 for (int j = 0; j < it.n_max && !failed; ++j) {
-                    for (int u = 0; u < (two_streams ? 2 : 1); ++u) {
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        if (u == 1 && !two_streams) continue;
                         if (two_streams && j >= it.n_tiles[u]) continue;
                         const int g = kvn[u]++, st = kv_slot(u, g);
                         const uint32_t ph = kv_phase(g);
@@ -268,129 +277,120 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                                         j * kBN, kv_row);
                     }
                 }
-                ++items;
             }
         }
-      } else if (warp == 9) {
-        // ------------------------------------------------------------------ MMA issuer
+      } else if (warp <= 10) {
+        // ------------------------------------------------------------------ MMA issuer of query tile t
         if (elect_one()) {
-            constexpr uint32_t idesc_s = make_idesc_bf16(kBM, kBN, false, false);
+            const int t = warp - 9;
+            const int u = two_streams ? t : 0;
+            constexpr uint32_t idesc_s = make_idesc_bf16(kBM, kHalf, false, false);
             constexpr uint32_t idesc_o = make_idesc_bf16(kBM, D, false, true);
-            const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
-            int kvbase[2] = {0, 0};          // per stream: ring position of the item's first KV tile
-            int k_waited[2] = {-1, -1}, v_waited[2] = {-1, -1};  // highest ring position seen to have arrived
-            int items = 0;                  // items with work so far
-            int its[kTilesPerCta] = {0, 0};     // tile iterations issued so far per query tile (barrier phases)
-            int used[kTilesPerCta] = {0, 0};    // items in which each query tile had work (phase of o_free)
+            const uint32_t q_addr = smem_u32(sQ) + t * L::kTileBytes, k_addr = smem_u32(sK), v_addr = smem_u32(sV);
+            const uint32_t s_tmem = tmem_base + kColS + t * kBN, o_tmem = tmem_base + kColO + t * D;
+            // descriptors differ only in the start-address field: build one per operand, then add
+            // (byte offset >> 4) for each step (the field cannot overflow below 256 KB)
+            const uint64_t qd = make_smem_desc(q_addr, 16, 1024);
+            int kvbase = 0;      // ring position of the item's first KV tile in this tile's stream
+            int q_uses = 0;      // items in which this tile had work (phases of q_full, o_free)
+            int steps0 = 0, steps1 = 0;  // half-steps issued so far per half (phases of p_ready)
 
             for (int r = 0; !failed; ++r) {
                 const int i = item_of_round(r);
                 if (i >= num_items) break;
                 const ItemInfo it = decode(i);
                 if (it.n_max == 0) continue;
+                const int nh = pick(it.nh, t), nt = pick(it.n_tiles, t);
 
-                int qk_issued = 0;
-                const int qk_total = it.n_tiles[0] + it.n_tiles[1];
-                // S_t(j) = Q_t K_j^T; the last tile that uses K_j releases its stage
-                auto issue_qk = [&](int t, int j) -> bool {
-                    const int u = two_streams ? t : 0, g = kvbase[u] + j, st = kv_slot(u, g);
-                    if (g > k_waited[u]) {
-                        if (!mbar_wait(&k_full[st], kv_phase(g))) return false;
-                        k_waited[u] = g;
-                    }
+                // S(g) = Q K(g)^T into half g % 2 of S_t
+                auto issue_qk = [&](int g) -> bool {
+                    const int j = g >> 1, hh = g & 1, pos = kvbase + j, st = kv_slot(u, pos);
+                    if (hh == 0 && !mbar_wait(&k_full[st], kv_phase(pos))) return false;
                     tc_fence_after_sync();
-                    // descriptors differ only in the start-address field: build one per operand, then add
-                    // (byte offset >> 4) for each 16-wide K step (the field cannot overflow below 256 KB)
-                    const uint64_t qd = make_smem_desc(q_addr + t * L::kTileBytes, 16, 1024);
-                    const uint64_t kd = make_smem_desc(k_addr + st * L::kTileBytes, 16, 1024);
+                    const uint64_t kd = make_smem_desc(k_addr + st * L::kTileBytes + hh * (kHalf * 128), 16, 1024);
 #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk) {
                         const uint32_t off = ((kk / 4) * L::kChunkBytes + (kk % 4) * 32) >> 4;
-                        mma_ss(tmem_base + kColS + t * kBN, qd + off, kd + off, idesc_s, kk != 0);
+                        mma_ss(s_tmem + hh * kHalf, qd + off, kd + off, idesc_s, kk != 0);
                     }
-                    bool last = true;  // no later tile reads this K tile (always so with separate streams)
-                    for (int t2 = t + 1; t2 < kTilesPerCta && !two_streams; ++t2) last = last && !(j < it.n_tiles[t2]);
-                    if (last) mma_commit(&k_empty[st]);
-                    mma_commit(&s_full[t]);
-                    // the item's last S = Q K^T: once it completes, the next item's Q tiles may be loaded
-                    if (++qk_issued == qk_total) mma_commit(q_empty);
+                    mma_commit(&s_full[t * 2 + hh]);
+                    if (hh == 1 || g == nh - 1) mma_commit(&k_empty[st]);  // this tile's last use of the K tile
+                    if (g == nh - 1) mma_commit(&q_empty[t]);              // and of Q
                     return true;
                 };
-                // O_t += P_t(j) V_j with P_t read from tensor memory
-                auto issue_pv = [&](int t, int j) -> bool {
-                    const int u = two_streams ? t : 0, g = kvbase[u] + j, st = kv_slot(u, g);
-                    if (!mbar_wait(&p_ready[t], its[t] & 1)) return false;
-                    if (g > v_waited[u]) {
-                        if (!mbar_wait(&v_full[st], kv_phase(g))) return false;
-                        v_waited[u] = g;
-                    }
+                // O_t += P(g) V(g) with P read from tensor memory
+                auto issue_pv = [&](int g) -> bool {
+                    const int j = g >> 1, hh = g & 1, pos = kvbase + j, st = kv_slot(u, pos);
+                    if (!mbar_wait(&p_ready[t * 2 + hh], (hh ? steps1 : steps0) & 1)) return false;
+                    if (hh) ++steps1; else ++steps0;
+                    if (hh == 0 && !mbar_wait(&v_full[st], kv_phase(pos))) return false;
                     // the first product of an item overwrites O_t: the previous item's epilogue must have read it
-                    if (j == 0 && !mbar_wait(&o_free[t], (used[t] & 1) ^ 1)) return false;
+                    if (g == 0 && !mbar_wait(&o_free[t], (q_uses & 1) ^ 1)) return false;
                     tc_fence_after_sync();
                     // P: 16 keys = 8 columns of packed bf16 pairs.  V: MN-major, 16 keys = two 1024-byte groups
                     // (2048 bytes per step); the 64-wide chunks of D are 16 KB apart.
-                    const uint64_t vd = make_smem_desc(v_addr + st * L::kTileBytes, L::kChunkBytes, 1024);
-                    const uint32_t o_tmem = tmem_base + kColO + t * D, p_tmem = tmem_base + kColS + t * kBN;
-                    if (j == 0) mma_ts(o_tmem, p_tmem, vd, idesc_o, 0u);
+                    const uint64_t vd = make_smem_desc(v_addr + st * L::kTileBytes + hh * (kHalf * 128), L::kChunkBytes, 1024);
+                    const uint32_t p_tmem = s_tmem + hh * kHalf;
+                    if (g == 0) mma_ts(o_tmem, p_tmem, vd, idesc_o, 0u);
                     else mma_ts(o_tmem, p_tmem, vd, idesc_o, 1u);
 #pragma unroll
-                    for (int kk = 1; kk < kBN / 16; ++kk) mma_ts(o_tmem, p_tmem + kk * 8, vd + kk * (2048 >> 4), idesc_o, 1u);
-                    bool last = true;
-                    for (int t2 = t + 1; t2 < kTilesPerCta && !two_streams; ++t2) last = last && !(j < it.n_tiles[t2]);
-                    if (last) mma_commit(&v_empty[st]);
-                    mma_commit(&pv_done[t]);
-                    ++its[t];
+                    for (int kk = 1; kk < kHalf / 16; ++kk) mma_ts(o_tmem, p_tmem + kk * 8, vd + kk * (2048 >> 4), idesc_o, 1u);
+                    mma_commit(&pv_done[t * 2 + hh]);
+                    if (hh == 1 || g == nh - 1) mma_commit(&v_empty[st]);
                     return true;
                 };
 
-                if (!mbar_wait(q_full, items & 1)) { failed = true; break; }
-                for (int t = 0; t < kTilesPerCta && !failed; ++t)
-                    if (it.n_tiles[t] > 0 && !issue_qk(t, 0)) failed = true;
-                for (int j = 0; j < it.n_max && !failed; ++j) {
-                    for (int t = 0; t < kTilesPerCta && !failed; ++t) {
-                        if (j >= it.n_tiles[t]) continue;
-                        if (!issue_pv(t, j)) { failed = true; break; }
-                        if (j + 1 < it.n_tiles[t] && !issue_qk(t, j + 1)) { failed = true; break; }
+                if (nh > 0) {
+                    if (!mbar_wait(&q_full[t], q_uses & 1)) { failed = true; break; }
+                    if (!issue_qk(0)) { failed = true; break; }
+                    if (nh > 1 && !issue_qk(1)) { failed = true; break; }
+                    for (int g = 0; g < nh; ++g) {
+                        if (!issue_pv(g)) { failed = true; break; }
+                        if (g + 2 < nh && !issue_qk(g + 2)) { failed = true; break; }
                     }
+                    if (failed) break;
+                    ++q_uses;
                 }
-                for (int t = 0; t < kTilesPerCta; ++t) used[t] += it.n_tiles[t] > 0;
-                if (two_streams) { kvbase[0] += it.n_tiles[0]; kvbase[1] += it.n_tiles[1]; }
-                else kvbase[0] += it.n_max;
-                ++items;
+                if (two_streams) {
+                    kvbase += nt;
+                } else {
+                    // K/V tiles that only the other query tile reads: release them once they have landed
+                    for (int j = nt; j < it.n_max; ++j) {
+                        const int pos = kvbase + j, st = kv_slot(0, pos);
+                        if (!mbar_wait(&k_full[st], kv_phase(pos))) { failed = true; break; }
+                        mbar_arrive(&k_empty[st]);
+                        if (!mbar_wait(&v_full[st], kv_phase(pos))) { failed = true; break; }
+                        mbar_arrive(&v_empty[st]);
+                    }
+                    kvbase += it.n_max;
+                }
             }
         }
       }
     } else {
         // ------------------------------------------------------------------ softmax / rescale / epilogue
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
         const int t = warp >> 2;       // query tile of this warp group
         const int quarter = warp & 3;  // TMEM lane quarter this warp may access
         const int row = quarter * 32 + lane;
-        const int wg_tid = threadIdx.x & 127;  // index inside the warp group of this tile
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
         const uint32_t col_s = kColS + t * kBN, col_o = kColO + t * D;
         const float sl2 = p.scale_log2;
-        int its = 0;  // tile iterations done so far (barrier phases run across items)
-        uint32_t wg_phase = 0;
-        // the four warps of this tile meet on an mbarrier: unlike bar.sync, the wait is bounded
-        auto wg_sync = [&]() -> bool {
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&wg_bar[t]);
-            const bool ok = warp_wait(&wg_bar[t], wg_phase);
-            wg_phase ^= 1;
-            return ok;
-        };
+        const float2 sl2v = make_float2(sl2, sl2);
+        uint8_t* stage_out = smem + L::kOutOff + warp * 4096;  // this warp's 32 rows x 128 bytes
+        int steps0 = 0, steps1 = 0;  // half-steps done so far per half (barrier phases run across items)
 
         for (int r = 0; !failed; ++r) {
             const int i = item_of_round(r);
             if (i >= num_items) break;
             const ItemInfo it = decode(i);
-            const int q0 = it.q0[t];
+            const int q0 = pick(it.q0, t);
             const int qi = q0 + row;
-            const int nt = it.n_tiles[t];
-            __nv_bfloat16* orow = p.out + ((size_t)(it.b * p.Hq + it.h[t]) * p.Sq + qi) * D;
-            if (nt == 0) {  // no visible key for any row of this tile (or the tile lies beyond Sq)
+            const int nh = pick(it.nh, t);
+            const int bh = it.b * p.Hq + pick(it.h, t);
+            if (nh == 0) {  // no visible key for any row of this tile (or the tile lies beyond Sq)
                 if (qi < p.Sq) {
+                    __nv_bfloat16* orow = p.out + ((size_t)bh * p.Sq + qi) * D;
 #pragma unroll
                     for (int c = 0; c < D / 8; ++c) reinterpret_cast<uint4*>(orow)[c] = make_uint4(0, 0, 0, 0);
                 }
@@ -398,74 +398,85 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             }
             float m_run = -INFINITY;  // running maximum of the raw scores (reference of the exponentials)
             float l_run = 0.f;
-            const int row_limit = causal ? qi + causal_off : 0x7fffffff;  // last visible key of this row
-            for (int j = 0; j < nt; ++j, ++its) {
-                // S_t(j) is complete, and so is every MMA issued before it: O_t holds all earlier P V
-                // products and P_t(j-1) has been consumed.
-                if (!warp_wait(&s_full[t], its & 1)) { failed = true; break; }
+            // last visible key of this row
+            const int row_limit = min(it.kvlen - 1, causal ? qi + causal_off : 0x7fffffff);
+#pragma unroll 1
+            for (int g = 0; g < nh; ++g) {
+                const int hh = g & 1;
+                const uint32_t col_h = col_s + hh * kHalf;
+                // S(g) is complete, and so is every MMA this tile's issuer issued before it: O_t holds the
+                // P V products up to g - 2 and P(g - 2) has been consumed.
+                if (!warp_wait(&s_full[t * 2 + hh], (hh ? steps1 : steps0) & 1)) { failed = true; break; }
+                if (hh) ++steps1; else ++steps0;
                 tc_fence_after_sync();
-                float s[kBN];
+                float s[kHalf];
 #pragma unroll
-                for (int c = 0; c < kBN / 32; ++c) {
-                    uint32_t r[32];
-                    tmem_ld_x32(lane_base + col_s + c * 32, r);
+                for (int c = 0; c < kHalf / 32; ++c) {
+                    uint32_t rr[32];
+                    tmem_ld_x32(lane_base + col_h + c * 32, rr);
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) s[c * 32 + i] = __uint_as_float(r[i]);
+                    for (int k = 0; k < 32; ++k) s[c * 32 + k] = __uint_as_float(rr[k]);
                 }
                 tmem_ld_wait();
 
-                const int j0 = j * kBN;
-                const bool need_mask = (j0 + kBN > it.kvlen) || (causal && (j0 + kBN - 1 > q0 + causal_off));
+                const int key0 = (g >> 1) * kBN + hh * kHalf;
+                const bool need_mask = (key0 + kHalf > it.kvlen) || (causal && (key0 + kHalf - 1 > q0 + causal_off));
+                bool stored = false;
                 if (need_mask) {
-                    const int lim = min(it.kvlen - 1, row_limit) - j0;  // last visible column of this tile
+                    const int lim = row_limit - key0;  // last visible column of this half
+                    if (__all_sync(0xffffffffu, lim < 0)) {
+                        // nothing visible for any row of this warp: P = 0
+                        uint32_t zeros[32];
 #pragma unroll
-                    for (int i = 0; i < kBN; ++i) s[i] = (i <= lim) ? s[i] : -INFINITY;
+                        for (int k = 0; k < 32; ++k) zeros[k] = 0u;
+                        tmem_st_x32(lane_base + col_h, zeros);
+                        stored = true;
+                    } else {
+                        // a masked score of -inf gives a probability of exactly 0 below (the scale is > 0)
+#pragma unroll
+                        for (int k = 0; k < kHalf; ++k) s[k] = (k <= lim) ? s[k] : -INFINITY;
+                    }
                 }
-                const float2 sl2v = make_float2(sl2, sl2);
-                // Fast path (full tiles once every row has a finite reference): exponentials against the
-                // current reference in the same pass that finds the tile maximum.  Valid as long as no row's
+                // Fast path (once every row of the warp has a finite reference): exponentials against the
+                // current reference in the same pass that finds the maximum.  Valid as long as no row's
                 // maximum exceeds its reference by more than the threshold, which is what the lazy rescale
-                // tolerates anyway; otherwise the tile is redone below with a new reference.
-                bool done = false;
-                if (!need_mask && __all_sync(0xffffffffu, m_run != -INFINITY)) {
+                // tolerates anyway; otherwise the half is redone below with a new reference.
+                if (!stored && __all_sync(0xffffffffu, m_run != -INFINITY)) {
                     const float2 neg_m = make_float2(-m_run * sl2, -m_run * sl2);
                     float2 lsum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
                     float mx[4] = {s[0], s[1], s[2], s[3]};
+                    uint32_t packed[32];
 #pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        uint32_t packed[32];
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            const float s0 = s[half * 64 + 2 * i], s1 = s[half * 64 + 2 * i + 1];
-                            mx[i & 3] = max3(mx[i & 3], s0, s1);
-                            const float2 x = ffma2(make_float2(s0, s1), sl2v, neg_m);
-                            const float2 pr = make_float2(ex2(x.x), ex2(x.y));
-                            lsum[i & 1] = fadd2(lsum[i & 1], pr);
-                            packed[i] = pack_bf16(pr.x, pr.y);
-                        }
-                        tmem_st_x32(lane_base + col_s + half * 32, packed);
+                    for (int k = 0; k < 32; ++k) {
+                        const float s0 = s[2 * k], s1 = s[2 * k + 1];
+                        mx[k & 3] = max3(mx[k & 3], s0, s1);
+                        const float2 x = ffma2(make_float2(s0, s1), sl2v, neg_m);
+                        const float2 pr = make_float2(ex2(x.x), ex2(x.y));
+                        lsum[k & 1] = fadd2(lsum[k & 1], pr);
+                        packed[k] = pack_bf16(pr.x, pr.y);
                     }
                     const float m_tile = max3(fmaxf(mx[0], mx[1]), mx[2], mx[3]);
                     if (!__any_sync(0xffffffffu, (m_tile - m_run) * sl2 > kRescaleThreshold)) {
+                        tmem_st_x32(lane_base + col_h, packed);
                         l_run += (lsum[0].x + lsum[0].y) + (lsum[1].x + lsum[1].y);
-                        done = true;
+                        stored = true;
                     }
                 }
-                if (!done) {
+                if (!stored) {
                     // row maximum: four independent chains of 3-input maxima
                     float mx[4] = {s[0], s[1], s[2], s[3]};
-    #pragma unroll
-                    for (int i = 4; i + 7 < kBN; i += 8) {
-                        mx[0] = max3(mx[0], s[i], s[i + 1]);
-                        mx[1] = max3(mx[1], s[i + 2], s[i + 3]);
-                        mx[2] = max3(mx[2], s[i + 4], s[i + 5]);
-                        mx[3] = max3(mx[3], s[i + 6], s[i + 7]);
+#pragma unroll
+                    for (int k = 4; k + 7 < kHalf; k += 8) {
+                        mx[0] = max3(mx[0], s[k], s[k + 1]);
+                        mx[1] = max3(mx[1], s[k + 2], s[k + 3]);
+                        mx[2] = max3(mx[2], s[k + 4], s[k + 5]);
+                        mx[3] = max3(mx[3], s[k + 6], s[k + 7]);
                     }
-                    mx[0] = max3(mx[0], s[kBN - 4], s[kBN - 3]);
-                    mx[1] = max3(mx[1], s[kBN - 2], s[kBN - 1]);
+                    mx[0] = max3(mx[0], s[kHalf - 4], s[kHalf - 3]);
+                    mx[1] = max3(mx[1], s[kHalf - 2], s[kHalf - 1]);
                     const float m_tile = max3(fmaxf(mx[0], mx[1]), mx[2], mx[3]);
 
-                    // Keep the old reference unless this tile's maximum exceeds it by more than the
+                    // Keep the old reference unless this half's maximum exceeds it by more than the
                     // threshold (in log2 units of the scaled scores); then every later exponent is <= 8.
                     float alpha = 1.f;
                     bool grow = (m_tile - m_run) * sl2 > kRescaleThreshold || m_run == -INFINITY;
@@ -475,58 +486,51 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                         alpha = (m_run == -INFINITY) ? 1.f : ex2((m_run - m_tile) * sl2);
                         m_run = m_tile;
                     }
-                    if (j > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-                        // rare after the first tiles: small chunks, not unrolled, to keep register pressure low
-    #pragma unroll 1
+                    if (g > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+                        // O_t must hold every product issued so far and none may be in flight: the product of
+                        // half-step g - 1 (the other half's latest) is the only one the barrier above does not cover.
+                        if (!warp_wait(&pv_done[t * 2 + (hh ^ 1)], ((hh ? steps0 : steps1) - 1) & 1)) { failed = true; break; }
+                        tc_fence_after_sync();
+                        // rare after the first steps: small chunks, not unrolled, to keep register pressure low
+#pragma unroll 1
                         for (int c = 0; c < D / 16; ++c) {
-                            uint32_t r[16];
-                            tmem_ld_x16(lane_base + col_o + c * 16, r);
+                            uint32_t rr[16];
+                            tmem_ld_x16(lane_base + col_o + c * 16, rr);
                             tmem_ld_wait();
-    #pragma unroll
-                            for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
-                            tmem_st_x16(lane_base + col_o + c * 16, r);
+#pragma unroll
+                            for (int k = 0; k < 16; ++k) rr[k] = __float_as_uint(__uint_as_float(rr[k]) * alpha);
+                            tmem_st_x16(lane_base + col_o + c * 16, rr);
                         }
                     }
                     const float m_ref = (m_run == -INFINITY) ? 0.f : m_run;
                     const float2 neg_m = make_float2(-m_ref * sl2, -m_ref * sl2);
                     float2 lsum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-                    // P = 2^(s * sl2 - m * sl2) as packed bf16 pairs, written over the first 64 columns of S_t
-                    // in two halves.  In masked tiles the probability of a masked key is forced to exactly 0
-                    // (that also covers sl2 == 0, where -inf * 0 would be NaN); full tiles skip the selects.
-                    auto exp_and_store = [&](auto masked_tag) {
-                        constexpr bool kMasked = decltype(masked_tag)::value;
-    #pragma unroll
-                        for (int half = 0; half < 2; ++half) {
-                            uint32_t packed[32];
-    #pragma unroll
-                            for (int i = 0; i < 32; ++i) {
-                                const float s0 = s[half * 64 + 2 * i], s1 = s[half * 64 + 2 * i + 1];
-                                const float2 x = ffma2(make_float2(s0, s1), sl2v, neg_m);
-                                float2 pr = make_float2(ex2(x.x), ex2(x.y));
-                                if constexpr (kMasked) {
-                                    pr.x = (s0 == -INFINITY) ? 0.f : pr.x;
-                                    pr.y = (s1 == -INFINITY) ? 0.f : pr.y;
-                                }
-                                lsum[i & 1] = fadd2(lsum[i & 1], pr);
-                                packed[i] = pack_bf16(pr.x, pr.y);
-                            }
-                            tmem_st_x32(lane_base + col_s + half * 32, packed);
-                        }
-                    };
-                    if (need_mask) exp_and_store(std::true_type{});
-                    else exp_and_store(std::false_type{});
+                    // P = 2^(s * sl2 - m * sl2) as packed bf16 pairs, written over the first 32 columns of this
+                    // half of S_t
+                    uint32_t packed[32];
+#pragma unroll
+                    for (int k = 0; k < 32; ++k) {
+                        const float2 x = ffma2(make_float2(s[2 * k], s[2 * k + 1]), sl2v, neg_m);
+                        const float2 pr = make_float2(ex2(x.x), ex2(x.y));
+                        lsum[k & 1] = fadd2(lsum[k & 1], pr);
+                        packed[k] = pack_bf16(pr.x, pr.y);
+                    }
+                    tmem_st_x32(lane_base + col_h, packed);
                     const float l_tile = (lsum[0].x + lsum[0].y) + (lsum[1].x + lsum[1].y);
                     l_run = l_run * alpha + l_tile;
                 }
                 tmem_st_wait();
                 tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&p_ready[t]);  // one arrival per warp
+                if (lane == 0) mbar_arrive(&p_ready[t * 2 + hh]);  // one arrival per warp
             }
             if (failed) break;
-            if (!warp_wait(&pv_done[t], (its - 1) & 1)) { failed = true; break; }
+            // The last product of either half (every S barrier seen covers that half's product before the
+            // latest, so each wait is at most one completion behind and the phase parity identifies it).
+            if (steps0 > 0 && !warp_wait(&pv_done[t * 2], (steps0 - 1) & 1)) { failed = true; break; }
+            if (steps1 > 0 && !warp_wait(&pv_done[t * 2 + 1], (steps1 - 1) & 1)) { failed = true; break; }
             tc_fence_after_sync();
-            // O_t -> registers, then hand O_t back to the MMA warp before the stores go out
+            // O_t -> registers, then hand O_t back to the issuer before the stores go out
             uint32_t o[D];
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
@@ -539,15 +543,15 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&o_free[t]);
-            // O / l as bf16 through a 128-byte-swizzled staging buffer and one TMA store per 64 columns
-            // (rows beyond Sq are clipped by the TMA unit).  The store drains while the next item starts.
+            // O / l as bf16 through this warp's 128-byte-swizzled staging rows and one TMA store per 64
+            // columns (rows beyond Sq are clipped by the TMA unit).  The store drains while the next item runs.
             {
                 const float inv = l_run > 0.f ? 1.f / l_run : 0.f;  // no visible key: zeros
-                uint8_t* stage_out = smem + L::kOutOff + t * L::kChunkBytes;
+                const int row0 = q0 + quarter * 32;
 #pragma unroll
                 for (int cb = 0; cb < D / 64; ++cb) {
-                    if (wg_tid == 0) tma_store_wait_read<0>();  // the previous store has read the buffer
-                    if (!wg_sync()) { failed = true; break; }
+                    if (lane == 0) tma_store_wait_read<0>();  // the previous store has read the staging rows
+                    __syncwarp();
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
                         uint32_t w[4];
@@ -555,19 +559,19 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                         for (int k = 0; k < 4; ++k)
                             w[k] = pack_bf16(__uint_as_float(o[cb * 64 + c * 8 + 2 * k]) * inv,
                                              __uint_as_float(o[cb * 64 + c * 8 + 2 * k + 1]) * inv);
-                        *reinterpret_cast<uint4*>(stage_out + row * 128 + ((c ^ (row & 7)) << 4)) =
+                        *reinterpret_cast<uint4*>(stage_out + lane * 128 + ((c ^ (lane & 7)) << 4)) =
                             make_uint4(w[0], w[1], w[2], w[3]);
                     }
                     fence_proxy_async_smem();
-                    if (!wg_sync()) { failed = true; break; }
-                    if (wg_tid == 0) {
-                        tma_store_3d(&tmap_o, stage_out, cb * 64, q0, it.b * p.Hq + it.h[t]);
+                    __syncwarp();
+                    if (lane == 0 && row0 < p.Sq) {
+                        tma_store_3d(&tmap_o, stage_out, cb * 64, row0, bh);
                         tma_store_commit();
                     }
                 }
             }
         }
-        if (wg_tid == 0) tma_store_wait_all<0>();  // every output tile has left shared memory and is written
+        if (lane == 0) tma_store_wait_all<0>();  // every output tile has left shared memory and is written
     }
 
     if (failed) {
@@ -601,9 +605,11 @@ int launch_attn(const void* q, const void* k, const void* v, void* out, int B, i
     }
     CUtensorMap to;
     {
+        // the output leaves in boxes of 32 rows, one per softmax warp
+        const uint32_t box_o[3] = {64, 32, 1};
         const uint64_t dims[3] = {(uint64_t)D, (uint64_t)Sq, (uint64_t)B * Hq};
         const uint64_t strides[2] = {(uint64_t)D * 2, (uint64_t)Sq * D * 2};
-        if (!encode_tmap_bf16_sw128(&to, out, 3, dims, strides, box)) return FORGE_ERR_CUDA;
+        if (!encode_tmap_bf16_sw128(&to, out, 3, dims, strides, box_o)) return FORGE_ERR_CUDA;
     }
     AttnParams p;
     p.out = static_cast<__nv_bfloat16*>(out);
@@ -611,6 +617,8 @@ int launch_attn(const void* q, const void* k, const void* v, void* out, int B, i
     p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.Sq = Sq; p.Skv = Skv;
     p.mask_kind = mask_kind;
     p.scale_log2 = scale * 1.4426950408889634f;
+    // scale = 0 (uniform weights): any positive multiplier whose products with the scores flush to zero
+    if (!(p.scale_log2 > 0.f)) p.scale_log2 = 1.17549435e-38f;
     p.status = device_status_word();
     if (!p.status) return FORGE_ERR_CUDA;
     auto kernel = attn_bf16_kernel<D>;

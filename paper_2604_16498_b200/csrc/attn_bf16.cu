@@ -8,7 +8,7 @@
 // Warp roles:
 //   warps 0-3 : softmax / rescale / epilogue of tile 0; thread = one query row (TMEM lane), so row
 //   warps 4-7 : the same for tile 1                    maxima and sums need no cross-thread reduction
-//   warp 8    : TMA producer: Q tiles, then K and V tiles (128 keys) through rings
+//   warp 8    : TMA producer: Q tiles, then K and V tiles (64 keys, one per half-step) through rings
 //   warp 9    : tcgen05.mma issuer of tile 0 (one elected lane), owns the TMEM allocation
 //   warp 10   : tcgen05.mma issuer of tile 1
 //   warp 11 only completes the third warpgroup, which hands registers to the other two
@@ -24,6 +24,8 @@
 // Q and K are K-major operands, V [keys, D] is the MN-major B operand of P V.
 #include <cuda_bf16.h>
 
+#include <type_traits>
+
 #include "forge_common.cuh"
 #include "sm100_ptx.cuh"
 #include "tmap.cuh"
@@ -35,24 +37,33 @@ using namespace ptx;
 
 constexpr int kBM = 128;          // query rows per tile
 constexpr int kTilesPerCta = 2;
-constexpr int kBN = 128;          // keys per K/V tile in shared memory
-constexpr int kHalf = 64;         // keys per half-step
+constexpr int kBN = 128;          // keys per tile of S (two half-steps)
+constexpr int kHalf = 64;         // keys per half-step and per K/V tile in shared memory
 constexpr int kThreads = 384;
 constexpr int kTmemCols = 512;
 constexpr int kColS = 0;          // S_t at t * 128
 constexpr int kColO = 256;        // O_t at 256 + t * D
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
+#ifndef FORGE_ATTN_FMA_EXP_PAIRS
+#define FORGE_ATTN_FMA_EXP_PAIRS 8
+#endif
+// of the 32 score pairs of a half-step, how many take their exponentials on the FMA pipe (unmasked steps)
+constexpr int kFmaExpPairs = FORGE_ATTN_FMA_EXP_PAIRS;
 
 template <int D>
 struct AttnSmem {
-    static constexpr int kChunkBytes = 128 * 128;              // 128 rows x 64 bf16 (one swizzle span wide)
-    static constexpr int kTileBytes = (D / 64) * kChunkBytes;  // a Q, K or V tile
-    static constexpr int kKVStages = (D == 64) ? 4 : 2;
+    static constexpr int kChunkBytes = 128 * 128;              // Q: 128 rows x 64 bf16 (one swizzle span wide)
+    static constexpr int kTileBytes = (D / 64) * kChunkBytes;  // a Q tile
+    static constexpr int kKVChunkBytes = kHalf * 128;          // K, V: 64 keys x 64 bf16
+    static constexpr int kKVTileBytes = (D / 64) * kKVChunkBytes;
+    static constexpr int kKVStages = (D == 64) ? 8 : 3;
     static constexpr int kQOff = 0;
     static constexpr int kKOff = kQOff + kTilesPerCta * kTileBytes;
-    static constexpr int kVOff = kKOff + kKVStages * kTileBytes;
-    static constexpr int kOutOff = kVOff + kKVStages * kTileBytes;  // output staging: 32 rows x 64 bf16 per softmax warp
-    static constexpr int kBarOff = kOutOff + 8 * 4096;
+    static constexpr int kVOff = kKOff + kKVStages * kKVTileBytes;
+    // output staging: 32 rows x 64 bf16 per softmax warp and 64-column block of D
+    static constexpr int kOutOff = kVOff + kKVStages * kKVTileBytes;
+    static constexpr int kOutWarpBytes = (D / 64) * 4096;
+    static constexpr int kBarOff = kOutOff + 8 * kOutWarpBytes;
     // q_full[2], q_empty[2], k/v full+empty per stage, s_full[4], p_ready[4], pv_done[4], o_free[2]
     static constexpr int kNumBars = 4 + 4 * kKVStages + 14;
     static constexpr int kTotal = kBarOff + kNumBars * 8 + 16;
@@ -92,9 +103,42 @@ __device__ __forceinline__ float2 fadd2(float2 a, float2 b) {
     return d;
 }
 
+// 2^x for two values on the FMA and integer pipes instead of the special-function unit (which is the
+// narrowest pipe of the softmax): x = n + f with n = round(x), f in [-0.5, 0.5]; 2^f by a cubic with a
+// relative error of 7.6e-5 (far below the bf16 rounding of P); n is added to the exponent field.
+// Inputs below -125 give 2^-125 rather than 0, so this is used only where no score is masked.
+__device__ __forceinline__ float2 ex2_fma2(float2 x) {
+    const float kMagic = 12582912.f;  // 1.5 * 2^23: adding it leaves round(x) in the low mantissa bits
+    x.x = fmaxf(x.x, -125.f);
+    x.y = fmaxf(x.y, -125.f);
+    const float2 t = fadd2(x, make_float2(kMagic, kMagic));
+    const float2 n = fadd2(t, make_float2(-kMagic, -kMagic));
+    const float2 f = ffma2(n, make_float2(-1.f, -1.f), x);
+    float2 q = ffma2(f, make_float2(0.05520550534f, 0.05520550534f), make_float2(0.2426139712f, 0.2426139712f));
+    q = ffma2(q, f, make_float2(0.6932547688f, 0.6932547688f));
+    q = ffma2(q, f, make_float2(0.9999276996f, 0.9999276996f));
+    return make_float2(__int_as_float(__float_as_int(q.x) + (__float_as_int(t.x) << 23)),
+                       __int_as_float(__float_as_int(q.y) + (__float_as_int(t.y) << 23)));
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Division by a divisor fixed at launch: floor(n / d) = high 64 bits of n * ceil(2^64 / d) for 0 <= n < 2^32.
+struct FastDiv {
+    unsigned long long m;  // ceil(2^64 / d); unused for d == 1
+    int d;
+};
+inline FastDiv make_fastdiv(int d) {
+    FastDiv f;
+    f.d = d;
+    f.m = d > 1 ? ~0ull / (unsigned long long)d + 1ull : 0ull;
+    return f;
+}
+__device__ __forceinline__ int fast_div(int n, const FastDiv& f) {
+    return f.d == 1 ? n : (int)__umul64hi((unsigned long long)(unsigned)n, f.m);
 }
 
 struct AttnParams {
@@ -103,6 +147,9 @@ struct AttnParams {
     int B, Hq, Hkv, Sq, Skv;
     int mask_kind;
     float scale_log2;  // > 0 (a zero scale is passed as the smallest normal number: every product flushes to 0)
+    FastDiv div_heads;  // by the number of items per query step
+    FastDiv div_inner;  // by the head pairs (or heads) per batch entry
+    FastDiv div_group;  // by the query heads per KV head
     int* status;
 };
 
@@ -113,8 +160,7 @@ struct ItemInfo {
     int q0[kTilesPerCta];       // first query row of each of the two tiles
     int h[kTilesPerCta];        // query head of each tile
     int nh[kTilesPerCta];       // 64-key half-steps visible to at least one row of each query tile (0: no work)
-    int n_tiles[kTilesPerCta];  // the same in 128-key tiles
-    int n_max;
+    int n_max;                  // the larger of the two
 };
 
 // element t of a two-element array without dynamic indexing (keeps the array in registers)
@@ -153,7 +199,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     const bool pair_heads = (G % 2) == 0;
     // With an odd group size and D = 64 (where shared memory has room for it) the two tiles are still two
     // heads on the same query rows, each with its own K/V stream through half of the stage ring.
-    const bool two_streams = !pair_heads && kKVStages >= 4;
+    const bool two_streams = !pair_heads && kKVStages >= 8;
     const int ring_len = two_streams ? kKVStages / 2 : kKVStages;
     const int num_q_tiles = (p.Sq + kBM - 1) / kBM;
     const int head_pairs = (p.Hq + 1) / 2;
@@ -175,22 +221,22 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     };
     auto decode = [&](int i) {
         ItemInfo it;
-        const int qstep = rows_of_items - 1 - i / heads;  // longest (causal) first
-        const int hb = i % heads;
+        const int round_q = fast_div(i, p.div_heads);
+        const int qstep = rows_of_items - 1 - round_q;  // longest (causal) first
+        const int hb = i - round_q * heads;
+        it.b = fast_div(hb, p.div_inner);
         if (pair_heads || two_streams) {
-            const int hp = hb % head_pairs;
-            it.b = hb / head_pairs;
+            const int hp = hb - it.b * head_pairs;
             it.h[0] = 2 * hp;
             it.h[1] = min(2 * hp + 1, p.Hq - 1);
             it.q0[0] = it.q0[1] = qstep * kBM;
             if (2 * hp + 1 >= p.Hq) it.q0[1] = num_q_tiles * kBM;  // odd head count: no second tile
         } else {
-            it.b = hb / p.Hq;
-            it.h[0] = it.h[1] = hb % p.Hq;
+            it.h[0] = it.h[1] = hb - it.b * p.Hq;
             it.q0[0] = 2 * qstep * kBM; it.q0[1] = (2 * qstep + 1) * kBM;
         }
-        it.kvh[0] = it.h[0] / G;
-        it.kvh[1] = it.h[1] / G;
+        it.kvh[0] = fast_div(it.h[0], p.div_group);
+        it.kvh[1] = fast_div(it.h[1], p.div_group);
         it.kvlen = p.Skv;
         if (p.mask_kind & FORGE_MASK_PADDING) it.kvlen = min(max(p.lens[it.b], 0), p.Skv);
         it.n_max = 0;
@@ -202,8 +248,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             if (q0 >= p.Sq) kv_end = 0;
             kv_end = max(kv_end, 0);
             it.nh[t] = (kv_end + kHalf - 1) / kHalf;
-            it.n_tiles[t] = (it.nh[t] + 1) / 2;
-            it.n_max = max(it.n_max, it.n_tiles[t]);
+            it.n_max = max(it.n_max, it.nh[t]);
         }
         return it;
     };
@@ -259,22 +304,22 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {
                         if (u == 1 && !two_streams) continue;
-                        if (two_streams && j >= it.n_tiles[u]) continue;
+                        if (two_streams && j >= it.nh[u]) continue;
                         const int g = kvn[u]++, st = kv_slot(u, g);
                         const uint32_t ph = kv_phase(g);
                         const int kv_row = it.b * p.Hkv + it.kvh[u];
                         if (!mbar_wait(&k_empty[st], ph ^ 1)) { failed = true; break; }
-                        mbar_expect_tx(&k_full[st], L::kTileBytes);
+                        mbar_expect_tx(&k_full[st], L::kKVTileBytes);
 #pragma unroll
                         for (int c = 0; c < D / 64; ++c)
-                            tma_load_3d(sK + st * L::kTileBytes + c * L::kChunkBytes, &tmap_k, &k_full[st], c * 64,
-                                        j * kBN, kv_row);
+                            tma_load_3d(sK + st * L::kKVTileBytes + c * L::kKVChunkBytes, &tmap_k, &k_full[st], c * 64,
+                                        j * kHalf, kv_row);
                         if (!mbar_wait(&v_empty[st], ph ^ 1)) { failed = true; break; }
-                        mbar_expect_tx(&v_full[st], L::kTileBytes);
+                        mbar_expect_tx(&v_full[st], L::kKVTileBytes);
 #pragma unroll
                         for (int c = 0; c < D / 64; ++c)
-                            tma_load_3d(sV + st * L::kTileBytes + c * L::kChunkBytes, &tmap_v, &v_full[st], c * 64,
-                                        j * kBN, kv_row);
+                            tma_load_3d(sV + st * L::kKVTileBytes + c * L::kKVChunkBytes, &tmap_v, &v_full[st], c * 64,
+                                        j * kHalf, kv_row);
                     }
                 }
             }
@@ -295,48 +340,55 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             int q_uses = 0;      // items in which this tile had work (phases of q_full, o_free)
             int steps0 = 0, steps1 = 0;  // half-steps issued so far per half (phases of p_ready)
 
-            for (int r = 0; !failed; ++r) {
-                const int i = item_of_round(r);
-                if (i >= num_items) break;
-                const ItemInfo it = decode(i);
-                if (it.n_max == 0) continue;
-                const int nh = pick(it.nh, t), nt = pick(it.n_tiles, t);
+            ItemInfo it;
+            int i_cur = item_of_round(0);
+            if (i_cur < num_items) it = decode(i_cur);
+            for (int r = 0; !failed && i_cur < num_items; ++r) {
+                const int i_next = item_of_round(r + 1);
+                ItemInfo it_next;
+                if (it.n_max == 0) {
+                    if (i_next < num_items) it_next = decode(i_next);
+                    it = it_next; i_cur = i_next;
+                    continue;
+                }
+                const int nh = pick(it.nh, t);
 
                 // S(g) = Q K(g)^T into half g % 2 of S_t
                 auto issue_qk = [&](int g) -> bool {
-                    const int j = g >> 1, hh = g & 1, pos = kvbase + j, st = kv_slot(u, pos);
-                    if (hh == 0 && !mbar_wait(&k_full[st], kv_phase(pos))) return false;
+                    const int hh = g & 1, pos = kvbase + g, st = kv_slot(u, pos);
+                    if (!mbar_wait(&k_full[st], kv_phase(pos))) return false;
                     tc_fence_after_sync();
-                    const uint64_t kd = make_smem_desc(k_addr + st * L::kTileBytes + hh * (kHalf * 128), 16, 1024);
+                    const uint64_t kd = make_smem_desc(k_addr + st * L::kKVTileBytes, 16, 1024);
 #pragma unroll
                     for (int kk = 0; kk < D / 16; ++kk) {
-                        const uint32_t off = ((kk / 4) * L::kChunkBytes + (kk % 4) * 32) >> 4;
-                        mma_ss(s_tmem + hh * kHalf, qd + off, kd + off, idesc_s, kk != 0);
+                        const uint32_t qoff = ((kk / 4) * L::kChunkBytes + (kk % 4) * 32) >> 4;
+                        const uint32_t koff = ((kk / 4) * L::kKVChunkBytes + (kk % 4) * 32) >> 4;
+                        mma_ss(s_tmem + hh * kHalf, qd + qoff, kd + koff, idesc_s, kk != 0);
                     }
                     mma_commit(&s_full[t * 2 + hh]);
-                    if (hh == 1 || g == nh - 1) mma_commit(&k_empty[st]);  // this tile's last use of the K tile
-                    if (g == nh - 1) mma_commit(&q_empty[t]);              // and of Q
+                    mma_commit(&k_empty[st]);                  // this tile is done with the K tile
+                    if (g == nh - 1) mma_commit(&q_empty[t]);  // and, after the item's last S, with Q
                     return true;
                 };
                 // O_t += P(g) V(g) with P read from tensor memory
                 auto issue_pv = [&](int g) -> bool {
-                    const int j = g >> 1, hh = g & 1, pos = kvbase + j, st = kv_slot(u, pos);
+                    const int hh = g & 1, pos = kvbase + g, st = kv_slot(u, pos);
                     if (!mbar_wait(&p_ready[t * 2 + hh], (hh ? steps1 : steps0) & 1)) return false;
                     if (hh) ++steps1; else ++steps0;
-                    if (hh == 0 && !mbar_wait(&v_full[st], kv_phase(pos))) return false;
+                    if (!mbar_wait(&v_full[st], kv_phase(pos))) return false;
                     // the first product of an item overwrites O_t: the previous item's epilogue must have read it
                     if (g == 0 && !mbar_wait(&o_free[t], (q_uses & 1) ^ 1)) return false;
                     tc_fence_after_sync();
                     // P: 16 keys = 8 columns of packed bf16 pairs.  V: MN-major, 16 keys = two 1024-byte groups
-                    // (2048 bytes per step); the 64-wide chunks of D are 16 KB apart.
-                    const uint64_t vd = make_smem_desc(v_addr + st * L::kTileBytes + hh * (kHalf * 128), L::kChunkBytes, 1024);
+                    // (2048 bytes per step); the 64-wide chunks of D are 8 KB apart.
+                    const uint64_t vd = make_smem_desc(v_addr + st * L::kKVTileBytes, L::kKVChunkBytes, 1024);
                     const uint32_t p_tmem = s_tmem + hh * kHalf;
                     if (g == 0) mma_ts(o_tmem, p_tmem, vd, idesc_o, 0u);
                     else mma_ts(o_tmem, p_tmem, vd, idesc_o, 1u);
 #pragma unroll
                     for (int kk = 1; kk < kHalf / 16; ++kk) mma_ts(o_tmem, p_tmem + kk * 8, vd + kk * (2048 >> 4), idesc_o, 1u);
                     mma_commit(&pv_done[t * 2 + hh]);
-                    if (hh == 1 || g == nh - 1) mma_commit(&v_empty[st]);
+                    mma_commit(&v_empty[st]);
                     return true;
                 };
 
@@ -344,6 +396,10 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     if (!mbar_wait(&q_full[t], q_uses & 1)) { failed = true; break; }
                     if (!issue_qk(0)) { failed = true; break; }
                     if (nh > 1 && !issue_qk(1)) { failed = true; break; }
+                }
+                // the next item's coordinates, worked out while the softmax warps are busy with the first S
+                if (i_next < num_items) it_next = decode(i_next);
+                if (nh > 0) {
                     for (int g = 0; g < nh; ++g) {
                         if (!issue_pv(g)) { failed = true; break; }
                         if (g + 2 < nh && !issue_qk(g + 2)) { failed = true; break; }
@@ -352,10 +408,10 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     ++q_uses;
                 }
                 if (two_streams) {
-                    kvbase += nt;
+                    kvbase += nh;
                 } else {
                     // K/V tiles that only the other query tile reads: release them once they have landed
-                    for (int j = nt; j < it.n_max; ++j) {
+                    for (int j = nh; j < it.n_max; ++j) {
                         const int pos = kvbase + j, st = kv_slot(0, pos);
                         if (!mbar_wait(&k_full[st], kv_phase(pos))) { failed = true; break; }
                         mbar_arrive(&k_empty[st]);
@@ -364,6 +420,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     }
                     kvbase += it.n_max;
                 }
+                it = it_next; i_cur = i_next;
             }
         }
       }
@@ -377,13 +434,15 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
         const uint32_t col_s = kColS + t * kBN, col_o = kColO + t * D;
         const float sl2 = p.scale_log2;
         const float2 sl2v = make_float2(sl2, sl2);
-        uint8_t* stage_out = smem + L::kOutOff + warp * 4096;  // this warp's 32 rows x 128 bytes
+        uint8_t* stage_out = smem + L::kOutOff + warp * L::kOutWarpBytes;  // this warp's 32 rows x 128 bytes per block
         int steps0 = 0, steps1 = 0;  // half-steps done so far per half (barrier phases run across items)
 
-        for (int r = 0; !failed; ++r) {
-            const int i = item_of_round(r);
-            if (i >= num_items) break;
-            const ItemInfo it = decode(i);
+        ItemInfo it;
+        int i_cur = item_of_round(0);
+        if (i_cur < num_items) it = decode(i_cur);
+        for (int r = 0; !failed && i_cur < num_items; ++r) {
+            const int i_next = item_of_round(r + 1);
+            ItemInfo it_next;
             const int q0 = pick(it.q0, t);
             const int qi = q0 + row;
             const int nh = pick(it.nh, t);
@@ -394,6 +453,8 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
 #pragma unroll
                     for (int c = 0; c < D / 8; ++c) reinterpret_cast<uint4*>(orow)[c] = make_uint4(0, 0, 0, 0);
                 }
+                if (i_next < num_items) it_next = decode(i_next);
+                it = it_next; i_cur = i_next;
                 continue;
             }
             float m_run = -INFINITY;  // running maximum of the raw scores (reference of the exponentials)
@@ -442,25 +503,32 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 // maximum exceeds its reference by more than the threshold, which is what the lazy rescale
                 // tolerates anyway; otherwise the half is redone below with a new reference.
                 if (!stored && __all_sync(0xffffffffu, m_run != -INFINITY)) {
-                    const float2 neg_m = make_float2(-m_run * sl2, -m_run * sl2);
-                    float2 lsum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-                    float mx[4] = {s[0], s[1], s[2], s[3]};
-                    uint32_t packed[32];
+                    auto fast_path = [&](auto fma_tag) {
+                        constexpr bool kUseFma = decltype(fma_tag)::value;
+                        const float2 neg_m = make_float2(-m_run * sl2, -m_run * sl2);
+                        float2 lsum[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+                        float mx[4] = {s[0], s[1], s[2], s[3]};
+                        uint32_t packed[32];
 #pragma unroll
-                    for (int k = 0; k < 32; ++k) {
-                        const float s0 = s[2 * k], s1 = s[2 * k + 1];
-                        mx[k & 3] = max3(mx[k & 3], s0, s1);
-                        const float2 x = ffma2(make_float2(s0, s1), sl2v, neg_m);
-                        const float2 pr = make_float2(ex2(x.x), ex2(x.y));
-                        lsum[k & 1] = fadd2(lsum[k & 1], pr);
-                        packed[k] = pack_bf16(pr.x, pr.y);
-                    }
-                    const float m_tile = max3(fmaxf(mx[0], mx[1]), mx[2], mx[3]);
-                    if (!__any_sync(0xffffffffu, (m_tile - m_run) * sl2 > kRescaleThreshold)) {
-                        tmem_st_x32(lane_base + col_h, packed);
-                        l_run += (lsum[0].x + lsum[0].y) + (lsum[1].x + lsum[1].y);
-                        stored = true;
-                    }
+                        for (int k = 0; k < 32; ++k) {
+                            const float s0 = s[2 * k], s1 = s[2 * k + 1];
+                            mx[k & 3] = max3(mx[k & 3], s0, s1);
+                            const float2 x = ffma2(make_float2(s0, s1), sl2v, neg_m);
+                            // evenly spaced pairs go to the FMA pipe, the rest to the special-function unit
+                            const bool on_fma = kUseFma && ((k + 1) * kFmaExpPairs / 32) != (k * kFmaExpPairs / 32);
+                            const float2 pr = on_fma ? ex2_fma2(x) : make_float2(ex2(x.x), ex2(x.y));
+                            lsum[k & 1] = fadd2(lsum[k & 1], pr);
+                            packed[k] = pack_bf16(pr.x, pr.y);
+                        }
+                        const float m_tile = max3(fmaxf(mx[0], mx[1]), mx[2], mx[3]);
+                        if (!__any_sync(0xffffffffu, (m_tile - m_run) * sl2 > kRescaleThreshold)) {
+                            tmem_st_x32(lane_base + col_h, packed);
+                            l_run += (lsum[0].x + lsum[0].y) + (lsum[1].x + lsum[1].y);
+                            stored = true;
+                        }
+                    };
+                    if (need_mask) fast_path(std::false_type{});
+                    else fast_path(std::true_type{});
                 }
                 if (!stored) {
                     // row maximum: four independent chains of 3-input maxima
@@ -525,51 +593,52 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 if (lane == 0) mbar_arrive(&p_ready[t * 2 + hh]);  // one arrival per warp
             }
             if (failed) break;
+            // the next item's coordinates, worked out while the last products are still running
+            if (i_next < num_items) it_next = decode(i_next);
             // The last product of either half (every S barrier seen covers that half's product before the
             // latest, so each wait is at most one completion behind and the phase parity identifies it).
             if (steps0 > 0 && !warp_wait(&pv_done[t * 2], (steps0 - 1) & 1)) { failed = true; break; }
             if (steps1 > 0 && !warp_wait(&pv_done[t * 2 + 1], (steps1 - 1) & 1)) { failed = true; break; }
             tc_fence_after_sync();
-            // O_t -> registers, then hand O_t back to the issuer before the stores go out
-            uint32_t o[D];
-#pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
-                uint32_t rr[32];
-                tmem_ld_x32(lane_base + col_o + c * 32, rr);
-#pragma unroll
-                for (int k = 0; k < 32; ++k) o[c * 32 + k] = rr[k];
-            }
-            tmem_ld_wait();
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&o_free[t]);
-            // O / l as bf16 through this warp's 128-byte-swizzled staging rows and one TMA store per 64
-            // columns (rows beyond Sq are clipped by the TMA unit).  The store drains while the next item runs.
+            // O / l as bf16 through this warp's 128-byte-swizzled staging rows (32 rows x 64 columns per
+            // block of D) and one TMA store per block; rows beyond Sq are clipped by the TMA unit.  A short
+            // rolled loop: the code runs once per item, so its footprint matters more than its issue count.
             {
                 const float inv = l_run > 0.f ? 1.f / l_run : 0.f;  // no visible key: zeros
-                const int row0 = q0 + quarter * 32;
+                if (lane == 0) tma_store_wait_read<0>();  // the previous item's stores have read the staging rows
+                __syncwarp();
+                uint32_t cur[32];
+                tmem_ld_x32(lane_base + col_o, cur);
+#pragma unroll 1
+                for (int c32 = 0; c32 < D / 32; ++c32) {
+                    tmem_ld_wait();
+                    uint32_t w[16];
 #pragma unroll
-                for (int cb = 0; cb < D / 64; ++cb) {
-                    if (lane == 0) tma_store_wait_read<0>();  // the previous store has read the staging rows
-                    __syncwarp();
+                    for (int k = 0; k < 16; ++k)
+                        w[k] = pack_bf16(__uint_as_float(cur[2 * k]) * inv, __uint_as_float(cur[2 * k + 1]) * inv);
+                    if (c32 + 1 < D / 32) tmem_ld_x32(lane_base + col_o + (c32 + 1) * 32, cur);
+                    // 32 columns = four 16-byte chunks of this row's 128-byte line in block c32 / 2
+                    uint8_t* line = stage_out + (c32 >> 1) * 4096 + lane * 128;
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        uint32_t w[4];
+                    for (int c = 0; c < 4; ++c)
+                        *reinterpret_cast<uint4*>(line + ((((c32 & 1) * 4 + c) ^ (lane & 7)) << 4)) =
+                            make_uint4(w[4 * c], w[4 * c + 1], w[4 * c + 2], w[4 * c + 3]);
+                }
+                // O_t is in shared memory: hand it back to the issuer before the stores go out
+                tc_fence_before_sync();
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(&o_free[t]);
+                    const int row0 = q0 + quarter * 32;
+                    if (row0 < p.Sq) {
 #pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            w[k] = pack_bf16(__uint_as_float(o[cb * 64 + c * 8 + 2 * k]) * inv,
-                                             __uint_as_float(o[cb * 64 + c * 8 + 2 * k + 1]) * inv);
-                        *reinterpret_cast<uint4*>(stage_out + lane * 128 + ((c ^ (lane & 7)) << 4)) =
-                            make_uint4(w[0], w[1], w[2], w[3]);
-                    }
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0 && row0 < p.Sq) {
-                        tma_store_3d(&tmap_o, stage_out, cb * 64, row0, bh);
+                        for (int cb = 0; cb < D / 64; ++cb) tma_store_3d(&tmap_o, stage_out + cb * 4096, cb * 64, row0, bh);
                         tma_store_commit();
                     }
                 }
             }
+            it = it_next; i_cur = i_next;
         }
         if (lane == 0) tma_store_wait_all<0>();  // every output tile has left shared memory and is written
     }
@@ -598,10 +667,11 @@ int launch_attn(const void* q, const void* k, const void* v, void* out, int B, i
         if (!encode_tmap_bf16_sw128(&tq, q, 3, dims, strides, box)) return FORGE_ERR_CUDA;
     }
     {
+        const uint32_t box_kv[3] = {64, (uint32_t)kHalf, 1};
         const uint64_t dims[3] = {(uint64_t)D, (uint64_t)Skv, (uint64_t)B * Hkv};
         const uint64_t strides[2] = {(uint64_t)D * 2, (uint64_t)Skv * D * 2};
-        if (!encode_tmap_bf16_sw128(&tk, k, 3, dims, strides, box)) return FORGE_ERR_CUDA;
-        if (!encode_tmap_bf16_sw128(&tv, v, 3, dims, strides, box)) return FORGE_ERR_CUDA;
+        if (!encode_tmap_bf16_sw128(&tk, k, 3, dims, strides, box_kv)) return FORGE_ERR_CUDA;
+        if (!encode_tmap_bf16_sw128(&tv, v, 3, dims, strides, box_kv)) return FORGE_ERR_CUDA;
     }
     CUtensorMap to;
     {
@@ -621,12 +691,20 @@ int launch_attn(const void* q, const void* k, const void* v, void* out, int B, i
     if (!(p.scale_log2 > 0.f)) p.scale_log2 = 1.17549435e-38f;
     p.status = device_status_word();
     if (!p.status) return FORGE_ERR_CUDA;
+    {
+        const int G = Hq / Hkv;
+        const bool by_pairs = (G % 2 == 0) || L::kKVStages >= 8;  // same rule as in the kernel
+        const int inner = by_pairs ? (Hq + 1) / 2 : Hq;
+        p.div_heads = make_fastdiv(inner * B);
+        p.div_inner = make_fastdiv(inner);
+        p.div_group = make_fastdiv(G);
+    }
     auto kernel = attn_bf16_kernel<D>;
     FORGE_SET_SMEM_ONCE(kernel, L::kAlloc);
     const int sms = sm_count();
     if (sms <= 0) return FORGE_ERR_CUDA;
     const int q_tiles = (Sq + kBM - 1) / kBM;
-    const bool head_pairs = ((Hq / Hkv) % 2 == 0) || L::kKVStages >= 4;  // same rule as in the kernel
+    const bool head_pairs = ((Hq / Hkv) % 2 == 0) || L::kKVStages >= 8;  // same rule as in the kernel
     const long long items = head_pairs ? (long long)((Hq + 1) / 2) * B * q_tiles
                                        : (long long)Hq * B * ((q_tiles + 1) / 2);
     const int grid = items < sms ? (int)items : sms;

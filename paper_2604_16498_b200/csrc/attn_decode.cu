@@ -12,7 +12,11 @@
 // 16-row blocks in shared memory filled by 16-byte asynchronous copies that run ahead across
 // item boundaries (8 warps x 24 KB in flight per SM, 512 contiguous bytes per instruction,
 // zero-fill instead of reads past the end of a split), and writes its partial straight from
-// registers.  No warp ever waits for another one.  The G = Hq / Hkv query heads that share a KV
+// registers.  No warp ever waits for another one.  Items differ in length by up to the ratio of the
+// longest to the shortest cached sequence, so they are dealt out longest sequence first and in
+// alternating direction from round to round (a worker that got one of the longest items in one round
+// gets one of the shortest in the next), which keeps the workers' totals close together.
+// The G = Hq / Hkv query heads that share a KV
 // head are processed together, so every cached row is read exactly once.  The dot products run
 // on warp-level tensor-core MMAs (m16n8k16) with fragments read from the swizzled ring; fp32 FMAs
 // with shuffle reductions were bound by instruction issue.
@@ -29,6 +33,7 @@ constexpr int kWarps = 8;
 constexpr int kThreads = kWarps * 32;
 constexpr int kBlockKeys = 16;             // cached rows per ring stage
 constexpr int kWarpRingBytes = 24 * 1024;  // per warp
+constexpr int kMaxSortedBatch = 64;        // batches up to this size are ordered by cached length
 
 // 16-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros and reads nothing.
 __device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gsrc, uint32_t src_bytes) {
@@ -72,12 +77,16 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
 struct Item {
     int b, kvh, split, s0, s1;
 };
-__device__ __forceinline__ Item make_item(int idx, const int32_t* lens, int Hkv, int Smax, int num_splits) {
+// idx counts items in dealing order: all (kv head, split) pairs of the longest sequence, then of the
+// next one, ...; order[r] is the batch entry with the r-th longest cached sequence (nullptr: identity).
+__device__ __forceinline__ Item make_item(int idx, const int32_t* lens, const int* order, int Hkv, int Smax,
+                                          int num_splits) {
     Item it;
     it.split = idx % num_splits;
     const int bk = idx / num_splits;
     it.kvh = bk % Hkv;
     it.b = bk / Hkv;
+    if (order) it.b = order[it.b];
     const int len = min(max(lens[it.b], 0), Smax);
     const int per = (len + num_splits - 1) / num_splits;
     it.s0 = it.split * per;
@@ -108,6 +117,10 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     constexpr int kStages = kWarpRingBytes / kStageBytes;  // 3 for D = 128, 6 for D = 64
     static_assert(kStages >= 2, "ring too small");
 
+    // Let the combine kernel (launched with programmatic stream serialisation) become resident right
+    // away: its CTAs are small, sit next to this one and block in griddepcontrol.wait until this grid
+    // has completed and its writes are visible, so the merge starts without a launch gap.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     extern __shared__ __align__(128) uint8_t ring_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, c = lane & 3;
@@ -117,13 +130,33 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     const int workers = gridDim.x * kWarps;
     const int worker = warp * gridDim.x + blockIdx.x;
 
-    // ---- prefetch cursor: runs kStages - 1 blocks ahead of the compute, across item boundaries
-    int p_idx = worker, p_j0 = 0, p_s1 = 0;
+    // ---- dealing order of the batch entries: longest cached sequence first (ties by index)
+    __shared__ int order_smem[kMaxSortedBatch];
+    const int* order = nullptr;
+    if (B <= kMaxSortedBatch) {
+        if (tid < B) {
+            const int mine = min(max(lens[tid], 0), Smax);
+            int rank = 0;
+            for (int o = 0; o < B; ++o) {
+                const int other = min(max(lens[o], 0), Smax);
+                rank += (other > mine) || (other == mine && o < tid);
+            }
+            order_smem[rank] = tid;
+        }
+        __syncthreads();
+        order = order_smem;
+    }
+    // the item of this worker in round r: rounds alternate in direction
+    auto item_of_round = [&](int r) { return r * workers + ((r & 1) ? workers - 1 - worker : worker); };
+
+    // ---- prefetch cursor: runs kStages blocks ahead of the compute, across item boundaries (a stage is
+    // refilled as soon as its fragments are in registers, before the MMAs on them)
+    int p_round = 0, p_idx = item_of_round(0), p_j0 = 0, p_s1 = 0;
     const __nv_bfloat16 *p_k = kc, *p_v = vc;
     int p_n = 0;  // blocks issued
     auto p_open = [&]() {  // position the cursor on the first block of the next non-empty item
         while (p_idx < num_items) {
-            const Item it = make_item(p_idx, lens, Hkv, Smax, num_splits);
+            const Item it = make_item(p_idx, lens, order, Hkv, Smax, num_splits);
             if (it.s1 > it.s0) {
                 p_j0 = it.s0;
                 p_s1 = it.s1;
@@ -131,7 +164,7 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                 p_v = vc + ((size_t)it.b * Hkv + it.kvh) * (size_t)Smax * D;
                 return;
             }
-            p_idx += workers;
+            p_idx = item_of_round(++p_round);
         }
     };
     auto issue = [&]() {  // lane l of copy i moves chunk i*32 + l of the block's 16 rows
@@ -148,13 +181,13 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
             }
             ++p_n;
             p_j0 += kBlockKeys;
-            if (p_j0 >= p_s1) { p_idx += workers; p_open(); }
+            if (p_j0 >= p_s1) { p_idx = item_of_round(++p_round); p_open(); }
         }
         cp_async_commit();  // an empty group keeps the group count uniform
     };
     p_open();
 #pragma unroll
-    for (int i = 0; i < kStages - 1; ++i) issue();
+    for (int i = 0; i < kStages; ++i) issue();
 
     // Q fragment of an item: head g (zero rows for g >= G), 8 dims at c*8 of every 32-dim block
     auto load_q = [&](const Item& it, uint32_t (&qr)[NKB][4]) {
@@ -169,20 +202,20 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
 
     Item nxt = {0, 0, 0, 0, 0};
     uint32_t qn[NKB][4];
-    if (worker < num_items) {
-        nxt = make_item(worker, lens, Hkv, Smax, num_splits);
+    if (item_of_round(0) < num_items) {
+        nxt = make_item(item_of_round(0), lens, order, Hkv, Smax, num_splits);
         load_q(nxt, qn);
     }
     int n = 0;  // blocks consumed
-    for (int idx = worker; idx < num_items; idx += workers) {
+    for (int round = 0; item_of_round(round) < num_items; ++round) {
         const Item it = nxt;
         uint32_t qr[NKB][4];
 #pragma unroll
         for (int kb = 0; kb < NKB; ++kb)
 #pragma unroll
             for (int i = 0; i < 4; ++i) qr[kb][i] = qn[kb][i];
-        if (idx + workers < num_items) {  // fetch the next item's range and Q rows early
-            nxt = make_item(idx + workers, lens, Hkv, Smax, num_splits);
+        if (item_of_round(round + 1) < num_items) {  // fetch the next item's range and Q rows early
+            nxt = make_item(item_of_round(round + 1), lens, order, Hkv, Smax, num_splits);
             load_q(nxt, qn);
         }
 
@@ -196,7 +229,6 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                 for (int i = 0; i < 4; ++i) acc[hb][t][i] = 0.f;
 
         for (int j0 = it.s0; j0 < it.s1; j0 += kBlockKeys, ++n) {
-            issue();                       // refills the stage that was read in the previous iteration
             cp_async_wait<kStages - 1>();  // this lane's copies of block n have landed
             __syncwarp();                  // ... and everyone else's
             const uint32_t sa = ring + (n % kStages) * kStageBytes;
@@ -215,6 +247,7 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                     vr[r][hb] = lds128(sa + kTensorBytes + row * kRowBytes + swz(row, hb * 8 + g) * 16);
             }
             __syncwarp();  // all fragment reads done before this stage is refilled
+            issue();
 
             // scores: s[u][0..1] = head g, keys j0 + u*8 + 2c + {0, 1}  (s[u][2..3] belong to zero rows)
             float s[2][4];
@@ -319,36 +352,46 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
         }
     }
     cp_async_wait<0>();
-
-    // Let the combine kernel (launched with programmatic stream serialisation) be scheduled once every
-    // CTA of this grid got here; it still waits for this grid's completion before it reads.
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
-// grid = B * Hq, block = D threads: merges the num_splits partials of one (batch, head).
+// grid = B * Hq, block = D threads: merges the num_splits partials of one (batch, head).  The
+// partials are read in groups of 16 with all loads of a group in flight together.
 template <int D>
 __global__ void __launch_bounds__(D)
 decode_combine_kernel(const float* __restrict__ ws_o, const float* __restrict__ ws_ml,
                       __nv_bfloat16* __restrict__ out, int num_splits) {
     const size_t bh = blockIdx.x;
     const int d = threadIdx.x;
-    const float* ml = ws_ml + bh * num_splits * 2;
+    const float2* ml = reinterpret_cast<const float2*>(ws_ml) + bh * num_splits;
+    const float* po = ws_o + bh * num_splits * D + d;
     // the split kernel's writes are visible only after this returns
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    float M = -INFINITY;
-#pragma unroll 8
-    for (int s = 0; s < num_splits; ++s) M = fmaxf(M, ml[2 * s]);
-    float L = 0.f, O = 0.f;
-    if (M != -INFINITY) {
-#pragma unroll 8
-        for (int s = 0; s < num_splits; ++s) {
-            const float ms = ml[2 * s];
-            // empty split: m = -inf gives weight 0; its output slot was never written, so do not read it
-            const float wgt = exp2f(ms - M);
-            const float o = (ms == -INFINITY) ? 0.f : ws_o[(bh * num_splits + s) * D + d];
-            L = fmaf(wgt, ml[2 * s + 1], L);
-            O = fmaf(wgt, o, O);
+    float M = -INFINITY, L = 0.f, O = 0.f;  // running merge over the groups
+    for (int s0 = 0; s0 < num_splits; s0 += 16) {
+        float2 mls[16];
+        float os[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const bool ok = s0 + i < num_splits;
+            mls[i] = ok ? ml[s0 + i] : make_float2(-INFINITY, 0.f);
+            // the output slot of an empty split (m = -inf) was never written: whatever is read gets weight 0
+            // through the select below
+            os[i] = ok ? po[(size_t)(s0 + i) * D] : 0.f;
         }
+        float Mg = M;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) Mg = fmaxf(Mg, mls[i].x);
+        if (Mg == -INFINITY) continue;
+        const float keep = exp2f(M - Mg);  // 0 while nothing has been merged yet
+        L *= keep;
+        O *= keep;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const float wgt = exp2f(mls[i].x - Mg);
+            L = fmaf(wgt, mls[i].y, L);
+            O = fmaf(wgt, (mls[i].x == -INFINITY) ? 0.f : os[i], O);
+        }
+        M = Mg;
     }
     out[bh * D + d] = __float2bfloat16_rn(L > 0.f ? O / L : 0.f);
 }

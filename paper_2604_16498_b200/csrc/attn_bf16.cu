@@ -275,6 +275,10 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_base_slot;
     bool failed = false;
+    // set-up done: the next kernel may move in as SMs free up; nothing global is touched before the
+    // previous kernel has completed
+    pdl_launch_dependents();
+    pdl_wait();
 
     if (warp >= 8) {
       asm volatile("setmaxnreg.dec.sync.aligned.u32 88;");
@@ -708,7 +712,7 @@ int launch_attn(const void* q, const void* k, const void* v, void* out, int B, i
     const long long items = head_pairs ? (long long)((Hq + 1) / 2) * B * q_tiles
                                        : (long long)Hq * B * ((q_tiles + 1) / 2);
     const int grid = items < sms ? (int)items : sms;
-    kernel<<<grid, kThreads, L::kAlloc, s>>>(tq, tk, tv, to, p);
+    FORGE_CUDA_TRY(launch_pdl(kernel, dim3(grid), dim3(kThreads), L::kAlloc, s, tq, tk, tv, to, p));
     return finish_launch(1);
 }
 

@@ -120,7 +120,8 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     // Let the combine kernel (launched with programmatic stream serialisation) become resident right
     // away: its CTAs are small, sit next to this one and block in griddepcontrol.wait until this grid
     // has completed and its writes are visible, so the merge starts without a launch gap.
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    pdl_launch_dependents();
+    pdl_wait();  // the previous kernel in the stream has completed (this kernel may have been resident before)
     extern __shared__ __align__(128) uint8_t ring_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, c = lane & 3;
@@ -364,8 +365,9 @@ decode_combine_kernel(const float* __restrict__ ws_o, const float* __restrict__ 
     const int d = threadIdx.x;
     const float2* ml = reinterpret_cast<const float2*>(ws_ml) + bh * num_splits;
     const float* po = ws_o + bh * num_splits * D + d;
+    pdl_launch_dependents();  // the next kernel in the stream may move in while this one runs
     // the split kernel's writes are visible only after this returns
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    pdl_wait();
     float M = -INFINITY, L = 0.f, O = 0.f;  // running merge over the groups
     for (int s0 = 0; s0 < num_splits; s0 += 16) {
         float2 mls[16];
@@ -407,9 +409,9 @@ int launch_split(const void* q, const void* kc, const void* vc, const int32_t* l
     const long long items = (long long)B * Hkv * num_splits;
     const long long ctas = (items + kWarps - 1) / kWarps;
     const int grid = ctas < sms ? (int)ctas : sms;
-    kernel<<<grid, kThreads, kSmem, s>>>(
-        static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(kc),
-        static_cast<const __nv_bfloat16*>(vc), lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2);
+    FORGE_CUDA_TRY(launch_pdl(kernel, dim3(grid), dim3(kThreads), kSmem, s, static_cast<const __nv_bfloat16*>(q),
+                              static_cast<const __nv_bfloat16*>(kc), static_cast<const __nv_bfloat16*>(vc), lens, ws_o,
+                              ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2));
     return FORGE_OK;
 }
 
@@ -460,22 +462,13 @@ extern "C" int forge_attn_decode_splitkv(const void* q, const void* k_cache, con
     if (st != FORGE_OK) return st;
     // The combine kernel is launched with programmatic stream serialisation: its CTAs may be placed
     // while the split kernel drains, and block in griddepcontrol.wait until that grid has completed.
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(B * Hq, 1, 1);
-    cfg.blockDim = dim3(D, 1, 1);
-    cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
     const float* cws_o = ws_o;
     const float* cws_ml = ws_ml;
     __nv_bfloat16* ob = static_cast<__nv_bfloat16*>(out);
     if (D == 64)
-        FORGE_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_combine_kernel<64>, cws_o, cws_ml, ob, num_splits));
+        FORGE_CUDA_TRY(launch_pdl(decode_combine_kernel<64>, dim3(B * Hq), dim3(64), 0, s, cws_o, cws_ml, ob, num_splits));
     else
-        FORGE_CUDA_TRY(cudaLaunchKernelEx(&cfg, decode_combine_kernel<128>, cws_o, cws_ml, ob, num_splits));
+        FORGE_CUDA_TRY(launch_pdl(decode_combine_kernel<128>, dim3(B * Hq), dim3(128), 0, s, cws_o, cws_ml, ob, num_splits));
     return finish_launch(1);
 }
 

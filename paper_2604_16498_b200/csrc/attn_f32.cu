@@ -31,6 +31,8 @@ attn_f32_kernel(const float* __restrict__ q, const float* __restrict__ k, const 
     float* sV = sK + kBN * LD;
     float* sP = sV + kBN * LD;
 
+    pdl_launch_dependents();  // the next kernel may move in; nothing global is touched before the previous one is done
+    pdl_wait();
     const int tid = threadIdx.x;
     const int q0 = blockIdx.x * kBM;
     const int h = blockIdx.y;
@@ -175,7 +177,8 @@ extern "C" int forge_attn_fused_f32(const void* q, const void* k, const void* v,
     float* of = static_cast<float*>(out);
     const size_t smem = sizeof(float) * ((size_t)(kBM + 2 * kBN) * (D + kPad) + kBM * (kBN + kPad));
     if (D == 64) {
-        attn_f32_kernel<64><<<grid, kThreads, smem, s>>>(qf, kf, vf, of, Hq, Hkv, Sq, Skv, mask_kind, lens, scale_log2);
+        FORGE_CUDA_TRY(launch_pdl(attn_f32_kernel<64>, grid, dim3(kThreads), smem, s, qf, kf, vf, of, Hq, Hkv, Sq, Skv,
+                                  mask_kind, lens, scale_log2));
     } else {
         static bool attr_set = false;  // opt in to > 48 KB of dynamic shared memory once
         if (!attr_set) {
@@ -183,7 +186,8 @@ extern "C" int forge_attn_fused_f32(const void* q, const void* k, const void* v,
                                                 (int)smem));
             attr_set = true;
         }
-        attn_f32_kernel<128><<<grid, kThreads, smem, s>>>(qf, kf, vf, of, Hq, Hkv, Sq, Skv, mask_kind, lens, scale_log2);
+        FORGE_CUDA_TRY(launch_pdl(attn_f32_kernel<128>, grid, dim3(kThreads), smem, s, qf, kf, vf, of, Hq, Hkv, Sq, Skv,
+                                  mask_kind, lens, scale_log2));
     }
     return finish_launch(1);
 }

@@ -30,6 +30,34 @@ inline int finish_launch(int nkernels) {
 // Number of SMs of the current device (looked up once per device).
 int sm_count();
 
+// Launches `kernel` with programmatic stream serialisation: its CTAs may become resident while the
+// previous kernel in the stream is still running (once that kernel has let its dependents go, or has
+// finished), so launch latency and the kernel's own set-up overlap the predecessor's tail.  Every kernel
+// of this library calls pdl_wait() before its first access to global memory, which blocks until the
+// predecessor has completed and its writes are visible; a predecessor that never lets go behaves as
+// with an ordinary launch.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem_bytes, cudaStream_t s,
+                              Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+#ifdef __CUDACC__
+// Device side of launch_pdl(): let the next kernel in the stream become resident / wait for the previous one.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#endif
+
 // Opts a kernel in to `bytes` of dynamic shared memory once per device and call site (the attribute
 // call costs microseconds, which matters for the latency-bound shapes).
 #define FORGE_SET_SMEM_ONCE(kernel, bytes)                                                          \

@@ -104,6 +104,10 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_base_slot;
     bool failed = false;
+    // set-up done: the next kernel may move in as SMs free up; nothing global is touched before the
+    // previous kernel has completed
+    pdl_launch_dependents();
+    pdl_wait();
 
     if (warp == 0) {
         if (elect_one()) {
@@ -278,8 +282,9 @@ int launch_linear(const void* x, const void* w, const void* b, const void* resid
     FORGE_SET_SMEM_ONCE(kernel, L::kAlloc);
     const int tiles = ((M + kBM - 1) / kBM) * ((N + BN - 1) / BN);
     const int grid = tiles < sms ? tiles : sms;
-    kernel<<<grid, kThreads, L::kAlloc, s>>>(tmap_x, tmap_w, tmap_y, static_cast<const __nv_bfloat16*>(b),
-                                             static_cast<const __nv_bfloat16*>(residual), M, N, K, status);
+    FORGE_CUDA_TRY(launch_pdl(kernel, dim3(grid), dim3(kThreads), L::kAlloc, s, tmap_x, tmap_w, tmap_y,
+                              static_cast<const __nv_bfloat16*>(b), static_cast<const __nv_bfloat16*>(residual),
+                              M, N, K, status));
     return finish_launch(1);
 }
 

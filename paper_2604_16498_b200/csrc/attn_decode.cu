@@ -9,10 +9,10 @@
 // with a deep queue of requests (pure streaming with 48 KB in flight per SM reaches 4.2 TB/s on
 // this part, with 250 KB 5.8 TB/s).  So the split kernel is persistent and every warp is an
 // independent worker: it owns whole (batch, kv head, split) items, keeps a private ring of
-// 16-row blocks in shared memory filled by 16-byte asynchronous copies that run ahead across
-// item boundaries (8 warps x 24 KB in flight per SM, 512 contiguous bytes per instruction,
-// zero-fill instead of reads past the end of a split), and writes its partial straight from
-// registers.  No warp ever waits for another one.  Items differ in length by up to the ratio of the
+// 16-row blocks in shared memory filled by TMA tile copies (16 rows x 64 columns each, 128-byte
+// swizzle, completion counted on an mbarrier per stage) that run ahead across item boundaries
+// (8 warps x 24 KB in flight per SM), and writes its partial straight from registers.  Split
+// boundaries are multiples of 16 rows, so a block never straddles two splits.  No warp ever waits for another one.  Items differ in length by up to the ratio of the
 // longest to the shortest cached sequence, so they are dealt out longest sequence first and in
 // alternating direction from round to round (a worker that got one of the longest items in one round
 // gets one of the shortest in the next), which keeps the workers' totals close together.
@@ -25,6 +25,8 @@
 #include <mutex>
 
 #include "forge_common.cuh"
+#include "sm100_ptx.cuh"
+#include "tmap.cuh"
 
 namespace forge {
 namespace {
@@ -35,27 +37,11 @@ constexpr int kBlockKeys = 16;             // cached rows per ring stage
 constexpr int kWarpRingBytes = 24 * 1024;  // per warp
 constexpr int kMaxSortedBatch = 64;        // batches up to this size are ordered by cached length
 
-// 16-byte asynchronous copy global -> shared; src_bytes = 0 writes zeros and reads nothing.
-__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gsrc, uint32_t src_bytes) {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_dst), "l"(gsrc), "r"(src_bytes)
-                 : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() {
-    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 r;
     asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "r"(addr));
     return r;
 }
-// Position of 16-byte chunk k of cached row r inside the row's shared-memory image.  Bits 1-2 of the
-// chunk index are XORed with a function of the row so that both fragment reads are free of bank
-// conflicts: per quarter-warp, K reads touch rows (r, r+1) x 4 consecutive chunks and V reads touch
-// rows (r, r+2, r+4, r+6) x 2 consecutive chunks.
-__device__ __forceinline__ int swz(int r, int k) { return k ^ ((((r >> 1) & 3) << 1) ^ ((r & 1) << 2)); }
-
 // D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col).  Lane = (g = lane / 4, c = lane % 4):
 //   A: a0 = (row g, k 2c..2c+1)  a1 = (row g+8, k 2c..)  a2 = (row g, k 2c+8..)  a3 = (row g+8, k 2c+8..)
 //   B: b0 = (k 2c..2c+1, col g)  b1 = (k 2c+8.., col g)
@@ -88,7 +74,8 @@ __device__ __forceinline__ Item make_item(int idx, const int32_t* lens, const in
     it.b = bk / Hkv;
     if (order) it.b = order[it.b];
     const int len = min(max(lens[it.b], 0), Smax);
-    const int per = (len + num_splits - 1) / num_splits;
+    // rows per split: the even share, rounded up to whole 16-row blocks
+    const int per = (((len + num_splits - 1) / num_splits) + kBlockKeys - 1) / kBlockKeys * kBlockKeys;
     it.s0 = it.split * per;
     it.s1 = min(it.s0 + per, len);
     if (it.s1 < it.s0) it.s1 = it.s0;
@@ -104,18 +91,19 @@ __device__ __forceinline__ Item make_item(int idx, const int32_t* lens, const in
 //                   probabilities exactly where the first MMA left them.
 template <int D, int G>
 __global__ void __launch_bounds__(kThreads, 1)
-decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ kc,
-                    const __nv_bfloat16* __restrict__ vc, const int32_t* __restrict__ lens,
+decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
+                    const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ lens,
                     float* __restrict__ ws_o, float* __restrict__ ws_ml,
-                    int B, int Hq, int Hkv, int Smax, int num_splits, float scale_log2) {
+                    int B, int Hq, int Hkv, int Smax, int num_splits, float scale_log2, int* status) {
     constexpr int NKB = D / 32;  // 32-dim blocks of the head dimension (two k16 MMAs each)
     constexpr int NHB = D / 64;  // 64-dim blocks of the output (four 16-dim MMAs each)
-    constexpr int kRowBytes = D * 2;
-    constexpr int kCPR = kRowBytes / 16;                  // 16-byte chunks per row
-    constexpr int kTensorBytes = kBlockKeys * kRowBytes;  // 16 rows of K (or of V)
-    constexpr int kStageBytes = 2 * kTensorBytes;
+    // A stage holds 16 rows of K and 16 rows of V as D / 64 tiles of 16 rows x 128 bytes each; 16-byte chunk
+    // k of row r of a tile sits at r * 128 + ((k ^ (r & 7)) << 4) (the TMA unit's 128-byte swizzle).
+    constexpr int kTileBytes = kBlockKeys * 128;
+    constexpr int kKBytes = (D / 64) * kTileBytes;
+    constexpr int kStageBytes = 2 * kKBytes;
     constexpr int kStages = kWarpRingBytes / kStageBytes;  // 3 for D = 128, 6 for D = 64
-    static_assert(kStages >= 2, "ring too small");
+    static_assert(kStages >= 2 && kStages <= 8, "ring size");
 
     // Let the combine kernel (launched with programmatic stream serialisation) become resident right
     // away: its CTAs are small, sit next to this one and block in griddepcontrol.wait until this grid
@@ -123,9 +111,20 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     pdl_launch_dependents();
     pdl_wait();  // the previous kernel in the stream has completed (this kernel may have been resident before)
     extern __shared__ __align__(128) uint8_t ring_raw[];
+    __shared__ uint64_t full_bars[kWarps][8];  // [warp][stage]: the stage's rows have landed
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, c = lane & 3;
-    const uint32_t ring = static_cast<uint32_t>(__cvta_generic_to_shared(ring_raw)) + warp * kWarpRingBytes;
+    // swizzled tiles need 1024-byte alignment
+    const uint32_t ring = ((static_cast<uint32_t>(__cvta_generic_to_shared(ring_raw)) + 1023u) & ~1023u) +
+                          warp * kWarpRingBytes;
+    uint64_t* full = full_bars[warp];
+    if (lane == 0) {
+        for (int i = 0; i < kStages; ++i) ptx::mbar_init(&full[i], 1);
+        ptx::fence_mbar_init();
+        ptx::prefetch_tmap(&tmap_k);
+        ptx::prefetch_tmap(&tmap_v);
+    }
+    __syncwarp();
 
     const int num_items = B * Hkv * num_splits;
     const int workers = gridDim.x * kWarps;
@@ -153,7 +152,7 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
     // ---- prefetch cursor: runs kStages blocks ahead of the compute, across item boundaries (a stage is
     // refilled as soon as its fragments are in registers, before the MMAs on them)
     int p_round = 0, p_idx = item_of_round(0), p_j0 = 0, p_s1 = 0;
-    const __nv_bfloat16 *p_k = kc, *p_v = vc;
+    int p_bk = 0;  // batch * Hkv + kv head of the cursor's item
     int p_n = 0;  // blocks issued
     auto p_open = [&]() {  // position the cursor on the first block of the next non-empty item
         while (p_idx < num_items) {
@@ -161,30 +160,28 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
             if (it.s1 > it.s0) {
                 p_j0 = it.s0;
                 p_s1 = it.s1;
-                p_k = kc + ((size_t)it.b * Hkv + it.kvh) * (size_t)Smax * D;
-                p_v = vc + ((size_t)it.b * Hkv + it.kvh) * (size_t)Smax * D;
+                p_bk = it.b * Hkv + it.kvh;
                 return;
             }
             p_idx = item_of_round(++p_round);
         }
     };
-    auto issue = [&]() {  // lane l of copy i moves chunk i*32 + l of the block's 16 rows
+    auto issue = [&]() {  // one lane starts the block's tile copies (rows past the cache's end are zero-filled)
         if (p_idx < num_items) {
-            const uint32_t dst = ring + (p_n % kStages) * kStageBytes;
+            if (lane == 0) {
+                const int st = p_n % kStages;
+                const uint32_t dst = ring + st * kStageBytes;
+                ptx::mbar_expect_tx(&full[st], kStageBytes);
 #pragma unroll
-            for (int i = 0; i < kTensorBytes / 512; ++i) {
-                const int id = i * 32 + lane, r = id / kCPR, k = id % kCPR;
-                const uint32_t ok = (p_j0 + r < p_s1) ? 16u : 0u;  // rows past the split: zeros, nothing read
-                const size_t goff = (size_t)(p_j0 + (ok ? r : 0)) * D + k * 8;
-                const uint32_t soff = r * kRowBytes + swz(r, k) * 16;
-                cp_async16(dst + soff, p_k + goff, ok);
-                cp_async16(dst + kTensorBytes + soff, p_v + goff, ok);
+                for (int cb = 0; cb < D / 64; ++cb) {
+                    ptx::tma_load_3d_addr(dst + cb * kTileBytes, &tmap_k, &full[st], cb * 64, p_j0, p_bk);
+                    ptx::tma_load_3d_addr(dst + kKBytes + cb * kTileBytes, &tmap_v, &full[st], cb * 64, p_j0, p_bk);
+                }
             }
             ++p_n;
             p_j0 += kBlockKeys;
             if (p_j0 >= p_s1) { p_idx = item_of_round(++p_round); p_open(); }
         }
-        cp_async_commit();  // an empty group keeps the group count uniform
     };
     p_open();
 #pragma unroll
@@ -208,6 +205,7 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
         load_q(nxt, qn);
     }
     int n = 0;  // blocks consumed
+    bool failed = false;
     for (int round = 0; item_of_round(round) < num_items; ++round) {
         const Item it = nxt;
         uint32_t qr[NKB][4];
@@ -230,8 +228,8 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                 for (int i = 0; i < 4; ++i) acc[hb][t][i] = 0.f;
 
         for (int j0 = it.s0; j0 < it.s1; j0 += kBlockKeys, ++n) {
-            cp_async_wait<kStages - 1>();  // this lane's copies of block n have landed
-            __syncwarp();                  // ... and everyone else's
+            // the rows of block n have landed (bounded wait: on expiry the kernel flags the error and leaves)
+            if (!ptx::warp_wait(&full[n % kStages], (n / kStages) & 1)) { failed = true; break; }
             const uint32_t sa = ring + (n % kStages) * kStageBytes;
             // K fragment: rows u*8 + g, chunk kb*4 + c.  V fragment: rows {2c, 2c+1, 2c+8, 2c+9}, chunk hb*8 + g.
             uint4 kr[2][NKB], vr[4][NHB];
@@ -239,15 +237,22 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
             for (int u = 0; u < 2; ++u)
 #pragma unroll
                 for (int kb = 0; kb < NKB; ++kb)
-                    kr[u][kb] = lds128(sa + (u * 8 + g) * kRowBytes + swz(u * 8 + g, kb * 4 + c) * 16);
+                    kr[u][kb] = lds128(sa + (kb / 2) * kTileBytes + (u * 8 + g) * 128 + ((((kb & 1) * 4 + c) ^ g) << 4));
 #pragma unroll
             for (int r = 0; r < 4; ++r) {
                 const int row = 2 * c + (r & 1) + (r >> 1) * 8;
 #pragma unroll
                 for (int hb = 0; hb < NHB; ++hb)
-                    vr[r][hb] = lds128(sa + kTensorBytes + row * kRowBytes + swz(row, hb * 8 + g) * 16);
+                    vr[r][hb] = lds128(sa + kKBytes + hb * kTileBytes + row * 128 + ((g ^ (row & 7)) << 4));
+                // a row past the sequence's end holds whatever the cache holds there: it must not reach the MMA
+                // (its probability is 0, but 0 x NaN is NaN)
+                if (j0 + row >= it.s1) {
+#pragma unroll
+                    for (int hb = 0; hb < NHB; ++hb) vr[r][hb] = make_uint4(0, 0, 0, 0);
+                }
             }
-            __syncwarp();  // all fragment reads done before this stage is refilled
+            __syncwarp();  // all fragment reads done before this stage is refilled ...
+            ptx::fence_proxy_async_smem();  // ... by the copy engine (reads before its writes)
             issue();
 
             // scores: s[u][0..1] = head g, keys j0 + u*8 + 2c + {0, 1}  (s[u][2..3] belong to zero rows)
@@ -325,6 +330,7 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
             }
         }
 
+        if (failed) break;
         // ---- this warp's partial is the item's partial: write it out from the fragments
         l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
         l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
@@ -352,7 +358,10 @@ decode_split_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __
                 }
         }
     }
-    cp_async_wait<0>();
+    if (failed) {
+        if (lane == 0) atomicExch(status, 1);
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);  // let copies in flight land before the ring goes away
+    }
 }
 
 // grid = B * Hq, block = D threads: merges the num_splits partials of one (batch, head).  The
@@ -401,7 +410,17 @@ decode_combine_kernel(const float* __restrict__ ws_o, const float* __restrict__ 
 template <int D, int G>
 int launch_split(const void* q, const void* kc, const void* vc, const int32_t* lens, float* ws_o, float* ws_ml,
                  int B, int Hq, int Hkv, int Smax, int num_splits, float scale_log2, cudaStream_t s) {
-    constexpr int kSmem = kWarps * kWarpRingBytes;
+    constexpr int kSmem = kWarps * kWarpRingBytes + 1024;
+    int* status = device_status_word();
+    if (!status) return FORGE_ERR_CUDA;
+    CUtensorMap tk, tv;
+    {
+        const uint32_t box[3] = {64, (uint32_t)kBlockKeys, 1};
+        const uint64_t dims[3] = {(uint64_t)D, (uint64_t)Smax, (uint64_t)B * Hkv};
+        const uint64_t strides[2] = {(uint64_t)D * 2, (uint64_t)Smax * D * 2};
+        if (!encode_tmap_bf16_sw128(&tk, kc, 3, dims, strides, box)) return FORGE_ERR_CUDA;
+        if (!encode_tmap_bf16_sw128(&tv, vc, 3, dims, strides, box)) return FORGE_ERR_CUDA;
+    }
     auto kernel = decode_split_kernel<D, G>;
     FORGE_SET_SMEM_ONCE(kernel, kSmem);
     const int sms = sm_count();
@@ -409,9 +428,8 @@ int launch_split(const void* q, const void* kc, const void* vc, const int32_t* l
     const long long items = (long long)B * Hkv * num_splits;
     const long long ctas = (items + kWarps - 1) / kWarps;
     const int grid = ctas < sms ? (int)ctas : sms;
-    FORGE_CUDA_TRY(launch_pdl(kernel, dim3(grid), dim3(kThreads), kSmem, s, static_cast<const __nv_bfloat16*>(q),
-                              static_cast<const __nv_bfloat16*>(kc), static_cast<const __nv_bfloat16*>(vc), lens, ws_o,
-                              ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2));
+    FORGE_CUDA_TRY(launch_pdl(kernel, dim3(grid), dim3(kThreads), kSmem, s, tk, tv, static_cast<const __nv_bfloat16*>(q),
+                              lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, status));
     return FORGE_OK;
 }
 

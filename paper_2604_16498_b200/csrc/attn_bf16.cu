@@ -357,10 +357,20 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 }
                 const int nh = pick(it.nh, t);
 
-                // S(g) = Q K(g)^T into half g % 2 of S_t
+                // A barrier poll costs a few hundred cycles even on a completed phase, so the operands of a step
+                // (V(g) for the product, K(g + 2) for the next scores) are waited for before the probabilities,
+                // while this thread has nothing to issue; once P(g) arrives the MMAs go out back to back.
+                auto wait_k = [&](int g) -> bool {
+                    const int pos = kvbase + g;
+                    return mbar_wait(&k_full[kv_slot(u, pos)], kv_phase(pos));
+                };
+                auto wait_v = [&](int g) -> bool {
+                    const int pos = kvbase + g;
+                    return mbar_wait(&v_full[kv_slot(u, pos)], kv_phase(pos));
+                };
+                // S(g) = Q K(g)^T into half g % 2 of S_t (K(g) has landed)
                 auto issue_qk = [&](int g) -> bool {
                     const int hh = g & 1, pos = kvbase + g, st = kv_slot(u, pos);
-                    if (!mbar_wait(&k_full[st], kv_phase(pos))) return false;
                     tc_fence_after_sync();
                     const uint64_t kd = make_smem_desc(k_addr + st * L::kKVTileBytes, 16, 1024);
 #pragma unroll
@@ -374,12 +384,11 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     if (g == nh - 1) mma_commit(&q_empty[t]);  // and, after the item's last S, with Q
                     return true;
                 };
-                // O_t += P(g) V(g) with P read from tensor memory
+                // O_t += P(g) V(g) with P read from tensor memory (V(g) has landed)
                 auto issue_pv = [&](int g) -> bool {
                     const int hh = g & 1, pos = kvbase + g, st = kv_slot(u, pos);
                     if (!mbar_wait(&p_ready[t * 2 + hh], (hh ? steps1 : steps0) & 1)) return false;
                     if (hh) ++steps1; else ++steps0;
-                    if (!mbar_wait(&v_full[st], kv_phase(pos))) return false;
                     // the first product of an item overwrites O_t: the previous item's epilogue must have read it
                     if (g == 0 && !mbar_wait(&o_free[t], (q_uses & 1) ^ 1)) return false;
                     tc_fence_after_sync();
@@ -398,13 +407,14 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
 
                 if (nh > 0) {
                     if (!mbar_wait(&q_full[t], q_uses & 1)) { failed = true; break; }
-                    if (!issue_qk(0)) { failed = true; break; }
-                    if (nh > 1 && !issue_qk(1)) { failed = true; break; }
+                    if (!wait_k(0) || !issue_qk(0)) { failed = true; break; }
+                    if (nh > 1 && (!wait_k(1) || !issue_qk(1))) { failed = true; break; }
                 }
                 // the next item's coordinates, worked out while the softmax warps are busy with the first S
                 if (i_next < num_items) it_next = decode(i_next);
                 if (nh > 0) {
                     for (int g = 0; g < nh; ++g) {
+                        if (!wait_v(g) || (g + 2 < nh && !wait_k(g + 2))) { failed = true; break; }
                         if (!issue_pv(g)) { failed = true; break; }
                         if (g + 2 < nh && !issue_qk(g + 2)) { failed = true; break; }
                     }

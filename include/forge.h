@@ -69,6 +69,18 @@ int forge_attn_fused(const void* q, const void* k, const void* v, void* out,
                      int mask_kind, const int32_t* lens, float scale, void* stream);
 
 /*
+ * Same operator, same kernel, with fp16 tensors in and out (fp32 accumulate; the
+ * probabilities are rounded to fp16 before the product with V).  fp16 is the
+ * inference precision of the paper's evaluation (Section 5.1, model table).
+ * Same arguments, limits and errors as forge_attn_fused.  |scale * q.k| beyond
+ * what fp32 holds is the caller's concern; outputs are convex combinations of V
+ * rows and cannot overflow fp16 unless V does.
+ */
+int forge_attn_fused_f16(const void* q, const void* k, const void* v, void* out,
+                         int B, int Hq, int Hkv, int Sq, int Skv, int D,
+                         int mask_kind, const int32_t* lens, float scale, void* stream);
+
+/*
  * Same operator with fp32 tensors in and out (fp32 FMA arithmetic, no reduced
  * precision inside).  D must be 64 or 128.
  */
@@ -82,7 +94,7 @@ int forge_attn_fused_f32(const void* q, const void* k, const void* v, void* out,
  *     q, out : [B, Hq, D] bf16       k_cache, v_cache : [B, Hkv, Smax, D] bf16
  * Sequence b attends rows 0 .. lens[b]-1 of its cache (lens[b] clamped to
  * [0, Smax]; 0 gives zeros).  Split s of sequence b covers rows
- * [s*c, min((s+1)*c, lens[b])) with c = ceil(lens[b] / num_splits); each split
+ * [s*c, min((s+1)*c, lens[b])) with c = ceil(lens[b] / num_splits) rounded up to a multiple of 16; each split
  * produces a partial (running max, running sum, unnormalised output) in
  * `workspace` (fp32), and a combine step merges them.  Empty splits are skipped.
  * The result does not depend on num_splits beyond rounding.

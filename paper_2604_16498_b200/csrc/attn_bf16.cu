@@ -1,5 +1,6 @@
-// Fused attention, bf16 in / fp32 accumulate / bf16 out (Eq. 8 / Eq. 9): scores, mask, online
-// softmax and the product with V in one kernel; S and P never reach global memory.
+// Fused attention, 16-bit in / fp32 accumulate / 16-bit out (Eq. 8 / Eq. 9): scores, mask, online
+// softmax and the product with V in one kernel; S and P never reach global memory.  The element type
+// is bf16 or fp16 (a template parameter: the MMA operand format and the two conversions differ).
 //
 // One work item = two 128-row query tiles (see the item decoding below).  Every 128-key tile of S is
 // computed, normalised and multiplied with V in two 64-key halves with their own barriers, so each
@@ -23,6 +24,7 @@
 // kept otherwise; the final division by l uses the same reference, so the result is unchanged).
 // Q and K are K-major operands, V [keys, D] is the MN-major B operand of P V.
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include <type_traits>
 
@@ -121,9 +123,16 @@ __device__ __forceinline__ float2 ex2_fma2(float2 x) {
                        __int_as_float(__float_as_int(q.y) + (__float_as_int(t.y) << 23)));
 }
 
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t*>(&v);
+// two fp32 values rounded to nearest even and packed as bf16 (F16 = false) or fp16 (F16 = true)
+template <bool F16>
+__device__ __forceinline__ uint32_t pack16(float lo, float hi) {
+    if constexpr (F16) {
+        __half2 v = __floats2half2_rn(lo, hi);
+        return *reinterpret_cast<uint32_t*>(&v);
+    } else {
+        __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+        return *reinterpret_cast<uint32_t*>(&v);
+    }
 }
 
 // Division by a divisor fixed at launch: floor(n / d) = high 64 bits of n * ceil(2^64 / d) for 0 <= n < 2^32.
@@ -142,7 +151,7 @@ __device__ __forceinline__ int fast_div(int n, const FastDiv& f) {
 }
 
 struct AttnParams {
-    __nv_bfloat16* out;
+    uint16_t* out;  // bf16 or fp16 elements
     const int32_t* lens;
     int B, Hq, Hkv, Sq, Skv;
     int mask_kind;
@@ -166,7 +175,7 @@ struct ItemInfo {
 // element t of a two-element array without dynamic indexing (keeps the array in registers)
 __device__ __forceinline__ int pick(const int (&a)[kTilesPerCta], int t) { return t ? a[1] : a[0]; }
 
-template <int D>
+template <int D, bool F16>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                  const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_o,
@@ -333,8 +342,8 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
         if (elect_one()) {
             const int t = warp - 9;
             const int u = two_streams ? t : 0;
-            constexpr uint32_t idesc_s = make_idesc_bf16(kBM, kHalf, false, false);
-            constexpr uint32_t idesc_o = make_idesc_bf16(kBM, D, false, true);
+            constexpr uint32_t idesc_s = F16 ? make_idesc_f16(kBM, kHalf, false, false) : make_idesc_bf16(kBM, kHalf, false, false);
+            constexpr uint32_t idesc_o = F16 ? make_idesc_f16(kBM, D, false, true) : make_idesc_bf16(kBM, D, false, true);
             const uint32_t q_addr = smem_u32(sQ) + t * L::kTileBytes, k_addr = smem_u32(sK), v_addr = smem_u32(sV);
             const uint32_t s_tmem = tmem_base + kColS + t * kBN, o_tmem = tmem_base + kColO + t * D;
             // descriptors differ only in the start-address field: build one per operand, then add
@@ -463,7 +472,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             const int bh = it.b * p.Hq + pick(it.h, t);
             if (nh == 0) {  // no visible key for any row of this tile (or the tile lies beyond Sq)
                 if (qi < p.Sq) {
-                    __nv_bfloat16* orow = p.out + ((size_t)bh * p.Sq + qi) * D;
+                    uint16_t* orow = p.out + ((size_t)bh * p.Sq + qi) * D;
 #pragma unroll
                     for (int c = 0; c < D / 8; ++c) reinterpret_cast<uint4*>(orow)[c] = make_uint4(0, 0, 0, 0);
                 }
@@ -532,7 +541,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                             const bool on_fma = kUseFma && ((k + 1) * kFmaExpPairs / 32) != (k * kFmaExpPairs / 32);
                             const float2 pr = on_fma ? ex2_fma2(x) : make_float2(ex2(x.x), ex2(x.y));
                             lsum[k & 1] = fadd2(lsum[k & 1], pr);
-                            packed[k] = pack_bf16(pr.x, pr.y);
+                            packed[k] = pack16<F16>(pr.x, pr.y);
                         }
                         const float m_tile = max3(fmaxf(mx[0], mx[1]), mx[2], mx[3]);
                         if (!__any_sync(0xffffffffu, (m_tile - m_run) * sl2 > kRescaleThreshold)) {
@@ -595,7 +604,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                         const float2 x = ffma2(make_float2(s[2 * k], s[2 * k + 1]), sl2v, neg_m);
                         const float2 pr = make_float2(ex2(x.x), ex2(x.y));
                         lsum[k & 1] = fadd2(lsum[k & 1], pr);
-                        packed[k] = pack_bf16(pr.x, pr.y);
+                        packed[k] = pack16<F16>(pr.x, pr.y);
                     }
                     tmem_st_x32(lane_base + col_h, packed);
                     const float l_tile = (lsum[0].x + lsum[0].y) + (lsum[1].x + lsum[1].y);
@@ -629,7 +638,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     uint32_t w[16];
 #pragma unroll
                     for (int k = 0; k < 16; ++k)
-                        w[k] = pack_bf16(__uint_as_float(cur[2 * k]) * inv, __uint_as_float(cur[2 * k + 1]) * inv);
+                        w[k] = pack16<F16>(__uint_as_float(cur[2 * k]) * inv, __uint_as_float(cur[2 * k + 1]) * inv);
                     if (c32 + 1 < D / 32) tmem_ld_x32(lane_base + col_o + (c32 + 1) * 32, cur);
                     // 32 columns = four 16-byte chunks of this row's 128-byte line in block c32 / 2
                     uint8_t* line = stage_out + (c32 >> 1) * 4096 + lane * 128;
@@ -669,7 +678,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     }
 }
 
-template <int D>
+template <int D, bool F16>
 int launch_attn(const void* q, const void* k, const void* v, void* out, int B, int Hq, int Hkv, int Sq, int Skv,
                 int mask_kind, const int32_t* lens, float scale, cudaStream_t s) {
     using L = AttnSmem<D>;
@@ -696,7 +705,7 @@ int launch_attn(const void* q, const void* k, const void* v, void* out, int B, i
         if (!encode_tmap_bf16_sw128(&to, out, 3, dims, strides, box_o)) return FORGE_ERR_CUDA;
     }
     AttnParams p;
-    p.out = static_cast<__nv_bfloat16*>(out);
+    p.out = static_cast<uint16_t*>(out);
     p.lens = lens;
     p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.Sq = Sq; p.Skv = Skv;
     p.mask_kind = mask_kind;
@@ -713,7 +722,7 @@ int launch_attn(const void* q, const void* k, const void* v, void* out, int B, i
         p.div_inner = make_fastdiv(inner);
         p.div_group = make_fastdiv(G);
     }
-    auto kernel = attn_bf16_kernel<D>;
+    auto kernel = attn_bf16_kernel<D, F16>;
     FORGE_SET_SMEM_ONCE(kernel, L::kAlloc);
     const int sms = sm_count();
     if (sms <= 0) return FORGE_ERR_CUDA;
@@ -738,6 +747,19 @@ extern "C" int forge_attn_fused(const void* q, const void* k, const void* v, voi
     if ((long long)Hq * B * ((Sq + 255) / 256) > 2147483647LL) return FORGE_ERR_UNSUPPORTED;
     if (!(scale >= 0.f)) return FORGE_ERR_UNSUPPORTED;  // the running maximum is taken on unscaled scores
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    return D == 64 ? launch_attn<64>(q, k, v, out, B, Hq, Hkv, Sq, Skv, mask_kind, lens, scale, s)
-                   : launch_attn<128>(q, k, v, out, B, Hq, Hkv, Sq, Skv, mask_kind, lens, scale, s);
+    return D == 64 ? launch_attn<64, false>(q, k, v, out, B, Hq, Hkv, Sq, Skv, mask_kind, lens, scale, s)
+                   : launch_attn<128, false>(q, k, v, out, B, Hq, Hkv, Sq, Skv, mask_kind, lens, scale, s);
+}
+
+extern "C" int forge_attn_fused_f16(const void* q, const void* k, const void* v, void* out,
+                                    int B, int Hq, int Hkv, int Sq, int Skv, int D,
+                                    int mask_kind, const int32_t* lens, float scale, void* stream) {
+    using namespace forge;
+    int st = check_attn_args(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens);
+    if (st != FORGE_OK) return st;
+    if ((long long)Hq * B * ((Sq + 255) / 256) > 2147483647LL) return FORGE_ERR_UNSUPPORTED;
+    if (!(scale >= 0.f)) return FORGE_ERR_UNSUPPORTED;  // the running maximum is taken on unscaled scores
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    return D == 64 ? launch_attn<64, true>(q, k, v, out, B, Hq, Hkv, Sq, Skv, mask_kind, lens, scale, s)
+                   : launch_attn<128, true>(q, k, v, out, B, Hq, Hkv, Sq, Skv, mask_kind, lens, scale, s);
 }

@@ -9,9 +9,9 @@ is ``mix(seed + (i + 1) * 0x9E3779B97F4A7C15)``), turned into standard normals
 by the Box-Muller transform.  Everything is numpy; values are bit-reproducible
 on any host.
 
-bf16 tensors are produced as fp64 -> fp32 -> bf16 (round to nearest even) and
-returned both as raw 16-bit patterns (what the GPU consumes) and as the exact
-fp64 widening of those patterns (what the oracle consumes).
+bf16 (and fp16) tensors are produced as fp64 -> fp32 -> 16 bits (round to nearest
+even) and returned both as raw 16-bit patterns (what the GPU consumes) and as the
+exact fp64 widening of those patterns (what the oracle consumes).
 """
 from __future__ import annotations
 
@@ -93,7 +93,7 @@ class Tensor:
     patterns, or float32 for the fp32 workload)."""
     values: np.ndarray
     device_bits: np.ndarray
-    dtype: str  # "bf16" | "f32"
+    dtype: str  # "bf16" | "f16" | "f32"
 
 
 def normal_tensor(seed: int, shape, dtype: str, std: float = 1.0) -> Tensor:
@@ -104,6 +104,9 @@ def normal_tensor(seed: int, shape, dtype: str, std: float = 1.0) -> Tensor:
     if dtype == "bf16":
         bits = f32_to_bf16_bits(x32)
         return Tensor(bf16_bits_to_f64(bits).reshape(shape), bits.reshape(shape), "bf16")
+    if dtype == "f16":  # numpy rounds fp32 -> fp16 to nearest even
+        h = x32.astype(np.float16)
+        return Tensor(h.astype(np.float64).reshape(shape), h.view(np.uint16).reshape(shape), "f16")
     raise ValueError(dtype)
 
 

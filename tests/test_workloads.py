@@ -50,3 +50,13 @@ def test_config_shapes_and_counts():
     assert lw.flops() * (8192 // 64) == 38_654_705_664
     c2 = wl.cfg2_attention(B=1)
     assert c2.flops() * 8 == 12_897_484_800 and c2.bytes() * 8 == 50_331_648
+
+
+def test_f16_rounding_matches_torch_rne():
+    """The fp16 tensors hold exactly what torch's fp32 -> fp16 conversion (round to nearest even) gives, and
+    the oracle's values are the exact widening of the patterns the GPU reads."""
+    t = wl.normal_tensor(77, (4096,), "f16")
+    x32 = wl.normal_f64(77, 4096).astype(np.float32)
+    ref = torch.from_numpy(x32).to(torch.float16)
+    assert np.array_equal(t.device_bits, ref.view(torch.int16).numpy().view(np.uint16))
+    assert np.array_equal(t.values, ref.double().numpy())

@@ -13,6 +13,8 @@ def to_device(t):
     """workloads.Tensor -> CUDA tensor holding exactly the same values."""
     if t.dtype == "f32":
         return torch.from_numpy(np.ascontiguousarray(t.device_bits)).cuda()
+    if t.dtype == "f16":
+        return torch.from_numpy(np.ascontiguousarray(t.device_bits).view(np.float16)).cuda()
     return torch.from_numpy(np.ascontiguousarray(t.device_bits).view(np.int16)).view(torch.bfloat16).cuda()
 
 

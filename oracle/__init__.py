@@ -6,6 +6,7 @@ benchmark's CPU-baseline leg.  The CUDA product path never imports this package.
 from .ref import (  # noqa: F401
     attn,
     attn_probs,
+    attn_bias,
     attn_decode,
     linear_bias_gelu,
     linear_act,

@@ -35,6 +35,11 @@
  * j <= i + (Skv - Sq).  lens[b] is clamped to [0, Skv].  A row with no allowed
  * key produces zeros (and an all-zero probability row).
  *
+ * Additive bias (the optional mask node of Eq. 8 as a tensor): bias [B, Hb, Sq, Skv]
+ * with Hb = 1 (shared by all heads) or Hb = Hq is added to the scaled scores before
+ * the softmax: s = scale * q.k + bias.  A bias of -infinity excludes the key, like
+ * the mask kinds do; the mask kinds still apply on top.
+ *
  * Every function returns 0 on success, 1 on an invalid argument.
  */
 #include <math.h>
@@ -77,30 +82,38 @@ static int check_attn_args(const void *q, const void *k, const void *v, const vo
  * doubles and receives the probabilities (exact 0.0 where masked).
  */
 static void attn_row(const double *qrow, const double *kmat, const double *vmat, double *orow,
-                     double *p, int i, int Sq, int Skv, int D, int mask_kind, int kvlen, double scale)
+                     double *p, int i, int Sq, int Skv, int D, int mask_kind, int kvlen, double scale,
+                     const double *bias_row)
 {
     double m = -INFINITY;
     int any = 0;
     for (int j = 0; j < Skv; ++j) {
-        if (!allowed(mask_kind, i, j, Sq, Skv, kvlen)) { p[j] = 0.0; continue; }
+        if (!allowed(mask_kind, i, j, Sq, Skv, kvlen) || (bias_row && bias_row[j] == -INFINITY)) {
+            p[j] = -INFINITY;  /* marks an excluded key until the probabilities are written */
+            continue;
+        }
         double s = 0.0;
         for (int d = 0; d < D; ++d) s += qrow[d] * kmat[(size_t)j * D + d];
         s *= scale;
+        if (bias_row) s += bias_row[j];
         p[j] = s;
         if (!any || s > m) m = s;
         any = 1;
     }
     for (int d = 0; d < D; ++d) orow[d] = 0.0;
-    if (!any) return;
+    if (!any) {
+        for (int j = 0; j < Skv; ++j) p[j] = 0.0;
+        return;
+    }
 
     double denom = 0.0;
     for (int j = 0; j < Skv; ++j) {
-        if (!allowed(mask_kind, i, j, Sq, Skv, kvlen)) continue;
+        if (p[j] == -INFINITY) continue;
         p[j] = exp(p[j] - m);
         denom += p[j];
     }
     for (int j = 0; j < Skv; ++j) {
-        if (!allowed(mask_kind, i, j, Sq, Skv, kvlen)) continue;
+        if (p[j] == -INFINITY) { p[j] = 0.0; continue; }
         p[j] /= denom;
         for (int d = 0; d < D; ++d) orow[d] += p[j] * vmat[(size_t)j * D + d];
     }
@@ -108,9 +121,10 @@ static void attn_row(const double *qrow, const double *kmat, const double *vmat,
 
 static int attn_impl(const double *q, const double *k, const double *v, double *out, double *probs,
                      int B, int Hq, int Hkv, int Sq, int Skv, int D,
-                     int mask_kind, const int32_t *lens, double scale)
+                     int mask_kind, const int32_t *lens, double scale, const double *bias, int Hb)
 {
     if (check_attn_args(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens)) return 1;
+    if (bias && Hb != 1 && Hb != Hq) return 1;
     const int G = Hq / Hkv;
     int failed = 0;
 #pragma omp parallel for collapse(2) schedule(dynamic, 1)
@@ -125,7 +139,8 @@ static int attn_impl(const double *q, const double *k, const double *v, double *
             for (int i = 0; i < Sq; ++i) {
                 size_t row = ((size_t)b * Hq + h) * (size_t)Sq + i;
                 double *p = probs ? probs + row * (size_t)Skv : scratch;
-                attn_row(q + row * D, kmat, vmat, out + row * D, p, i, Sq, Skv, D, mask_kind, kvlen, scale);
+                const double *bias_row = bias ? bias + (((size_t)b * Hb + (Hb == 1 ? 0 : h)) * (size_t)Sq + i) * (size_t)Skv : NULL;
+                attn_row(q + row * D, kmat, vmat, out + row * D, p, i, Sq, Skv, D, mask_kind, kvlen, scale, bias_row);
             }
             free(scratch);
         }
@@ -138,7 +153,7 @@ int forge_ref_attn(const double *q, const double *k, const double *v, double *ou
                    int B, int Hq, int Hkv, int Sq, int Skv, int D,
                    int mask_kind, const int32_t *lens, double scale)
 {
-    return attn_impl(q, k, v, out, NULL, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale);
+    return attn_impl(q, k, v, out, NULL, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, NULL, 0);
 }
 
 /* Same, and also returns the probability matrix softmax(mask(scale Q K^T)) that the
@@ -148,7 +163,17 @@ int forge_ref_attn_probs(const double *q, const double *k, const double *v, doub
                          int mask_kind, const int32_t *lens, double scale)
 {
     if (!probs) return 1;
-    return attn_impl(q, k, v, out, probs, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale);
+    return attn_impl(q, k, v, out, probs, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, NULL, 0);
+}
+
+/* Fused attention with an additive bias tensor [B, Hb, Sq, Skv] on the scaled scores (Eq. 8 with its
+ * optional mask node as a tensor).  probs may be NULL. */
+int forge_ref_attn_bias(const double *q, const double *k, const double *v, double *out, double *probs,
+                        int B, int Hq, int Hkv, int Sq, int Skv, int D,
+                        int mask_kind, const int32_t *lens, double scale, const double *bias, int Hb)
+{
+    if (!bias) return 1;
+    return attn_impl(q, k, v, out, probs, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, bias, Hb);
 }
 
 /*
@@ -159,7 +184,7 @@ int forge_ref_attn_decode(const double *q, const double *k_cache, const double *
                           int B, int Hq, int Hkv, int Smax, int D, const int32_t *lens, double scale)
 {
     if (!lens) return 1;
-    return attn_impl(q, k_cache, v_cache, out, NULL, B, Hq, Hkv, 1, Smax, D, 2, lens, scale);
+    return attn_impl(q, k_cache, v_cache, out, NULL, B, Hq, Hkv, 1, Smax, D, 2, lens, scale, NULL, 0);
 }
 
 /* tanh form of GELU: 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3))). */

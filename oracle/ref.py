@@ -34,6 +34,7 @@ def _configure(lib):
     i = ctypes.c_int
     lib.forge_ref_attn.argtypes = [_dp, _dp, _dp, _dp, i, i, i, i, i, i, i, _ip, ctypes.c_double]
     lib.forge_ref_attn_probs.argtypes = [_dp, _dp, _dp, _dp, _dp, i, i, i, i, i, i, i, _ip, ctypes.c_double]
+    lib.forge_ref_attn_bias.argtypes = [_dp, _dp, _dp, _dp, _dp, i, i, i, i, i, i, i, _ip, ctypes.c_double, _dp, i]
     lib.forge_ref_attn_decode.argtypes = [_dp, _dp, _dp, _dp, i, i, i, i, i, _ip, ctypes.c_double]
     lib.forge_ref_linear_bias_gelu.argtypes = [_dp, _dp, _dp, _dp, i, i, i]
     lib.forge_ref_linear_act.argtypes = [_dp, _dp, _dp, _dp, _dp, i, i, i, i, i]
@@ -100,6 +101,23 @@ def attn_probs(q, k, v, mask_kind=0, lens=None, scale=1.0):
     _check(_load().forge_ref_attn_probs(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(probs), B, Hq, Hkv,
                                         Sq, Skv, D, int(mask_kind), lp, float(scale)), "forge_ref_attn_probs")
     return out, probs
+
+
+def attn_bias(q, k, v, bias, mask_kind=0, lens=None, scale=1.0, return_probs=False):
+    """Attention with an additive bias [B, Hb, Sq, Skv] (Hb = 1 or Hq) on the scaled scores."""
+    q, k, v, bias = _f64(q), _f64(k), _f64(v), _f64(bias)
+    B, Hq, Sq, D = q.shape
+    _, Hkv, Skv, _ = k.shape
+    assert k.shape == v.shape == (B, Hkv, Skv, D)
+    Hb = bias.shape[1]
+    assert bias.shape == (B, Hb, Sq, Skv)
+    out = np.empty_like(q)
+    probs = np.empty((B, Hq, Sq, Skv), dtype=np.float64) if return_probs else None
+    keep, lp = _lens_ptr(lens)
+    _check(_load().forge_ref_attn_bias(_ptr(q), _ptr(k), _ptr(v), _ptr(out), None if probs is None else _ptr(probs),
+                                       B, Hq, Hkv, Sq, Skv, D, int(mask_kind), lp, float(scale), _ptr(bias), Hb),
+           "forge_ref_attn_bias")
+    return (out, probs) if return_probs else out
 
 
 def attn_decode(q, k_cache, v_cache, lens, scale=1.0):

@@ -33,6 +33,11 @@ MUTANTS = {
     "W indexed [N,K]": ("w[(size_t)kk * N + n]", "w[(size_t)n * K + kk]"),
     "bias dropped": ("forge_ref_gelu_tanh(acc + b[n])", "forge_ref_gelu_tanh(acc)"),
     "bias indexed by row": ("forge_ref_gelu_tanh(acc + b[n])", "forge_ref_gelu_tanh(acc + b[m % N])"),
+    "attention bias dropped": ("        if (bias_row) s += bias_row[j];\n", ""),
+    "attention bias scaled": ("        s *= scale;\n        if (bias_row) s += bias_row[j];", "        if (bias_row) s += bias_row[j];\n        s *= scale;"),
+    "attention bias subtracted": ("if (bias_row) s += bias_row[j];", "if (bias_row) s -= bias_row[j];"),
+    "attention bias of another head": ("(Hb == 1 ? 0 : h)) * (size_t)Sq + i)", "(Hb == 1 ? 0 : (h + 1) % Hq)) * (size_t)Sq + i)"),
+    "attention bias transposed": ("(Hb == 1 ? 0 : h)) * (size_t)Sq + i) * (size_t)Skv", "(Hb == 1 ? 0 : h)) * (size_t)Sq) * (size_t)Skv + i"),
 }
 
 
@@ -64,6 +69,17 @@ def _pins():
     tq, tk, tv = (torch.from_numpy(a) for a in (q, k, v))
     ref_out = torch.nn.functional.scaled_dot_product_attention(tq, tk, tv, scale=0.4).numpy()
     np.testing.assert_allclose(oracle.attn(q, k, v, 0, None, 0.4), ref_out, atol=1e-13)
+    # additive bias tensor: exact hand weights, unscaled, per head, -inf excludes (also a whole row)
+    q0 = np.zeros((1, 2, 2, 2)); kb = RNG.standard_normal((1, 1, 3, 2)); vb = np.array([[[[8.0, 0.0], [0.0, 8.0], [16.0, 16.0]]]])
+    bias = np.zeros((1, 2, 2, 3)); bias[0, 1, 1] = [0.0, ln(2), ln(5)]; bias[0, 0, 1] = [0.0, -np.inf, -np.inf]
+    bias[0, 1, 0] = -np.inf
+    ob = oracle.attn_bias(q0, kb, vb, bias, 0, None, 0.37)
+    np.testing.assert_allclose(ob[0, 1, 1], [11.0, 12.0], atol=1e-14)
+    np.testing.assert_allclose(ob[0, 0, 1], [8.0, 0.0], atol=1e-14)
+    np.testing.assert_allclose(ob[0, 0, 0], [8.0, 8.0], atol=1e-14)
+    assert np.all(ob[0, 1, 0] == 0.0)
+    q1 = np.array([[[[1.0]]]]); k1 = np.array([[[[0.0], [2 * ln(3)]]]]); v1 = np.array([[[[10.0], [0.0]]]])
+    np.testing.assert_allclose(oracle.attn_bias(q1, k1, v1, np.array([[[[ln(2), 0.0]]]]), 0, None, 0.5), [[[[4.0]]]], atol=1e-14)
     # GELU and linear
     assert abs(oracle.gelu_tanh(1.0) - 0.841192) < 5e-7
     assert abs(oracle.gelu_tanh(3.0) - oracle.gelu_tanh(-3.0) - 3.0) < 1e-14

@@ -81,6 +81,22 @@ int forge_attn_fused_f16(const void* q, const void* k, const void* v, void* out,
                          int mask_kind, const int32_t* lens, float scale, void* stream);
 
 /*
+ * forge_attn_fused with the optional mask node of the fused pattern (Eq. 8) given as a
+ * tensor: bias [B, bias_heads, Sq, Skv] fp32 on the device (16-byte aligned, contiguous),
+ * bias_heads = 1 (shared by all query heads) or Hq, is added to the scaled scores before
+ * the softmax:  softmax_j(scale * q.k_j + bias[b, h, i, j]).  An entry of -infinity
+ * excludes the key; a row whose keys are all excluded gives zeros.  Finite entries are
+ * arbitrary (relative-position or ALiBi-style biases), but a "large negative" stand-in
+ * for -infinity must stay finite after division by scale.  mask_kind / lens apply on top.
+ * bf16 q, k, v, out as in forge_attn_fused.  scale must be > 0 (FORGE_ERR_UNSUPPORTED
+ * otherwise); other errors as forge_attn_fused.
+ */
+int forge_attn_fused_bias(const void* q, const void* k, const void* v, void* out,
+                          int B, int Hq, int Hkv, int Sq, int Skv, int D,
+                          int mask_kind, const int32_t* lens, const float* bias, int bias_heads,
+                          float scale, void* stream);
+
+/*
  * Same operator with fp32 tensors in and out (fp32 FMA arithmetic, no reduced
  * precision inside).  D must be 64 or 128.
  */

@@ -26,6 +26,7 @@ SIGNATURES = {
     "forge_attn_fused": (_i, _ATTN + [_vp]),
     "forge_attn_fused_f32": (_i, _ATTN + [_vp]),
     "forge_attn_fused_f16": (_i, _ATTN + [_vp]),
+    "forge_attn_fused_bias": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _i, _vp, _vp, _i, _f, _vp]),
     "forge_attn_decode_splitkv": (_i, _DEC + [_vp, _sz, _vp]),
     "forge_attn_decode_workspace_bytes": (_sz, [_i, _i, _i, _i]),
     "forge_attn_decode_splitkv_static": (_i, _DEC + [_vp]),
@@ -122,6 +123,21 @@ def attn_fused_f16(q, k, v, mask_kind=MASK_NONE, lens=None, scale=None, out=None
     _check("forge_attn_fused_f16", load().forge_attn_fused_f16(
         _dev(q, torch.float16, "q"), _dev(k, torch.float16, "k"), _dev(v, torch.float16, "v"),
         _dev(out, torch.float16, "out"), B, Hq, Hkv, Sq, Skv, D, int(mask_kind), lp, float(scale), _stream()))
+    return out
+
+
+def attn_fused_bias(q, k, v, bias, mask_kind=MASK_NONE, lens=None, scale=None, out=None):
+    """forge_attn_fused_bias: bf16 q/k/v and an fp32 additive bias [B, 1 or Hq, Sq, Skv] on the scaled scores."""
+    B, Hq, Hkv, Sq, Skv, D = _attn_dims(q, k, v)
+    if bias.dim() != 4 or bias.shape[0] != B or bias.shape[2] != Sq or bias.shape[3] != Skv:
+        raise ValueError("bias [B, 1 or Hq, Sq, Skv] expected")
+    out = torch.empty_like(q) if out is None else out
+    scale = D ** -0.5 if scale is None else scale
+    lp = None if lens is None else _dev(lens, torch.int32, "lens")
+    _check("forge_attn_fused_bias", load().forge_attn_fused_bias(
+        _dev(q, torch.bfloat16, "q"), _dev(k, torch.bfloat16, "k"), _dev(v, torch.bfloat16, "v"),
+        _dev(out, torch.bfloat16, "out"), B, Hq, Hkv, Sq, Skv, D, int(mask_kind), lp,
+        _dev(bias, torch.float32, "bias"), int(bias.shape[1]), float(scale), _stream()))
     return out
 
 

@@ -153,6 +153,9 @@ __device__ __forceinline__ int fast_div(int n, const FastDiv& f) {
 struct AttnParams {
     uint16_t* out;  // bf16 or fp16 elements
     const int32_t* lens;
+    const float* bias;  // additive bias on the scaled scores [B, bias_heads, Sq, Skv], or nullptr
+    int bias_heads;     // 1 (shared by all heads) or Hq
+    float inv_scale;    // 1 / scale: the bias is added to the unscaled scores as bias / scale
     int B, Hq, Hkv, Sq, Skv;
     int mask_kind;
     float scale_log2;  // > 0 (a zero scale is passed as the smallest normal number: every product flushes to 0)
@@ -175,7 +178,7 @@ struct ItemInfo {
 // element t of a two-element array without dynamic indexing (keeps the array in registers)
 __device__ __forceinline__ int pick(const int (&a)[kTilesPerCta], int t) { return t ? a[1] : a[0]; }
 
-template <int D, bool F16>
+template <int D, bool F16, bool BIAS>
 __global__ void __launch_bounds__(kThreads, 1)
 attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                  const __grid_constant__ CUtensorMap tmap_v, const __grid_constant__ CUtensorMap tmap_o,
@@ -504,7 +507,30 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 tmem_ld_wait();
 
                 const int key0 = (g >> 1) * kBN + hh * kHalf;
-                const bool need_mask = (key0 + kHalf > it.kvlen) || (causal && (key0 + kHalf - 1 > q0 + causal_off));
+                const bool need_mask = (key0 + kHalf > it.kvlen) || (causal && (key0 + kHalf - 1 > q0 + causal_off)) ||
+                                       BIAS;  // a bias may hold -inf: the path that tolerates it
+                if constexpr (BIAS) {
+                    // Eq. 8's mask node as a tensor: scale * s + bias = scale * (s + bias / scale)
+                    const int hb = p.bias_heads == 1 ? 0 : pick(it.h, t);
+                    const float* brow = p.bias + (((size_t)it.b * p.bias_heads + hb) * p.Sq + min(qi, p.Sq - 1)) * (size_t)p.Skv + key0;
+                    const int nvalid = min(kHalf, p.Skv - key0);  // columns beyond Skv are masked below
+                    if ((p.Skv & 3) == 0) {  // rows start on 16-byte boundaries
+#pragma unroll
+                        for (int c = 0; c < kHalf / 4; ++c) {
+                            if (c * 4 < nvalid) {
+                                const float4 bv = __ldg(reinterpret_cast<const float4*>(brow) + c);
+                                s[4 * c] = fmaf(bv.x, p.inv_scale, s[4 * c]);
+                                s[4 * c + 1] = fmaf(bv.y, p.inv_scale, s[4 * c + 1]);
+                                s[4 * c + 2] = fmaf(bv.z, p.inv_scale, s[4 * c + 2]);
+                                s[4 * c + 3] = fmaf(bv.w, p.inv_scale, s[4 * c + 3]);
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int k = 0; k < kHalf; ++k)
+                            if (k < nvalid) s[k] = fmaf(__ldg(brow + k), p.inv_scale, s[k]);
+                    }
+                }
                 bool stored = false;
                 if (need_mask) {
                     const int lim = row_limit - key0;  // last visible column of this half
@@ -678,9 +704,10 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     }
 }
 
-template <int D, bool F16>
+template <int D, bool F16, bool BIAS = false>
 int launch_attn(const void* q, const void* k, const void* v, void* out, int B, int Hq, int Hkv, int Sq, int Skv,
-                int mask_kind, const int32_t* lens, float scale, cudaStream_t s) {
+                int mask_kind, const int32_t* lens, float scale, cudaStream_t s, const float* bias = nullptr,
+                int bias_heads = 1) {
     using L = AttnSmem<D>;
     CUtensorMap tq, tk, tv;
     const uint32_t box[3] = {64, 128, 1};
@@ -707,6 +734,9 @@ int launch_attn(const void* q, const void* k, const void* v, void* out, int B, i
     AttnParams p;
     p.out = static_cast<uint16_t*>(out);
     p.lens = lens;
+    p.bias = bias;
+    p.bias_heads = bias_heads;
+    p.inv_scale = scale > 0.f ? 1.f / scale : 0.f;
     p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.Sq = Sq; p.Skv = Skv;
     p.mask_kind = mask_kind;
     p.scale_log2 = scale * 1.4426950408889634f;
@@ -722,7 +752,7 @@ int launch_attn(const void* q, const void* k, const void* v, void* out, int B, i
         p.div_inner = make_fastdiv(inner);
         p.div_group = make_fastdiv(G);
     }
-    auto kernel = attn_bf16_kernel<D, F16>;
+    auto kernel = attn_bf16_kernel<D, F16, BIAS>;
     FORGE_SET_SMEM_ONCE(kernel, L::kAlloc);
     const int sms = sm_count();
     if (sms <= 0) return FORGE_ERR_CUDA;
@@ -762,4 +792,20 @@ extern "C" int forge_attn_fused_f16(const void* q, const void* k, const void* v,
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     return D == 64 ? launch_attn<64, true>(q, k, v, out, B, Hq, Hkv, Sq, Skv, mask_kind, lens, scale, s)
                    : launch_attn<128, true>(q, k, v, out, B, Hq, Hkv, Sq, Skv, mask_kind, lens, scale, s);
+}
+
+extern "C" int forge_attn_fused_bias(const void* q, const void* k, const void* v, void* out,
+                                     int B, int Hq, int Hkv, int Sq, int Skv, int D,
+                                     int mask_kind, const int32_t* lens, const float* bias, int bias_heads,
+                                     float scale, void* stream) {
+    using namespace forge;
+    int st = check_attn_args(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens);
+    if (st != FORGE_OK) return st;
+    if (!bias || (reinterpret_cast<uintptr_t>(bias) & 15u)) return FORGE_ERR_INVALID_ARG;
+    if (bias_heads != 1 && bias_heads != Hq) return FORGE_ERR_INVALID_ARG;
+    if ((long long)Hq * B * ((Sq + 255) / 256) > 2147483647LL) return FORGE_ERR_UNSUPPORTED;
+    if (!(scale > 0.f)) return FORGE_ERR_UNSUPPORTED;  // the bias enters the kernel as bias / scale
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    return D == 64 ? launch_attn<64, false, true>(q, k, v, out, B, Hq, Hkv, Sq, Skv, mask_kind, lens, scale, s, bias, bias_heads)
+                   : launch_attn<128, false, true>(q, k, v, out, B, Hq, Hkv, Sq, Skv, mask_kind, lens, scale, s, bias, bias_heads);
 }

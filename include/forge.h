@@ -183,6 +183,18 @@ int forge_linear_act(const void* x, const void* w, const void* b, const void* re
                      int M, int N, int K, int act, int w_layout, void* stream);
 
 /*
+ * Gated MLP input of the 1B-8B decoder models of the evaluation (SwiGLU; Section 2, model overview): the
+ * linear+silu pattern of the operator-fusion pass and the element-wise product with the second
+ * projection, in one kernel:
+ *     y[m,n] = silu(sum_k x[m,k] * Wg(k,n)) * (sum_k x[m,k] * Wu(k,n)),   silu(z) = z / (1 + exp(-z))
+ * x [M,K], w_gate and w_up both [K,N] (FORGE_W_KN) or both [N,K] (FORGE_W_NK), y [M,N]; bf16 in and
+ * out, fp32 accumulation; neither product reaches memory.  No bias (these models have none here).
+ * K and N must be multiples of 8.  Errors as forge_linear_act.
+ */
+int forge_linear_swiglu(const void* x, const void* w_gate, const void* w_up, void* y,
+                        int M, int N, int K, int w_layout, void* stream);
+
+/*
  * Host-buffer variants: the same operators for callers whose tensors live in
  * HOST memory (pinned memory makes the copies asynchronous).  Inputs are copied
  * to `dev_scratch`, the operator runs there, and the result is copied back to the

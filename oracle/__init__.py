@@ -10,6 +10,7 @@ from .ref import (  # noqa: F401
     attn_decode,
     linear_bias_gelu,
     linear_act,
+    linear_swiglu,
     ACT_GELU_TANH,
     ACT_GELU_ERF,
     ACT_RELU,

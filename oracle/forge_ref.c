@@ -254,3 +254,29 @@ int forge_ref_num_threads(void) { return omp_get_max_threads(); }
 #else
 int forge_ref_num_threads(void) { return 1; }
 #endif
+
+/*
+ * Gated MLP input (SwiGLU, the form the 1B-8B decoder models of the evaluation use; the operator-fusion
+ * pass's linear+silu pattern followed by the element-wise product with a second projection):
+ *     y[m, n] = silu(sum_k x[m, k] wg(k, n)) * (sum_k x[m, k] wu(k, n)),   silu(z) = z / (1 + exp(-z))
+ * wg, wu stored [K, N] (w_layout 0) or [N, K] (w_layout 1).
+ */
+int forge_ref_linear_swiglu(const double *x, const double *wg, const double *wu, double *y,
+                            int M, int N, int K, int w_layout)
+{
+    if (!x || !wg || !wu || !y || M <= 0 || N <= 0 || K <= 0) return 1;
+    if (w_layout < 0 || w_layout > 1) return 1;
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        for (int n = 0; n < N; ++n) {
+            double gate = 0.0, up = 0.0;
+            for (int kk = 0; kk < K; ++kk) {
+                const size_t wi = w_layout == 0 ? (size_t)kk * N + n : (size_t)n * K + kk;
+                gate += x[(size_t)m * K + kk] * wg[wi];
+                up += x[(size_t)m * K + kk] * wu[wi];
+            }
+            y[(size_t)m * N + n] = gate / (1.0 + exp(-gate)) * up;
+        }
+    }
+    return 0;
+}

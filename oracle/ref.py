@@ -38,6 +38,7 @@ def _configure(lib):
     lib.forge_ref_attn_decode.argtypes = [_dp, _dp, _dp, _dp, i, i, i, i, i, _ip, ctypes.c_double]
     lib.forge_ref_linear_bias_gelu.argtypes = [_dp, _dp, _dp, _dp, i, i, i]
     lib.forge_ref_linear_act.argtypes = [_dp, _dp, _dp, _dp, _dp, i, i, i, i, i]
+    lib.forge_ref_linear_swiglu.argtypes = [_dp, _dp, _dp, _dp, i, i, i, i]
     lib.forge_ref_gelu_tanh.argtypes = [ctypes.c_double]
     lib.forge_ref_gelu_tanh.restype = ctypes.c_double
     lib.forge_ref_num_threads.restype = i
@@ -160,6 +161,18 @@ def linear_act(x, w, b=None, residual=None, act=ACT_GELU_TANH, w_layout=0):
     _check(_load().forge_ref_linear_act(_ptr(x), _ptr(w), None if b is None else _ptr(b),
                                         None if residual is None else _ptr(residual), _ptr(y), M, N, K,
                                         int(act), int(w_layout)), "forge_ref_linear_act")
+    return y
+
+
+def linear_swiglu(x, wg, wu, w_layout=0):
+    """silu(x Wg) * (x Wu); Wg, Wu are [K,N] (w_layout 0) or [N,K] (w_layout 1)."""
+    x, wg, wu = _f64(x), _f64(wg), _f64(wu)
+    M, K = x.shape
+    N = wg.shape[1] if w_layout == 0 else wg.shape[0]
+    assert wg.shape == wu.shape == ((K, N) if w_layout == 0 else (N, K))
+    y = np.empty((M, N), dtype=np.float64)
+    _check(_load().forge_ref_linear_swiglu(_ptr(x), _ptr(wg), _ptr(wu), _ptr(y), M, N, K, int(w_layout)),
+           "forge_ref_linear_swiglu")
     return y
 
 

@@ -32,6 +32,7 @@ SIGNATURES = {
     "forge_attn_decode_splitkv_static": (_i, _DEC + [_vp]),
     "forge_linear_bias_gelu": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
     "forge_linear_act": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]),
+    "forge_linear_swiglu": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp]),
     "forge_attn_host_scratch_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _i]),
     "forge_attn_fused_host": (_i, _ATTN + [_vp, _sz, _vp]),
     "forge_attn_fused_f32_host": (_i, _ATTN + [_vp, _sz, _vp]),
@@ -229,6 +230,21 @@ def linear_act(x, w, b=None, residual=None, act=ACT_GELU_TANH, w_layout=W_KN, ou
         _dev(x, bf, "x"), _dev(w, bf, "w"), None if b is None else _dev(b, bf, "b"),
         None if residual is None else _dev(residual, bf, "residual"), _dev(out, bf, "out"),
         M, N, K, int(act), int(w_layout), _stream()))
+    return out
+
+
+def linear_swiglu(x, w_gate, w_up, w_layout=W_KN, out=None):
+    """forge_linear_swiglu: silu(x @ Wg) * (x @ Wu); both weights [K,N] (W_KN) or [N,K] (W_NK)."""
+    M, K = x.shape
+    N = w_gate.shape[1] if w_layout == W_KN else w_gate.shape[0]
+    want = (K, N) if w_layout == W_KN else (N, K)
+    if tuple(w_gate.shape) != want or tuple(w_up.shape) != want:
+        raise ValueError("w_gate and w_up must both be [K,N] for W_KN or [N,K] for W_NK")
+    out = torch.empty((M, N), dtype=torch.bfloat16, device=x.device) if out is None else out
+    bf = torch.bfloat16
+    _check("forge_linear_swiglu", load().forge_linear_swiglu(
+        _dev(x, bf, "x"), _dev(w_gate, bf, "w_gate"), _dev(w_up, bf, "w_up"), _dev(out, bf, "out"),
+        M, N, K, int(w_layout), _stream()))
     return out
 
 

@@ -9,6 +9,10 @@
 // Two TMEM accumulators: the epilogue of tile i overlaps the main loop of tile i+1.
 // X [M,K] is the K-major A operand; W [K,N] (N contiguous) is the MN-major B operand, so no
 // transposed copy of the weights is needed.
+// Gated form (SwiGLU, the MLP of the 1B-8B decoder models): Y = silu(X Wg) * (X Wu).  One tile holds
+// 128 output columns; its accumulator is 256 columns wide, the gate product in the first half and the
+// up product in the second (the B operand of a stage is the gate tile followed by the up tile, one MMA
+// of N = 256 per k-step), and the epilogue multiplies the two halves as it reads them back.
 #include <cuda_bf16.h>
 
 #include "forge_common.cuh"
@@ -66,10 +70,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 }
 
 // ACT: activation; W_NK: W is stored [N, K] (K-major B operand) instead of [K, N] (MN-major B operand).
+// GATED: two weight matrices (tmap_w = gate, tmap_w2 = up), output silu(gate) * up, BN / 2 output columns per tile.
 // bias and residual may be null.
-template <int BN, int STAGES, int ACT, bool W_NK>
+template <int BN, int STAGES, int ACT, bool W_NK, bool GATED>
 __global__ void __launch_bounds__(kThreads, 1)
 linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+                        const __grid_constant__ CUtensorMap tmap_w2,
                         const __grid_constant__ CUtensorMap tmap_y, const __nv_bfloat16* __restrict__ bias,
                         const __nv_bfloat16* __restrict__ residual, int M, int N, int K, int* __restrict__ status) {
     using L = LinearSmem<BN, STAGES>;
@@ -83,7 +89,8 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
     float* s_bias = reinterpret_cast<float*>(smem + L::kBiasOffset);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tiles_m = (M + kBM - 1) / kBM, tiles_n = (N + BN - 1) / BN;
+    constexpr int BNO = GATED ? BN / 2 : BN;  // output columns per tile
+    const int tiles_m = (M + kBM - 1) / kBM, tiles_n = (N + BNO - 1) / BNO;
     const int num_tiles = tiles_m * tiles_n;
     const int kblocks = (K + kBK - 1) / kBK;
 
@@ -93,6 +100,7 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
         fence_mbar_init();
         prefetch_tmap(&tmap_x);
         prefetch_tmap(&tmap_w);
+        if constexpr (GATED) prefetch_tmap(&tmap_w2);
         prefetch_tmap(&tmap_y);
     }
     if (warp == 1) {
@@ -114,7 +122,7 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
             int stage = 0;
             uint32_t phase = 0;
             for (int tile = blockIdx.x; tile < num_tiles && !failed; tile += gridDim.x) {
-                const int m0 = (tile / tiles_n) * kBM, n0 = (tile % tiles_n) * BN;
+                const int m0 = (tile / tiles_n) * kBM, n0 = (tile % tiles_n) * BNO;
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!mbar_wait(&empty[stage], phase ^ 1)) { failed = true; break; }
                     uint8_t* sa = smem + stage * L::kStageBytes;
@@ -123,10 +131,16 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
                     tma_load_2d(sa, &tmap_x, &full[stage], kb * kBK, m0);
                     if constexpr (W_NK) {  // BN rows of W, 64 K-elements (one swizzle span) each
                         tma_load_2d(sb, &tmap_w, &full[stage], kb * kBK, n0);
+                        if constexpr (GATED)  // rows BN/2.. of the operand: the up weights of the same columns
+                            tma_load_2d(sb + (BN / 2) * 128, &tmap_w2, &full[stage], kb * kBK, n0);
                     } else {
 #pragma unroll
-                        for (int c = 0; c < BN / 64; ++c)
-                            tma_load_2d(sb + c * (kBK * 128), &tmap_w, &full[stage], n0 + c * 64, kb * kBK);
+                        for (int c = 0; c < BN / 64; ++c) {
+                            if (GATED && c >= BN / 128)
+                                tma_load_2d(sb + c * (kBK * 128), &tmap_w2, &full[stage], n0 + (c - BN / 128) * 64, kb * kBK);
+                            else
+                                tma_load_2d(sb + c * (kBK * 128), &tmap_w, &full[stage], n0 + c * 64, kb * kBK);
+                        }
                     }
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
@@ -173,11 +187,11 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
         int it = 0;
         int out_blocks = 0;  // 64-column blocks stored so far (selects the staging buffer)
         for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++it) {
-            const int m0 = (tile / tiles_n) * kBM, n0 = (tile % tiles_n) * BN;
+            const int m0 = (tile / tiles_n) * kBM, n0 = (tile % tiles_n) * BNO;
             const int acc = it & 1;
             const uint32_t acc_phase = (it >> 1) & 1;
             float* bias_s = s_bias + acc * BN;
-            for (int i = etid; i < BN; i += kEpiThreads)
+            for (int i = etid; i < BNO; i += kEpiThreads)
                 bias_s[i] = (bias != nullptr && n0 + i < N) ? __bfloat162float(bias[n0 + i]) : 0.f;
             asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
             // A warp that gave up keeps taking part in the named barrier above (so the others never
@@ -190,10 +204,18 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
             // 64 output columns at a time: registers -> bf16 -> swizzled staging buffer -> one TMA store.
             // Two staging buffers: the store of one block drains while the next block is computed.
 #pragma unroll 1
-            for (int blk = 0; blk < BN / 64; ++blk, ++out_blocks) {
+            for (int blk = 0; blk < BNO / 64; ++blk, ++out_blocks) {
                 uint8_t* stage_out = smem + L::kOutOffset + (out_blocks & 1) * L::kOutBytes;
                 uint32_t r[32];
                 tmem_ld_x32(taddr + blk * 64 + chalf * 32, r);
+                if constexpr (GATED) {  // silu(gate) * up, the up product sits BN / 2 columns further
+                    uint32_t r2[32];
+                    tmem_ld_x32(taddr + BN / 2 + blk * 64 + chalf * 32, r2);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        r[i] = __float_as_uint(activate<FORGE_ACT_SILU>(__uint_as_float(r[i])) * __uint_as_float(r2[i]));
+                }
                 tmem_ld_wait();
                 // the store issued two blocks ago has finished reading this buffer
                 if (etid == 0) tma_store_wait_read<1>();
@@ -212,8 +234,8 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
                         const int col = c * 8 + 2 * i;
                         const float z0 = __uint_as_float(r[col]) + bias_s[blk * 64 + chalf * 32 + col];
                         const float z1 = __uint_as_float(r[col + 1]) + bias_s[blk * 64 + chalf * 32 + col + 1];
-                        w[i] = pack_bf16(activate<ACT>(z0) + __uint_as_float(rw[i] << 16),
-                                         activate<ACT>(z1) + __uint_as_float(rw[i] & 0xffff0000u));
+                        w[i] = pack_bf16(activate<GATED ? FORGE_ACT_NONE : ACT>(z0) + __uint_as_float(rw[i] << 16),
+                                         activate<GATED ? FORGE_ACT_NONE : ACT>(z1) + __uint_as_float(rw[i] & 0xffff0000u));
                     }
                     *reinterpret_cast<uint4*>(stage_out + row * 128 + (((chalf * 4 + c) ^ (row & 7)) << 4)) =
                         make_uint4(w[0], w[1], w[2], w[3]);
@@ -246,11 +268,12 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
     }
 }
 
-template <int BN, int STAGES, int ACT, bool W_NK>
+template <int BN, int STAGES, int ACT, bool W_NK, bool GATED = false>
 int launch_linear(const void* x, const void* w, const void* b, const void* residual, void* y, int M, int N, int K,
-                  cudaStream_t s) {
+                  cudaStream_t s, const void* w_up = nullptr) {
     using L = LinearSmem<BN, STAGES>;
-    CUtensorMap tmap_x, tmap_w, tmap_y;
+    constexpr int BNO = GATED ? BN / 2 : BN;
+    CUtensorMap tmap_x, tmap_w, tmap_w2, tmap_y;
     {
         const uint64_t dims[2] = {(uint64_t)K, (uint64_t)M};
         const uint64_t strides[1] = {(uint64_t)K * 2};
@@ -260,13 +283,15 @@ int launch_linear(const void* x, const void* w, const void* b, const void* resid
     if (W_NK) {  // w[N, K]: rows of 64 K-elements
         const uint64_t dims[2] = {(uint64_t)K, (uint64_t)N};
         const uint64_t strides[1] = {(uint64_t)K * 2};
-        const uint32_t box[2] = {kBK, BN};
+        const uint32_t box[2] = {kBK, BNO};
         if (!encode_tmap_bf16_sw128(&tmap_w, w, 2, dims, strides, box)) return FORGE_ERR_CUDA;
+        if (!encode_tmap_bf16_sw128(&tmap_w2, GATED ? w_up : w, 2, dims, strides, box)) return FORGE_ERR_CUDA;
     } else {     // w[K, N]: 64 K-rows of 64 N-elements per box
         const uint64_t dims[2] = {(uint64_t)N, (uint64_t)K};
         const uint64_t strides[1] = {(uint64_t)N * 2};
         const uint32_t box[2] = {64, kBK};
         if (!encode_tmap_bf16_sw128(&tmap_w, w, 2, dims, strides, box)) return FORGE_ERR_CUDA;
+        if (!encode_tmap_bf16_sw128(&tmap_w2, GATED ? w_up : w, 2, dims, strides, box)) return FORGE_ERR_CUDA;
     }
     {
         const uint64_t dims[2] = {(uint64_t)N, (uint64_t)M};
@@ -278,11 +303,11 @@ int launch_linear(const void* x, const void* w, const void* b, const void* resid
     if (!status) return FORGE_ERR_CUDA;
     const int sms = sm_count();
     if (sms <= 0) return FORGE_ERR_CUDA;
-    auto kernel = linear_bias_gelu_kernel<BN, STAGES, ACT, W_NK>;
+    auto kernel = linear_bias_gelu_kernel<BN, STAGES, ACT, W_NK, GATED>;
     FORGE_SET_SMEM_ONCE(kernel, L::kAlloc);
-    const int tiles = ((M + kBM - 1) / kBM) * ((N + BN - 1) / BN);
+    const int tiles = ((M + kBM - 1) / kBM) * ((N + BNO - 1) / BNO);
     const int grid = tiles < sms ? tiles : sms;
-    FORGE_CUDA_TRY(launch_pdl(kernel, dim3(grid), dim3(kThreads), L::kAlloc, s, tmap_x, tmap_w, tmap_y,
+    FORGE_CUDA_TRY(launch_pdl(kernel, dim3(grid), dim3(kThreads), L::kAlloc, s, tmap_x, tmap_w, tmap_w2, tmap_y,
                               static_cast<const __nv_bfloat16*>(b), static_cast<const __nv_bfloat16*>(residual),
                               M, N, K, status));
     return finish_launch(1);
@@ -322,4 +347,18 @@ extern "C" int forge_linear_bias_gelu(const void* x, const void* w, const void* 
                                       int M, int N, int K, void* stream) {
     if (!b) return FORGE_ERR_INVALID_ARG;
     return forge_linear_act(x, w, b, nullptr, y, M, N, K, FORGE_ACT_GELU_TANH, FORGE_W_KN, stream);
+}
+
+extern "C" int forge_linear_swiglu(const void* x, const void* w_gate, const void* w_up, void* y,
+                                   int M, int N, int K, int w_layout, void* stream) {
+    using namespace forge;
+    if (!x || !w_gate || !w_up || !y) return FORGE_ERR_INVALID_ARG;
+    if (M <= 0 || N <= 0 || K <= 0) return FORGE_ERR_INVALID_ARG;
+    if (w_layout != FORGE_W_KN && w_layout != FORGE_W_NK) return FORGE_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(w_gate) || !aligned16(w_up) || !aligned16(y)) return FORGE_ERR_INVALID_ARG;
+    if ((K % 8) != 0 || (N % 8) != 0) return FORGE_ERR_UNSUPPORTED;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    return w_layout == FORGE_W_NK
+               ? launch_linear<256, 3, FORGE_ACT_SILU, true, true>(x, w_gate, nullptr, nullptr, y, M, N, K, s, w_up)
+               : launch_linear<256, 3, FORGE_ACT_SILU, false, true>(x, w_gate, nullptr, nullptr, y, M, N, K, s, w_up);
 }

@@ -132,3 +132,34 @@ def test_linear_act_matches_the_gelu_entry_and_mm_add():
     np.testing.assert_allclose(oracle.linear_act(x, w, None, r, oracle.ACT_NONE), x @ w + r, rtol=0, atol=1e-14)
     with pytest.raises(ValueError):
         oracle.linear_act(x, w, b, None, 9)
+
+
+# ---- gated form: silu(x Wg) * (x Wu)
+def test_swiglu_hand_values_and_closed_forms():
+    """K = 1: y = silu(x wg) * x wu.  silu(ln 3) = ln 3 / (1 + 1/3) = 0.75 ln 3; silu(0) = 0; wu = 0 gives 0."""
+    import math
+    x = np.array([[1.0], [2.0]]); wg = np.array([[math.log(3), 0.0]]); wu = np.array([[2.0, 5.0]])
+    y = oracle.linear_swiglu(x, wg, wu)
+    np.testing.assert_allclose(y[0], [0.75 * math.log(3) * 2.0, 0.0], atol=1e-15)
+    # row 1: gate = 2 ln 3 = ln 9: silu = ln 9 * 0.9; up = 4
+    np.testing.assert_allclose(y[1], [0.9 * math.log(9) * 4.0, 0.0], atol=1e-14)
+    assert np.all(oracle.linear_swiglu(RNG.standard_normal((3, 4)), RNG.standard_normal((4, 5)), np.zeros((4, 5))) == 0)
+    # the gate is the activated branch: swapping the weights changes the result
+    a = RNG.standard_normal((3, 4)); g = RNG.standard_normal((4, 5)); u = RNG.standard_normal((4, 5))
+    assert np.abs(oracle.linear_swiglu(a, g, u) - oracle.linear_swiglu(a, u, g)).max() > 1e-3
+    # silu(z) - silu(-z) = z: with the up projection fixed to ones, y(x) - y(-x)... uses gate only
+    ones = np.ones((4, 5))
+    up = a @ ones
+    d = oracle.linear_swiglu(a, g, ones) / up + oracle.linear_swiglu(-a, g, ones) / up   # silu(z) - silu(-z)
+    np.testing.assert_allclose(d, a @ g, atol=1e-12)
+
+
+@pytest.mark.parametrize("w_layout", [0, 1])
+def test_swiglu_against_torch_cpu(w_layout):
+    x = RNG.standard_normal((7, 9)); g = RNG.standard_normal((9, 6)); u = RNG.standard_normal((9, 6))
+    want = (torch.nn.functional.silu(torch.from_numpy(x @ g)) * torch.from_numpy(x @ u)).numpy()
+    gg, uu = (g, u) if w_layout == 0 else (np.ascontiguousarray(g.T), np.ascontiguousarray(u.T))
+    np.testing.assert_allclose(oracle.linear_swiglu(x, gg, uu, w_layout), want, atol=1e-13)
+    # equals the already pinned linear+silu pattern times a plain matrix product
+    np.testing.assert_allclose(oracle.linear_swiglu(x, g, u),
+                               oracle.linear_act(x, g, None, None, oracle.ACT_SILU) * (x @ u), atol=1e-13)

@@ -33,6 +33,10 @@ MUTANTS = {
     "W indexed [N,K]": ("w[(size_t)kk * N + n]", "w[(size_t)n * K + kk]"),
     "bias dropped": ("forge_ref_gelu_tanh(acc + b[n])", "forge_ref_gelu_tanh(acc)"),
     "bias indexed by row": ("forge_ref_gelu_tanh(acc + b[n])", "forge_ref_gelu_tanh(acc + b[m % N])"),
+    "swiglu gate and up swapped": ("y[(size_t)m * N + n] = gate / (1.0 + exp(-gate)) * up;", "y[(size_t)m * N + n] = up / (1.0 + exp(-up)) * gate;"),
+    "swiglu product dropped": ("gate / (1.0 + exp(-gate)) * up;", "gate / (1.0 + exp(-gate));"),
+    "swiglu sigmoid instead of silu": ("gate / (1.0 + exp(-gate)) * up;", "1.0 / (1.0 + exp(-gate)) * up;"),
+    "swiglu up weights transposed": ("up += x[(size_t)m * K + kk] * wu[wi];", "up += x[(size_t)m * K + kk] * wu[w_layout == 0 ? (size_t)n * K + kk : (size_t)kk * N + n];"),
     "attention bias dropped": ("        if (bias_row) s += bias_row[j];\n", ""),
     "attention bias scaled": ("        s *= scale;\n        if (bias_row) s += bias_row[j];", "        if (bias_row) s += bias_row[j];\n        s *= scale;"),
     "attention bias subtracted": ("if (bias_row) s += bias_row[j];", "if (bias_row) s -= bias_row[j];"),
@@ -80,6 +84,12 @@ def _pins():
     assert np.all(ob[0, 1, 0] == 0.0)
     q1 = np.array([[[[1.0]]]]); k1 = np.array([[[[0.0], [2 * ln(3)]]]]); v1 = np.array([[[[10.0], [0.0]]]])
     np.testing.assert_allclose(oracle.attn_bias(q1, k1, v1, np.array([[[[ln(2), 0.0]]]]), 0, None, 0.5), [[[[4.0]]]], atol=1e-14)
+    # gated MLP input: hand values (silu(ln 3) = 0.75 ln 3) and torch's silu on non-square weights
+    np.testing.assert_allclose(oracle.linear_swiglu(np.array([[1.0]]), np.array([[ln(3), 0.0]]), np.array([[2.0, 5.0]])),
+                               [[1.5 * ln(3), 0.0]], atol=1e-15)
+    xs = RNG.standard_normal((4, 5)); gs = RNG.standard_normal((5, 3)); us = RNG.standard_normal((5, 3))
+    np.testing.assert_allclose(oracle.linear_swiglu(xs, gs, us),
+                               (torch.nn.functional.silu(torch.from_numpy(xs @ gs)) * torch.from_numpy(xs @ us)).numpy(), atol=1e-13)
     # GELU and linear
     assert abs(oracle.gelu_tanh(1.0) - 0.841192) < 5e-7
     assert abs(oracle.gelu_tanh(3.0) - oracle.gelu_tanh(-3.0) - 3.0) < 1e-14

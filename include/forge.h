@@ -124,6 +124,13 @@ int forge_attn_decode_splitkv(const void* q, const void* k_cache, const void* v_
                               const int32_t* lens, int num_splits, float scale,
                               void* workspace, size_t workspace_bytes, void* stream);
 
+/* The same decode step with fp16 q, caches and out (the paper's inference precision); everything else,
+ * including the workspace size, as forge_attn_decode_splitkv. */
+int forge_attn_decode_splitkv_f16(const void* q, const void* k_cache, const void* v_cache, void* out,
+                                  int B, int Hq, int Hkv, int Smax, int D,
+                                  const int32_t* lens, int num_splits, float scale,
+                                  void* workspace, size_t workspace_bytes, void* stream);
+
 /* Bytes of workspace forge_attn_decode_splitkv needs; 0 for invalid arguments. */
 size_t forge_attn_decode_workspace_bytes(int B, int Hq, int D, int num_splits);
 
@@ -181,6 +188,10 @@ enum { FORGE_ACT_GELU_TANH = 0, FORGE_ACT_GELU_ERF = 1, FORGE_ACT_RELU = 2, FORG
 enum { FORGE_W_KN = 0, FORGE_W_NK = 1 };
 int forge_linear_act(const void* x, const void* w, const void* b, const void* residual, void* y,
                      int M, int N, int K, int act, int w_layout, void* stream);
+
+/* forge_linear_act with fp16 x, w, b, residual and y (fp32 accumulation; same arguments and limits). */
+int forge_linear_act_f16(const void* x, const void* w, const void* b, const void* residual, void* y,
+                         int M, int N, int K, int act, int w_layout, void* stream);
 
 /*
  * Gated MLP input of the 1B-8B decoder models of the evaluation (SwiGLU; Section 2, model overview): the

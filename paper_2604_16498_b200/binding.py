@@ -28,10 +28,12 @@ SIGNATURES = {
     "forge_attn_fused_f16": (_i, _ATTN + [_vp]),
     "forge_attn_fused_bias": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _i, _vp, _vp, _i, _f, _vp]),
     "forge_attn_decode_splitkv": (_i, _DEC + [_vp, _sz, _vp]),
+    "forge_attn_decode_splitkv_f16": (_i, _DEC + [_vp, _sz, _vp]),
     "forge_attn_decode_workspace_bytes": (_sz, [_i, _i, _i, _i]),
     "forge_attn_decode_splitkv_static": (_i, _DEC + [_vp]),
     "forge_linear_bias_gelu": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
     "forge_linear_act": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]),
+    "forge_linear_act_f16": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]),
     "forge_linear_swiglu": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp]),
     "forge_attn_host_scratch_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _i]),
     "forge_attn_fused_host": (_i, _ATTN + [_vp, _sz, _vp]),
@@ -159,7 +161,8 @@ def attn_decode_workspace_bytes(B, Hq, D, num_splits) -> int:
 
 
 def attn_decode_splitkv(q, k_cache, v_cache, lens, num_splits, scale=None, out=None, workspace=None):
-    """forge_attn_decode_splitkv: q [B,Hq,D], caches [B,Hkv,Smax,D] (bf16), lens int32 [B]."""
+    """forge_attn_decode_splitkv (bf16 tensors) or forge_attn_decode_splitkv_f16 (fp16 tensors), chosen by
+    q.dtype: q [B,Hq,D], caches [B,Hkv,Smax,D], lens int32 [B]."""
     B, Hq, D = q.shape
     Bk, Hkv, Smax, Dk = k_cache.shape
     if (Bk, Dk) != (B, D) or tuple(v_cache.shape) != tuple(k_cache.shape):
@@ -169,9 +172,11 @@ def attn_decode_splitkv(q, k_cache, v_cache, lens, num_splits, scale=None, out=N
     need = attn_decode_workspace_bytes(B, Hq, D, num_splits)
     if workspace is None:
         workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=q.device)
-    _check("forge_attn_decode_splitkv", load().forge_attn_decode_splitkv(
-        _dev(q, torch.bfloat16, "q"), _dev(k_cache, torch.bfloat16, "k_cache"),
-        _dev(v_cache, torch.bfloat16, "v_cache"), _dev(out, torch.bfloat16, "out"),
+    dt = torch.float16 if q.dtype == torch.float16 else torch.bfloat16
+    name = "forge_attn_decode_splitkv_f16" if dt == torch.float16 else "forge_attn_decode_splitkv"
+    _check(name, getattr(load(), name)(
+        _dev(q, dt, "q"), _dev(k_cache, dt, "k_cache"),
+        _dev(v_cache, dt, "v_cache"), _dev(out, dt, "out"),
         B, Hq, Hkv, Smax, D, _dev(lens, torch.int32, "lens"), int(num_splits), float(scale),
         _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream()))
     return out
@@ -215,7 +220,8 @@ W_KN, W_NK = 0, 1
 
 
 def linear_act(x, w, b=None, residual=None, act=ACT_GELU_TANH, w_layout=W_KN, out=None):
-    """forge_linear_act: act(x @ W + b) + residual with W given as [K,N] (W_KN) or [N,K] (W_NK)."""
+    """forge_linear_act (bf16 tensors) or forge_linear_act_f16 (fp16 tensors), chosen by x.dtype:
+    act(x @ W + b) + residual with W given as [K,N] (W_KN) or [N,K] (W_NK)."""
     M, K = x.shape
     N = w.shape[1] if w_layout == W_KN else w.shape[0]
     if tuple(w.shape) != ((K, N) if w_layout == W_KN else (N, K)):
@@ -224,9 +230,10 @@ def linear_act(x, w, b=None, residual=None, act=ACT_GELU_TANH, w_layout=W_KN, ou
         raise ValueError("b [N] expected")
     if residual is not None and tuple(residual.shape) != (M, N):
         raise ValueError("residual [M,N] expected")
-    out = torch.empty((M, N), dtype=torch.bfloat16, device=x.device) if out is None else out
-    bf = torch.bfloat16
-    _check("forge_linear_act", load().forge_linear_act(
+    out = torch.empty((M, N), dtype=x.dtype, device=x.device) if out is None else out
+    bf = torch.float16 if x.dtype == torch.float16 else torch.bfloat16
+    name = "forge_linear_act_f16" if bf == torch.float16 else "forge_linear_act"
+    _check(name, getattr(load(), name)(
         _dev(x, bf, "x"), _dev(w, bf, "w"), None if b is None else _dev(b, bf, "b"),
         None if residual is None else _dev(residual, bf, "residual"), _dev(out, bf, "out"),
         M, N, K, int(act), int(w_layout), _stream()))

@@ -21,6 +21,7 @@
 // on warp-level tensor-core MMAs (m16n8k16) with fragments read from the swizzled ring; fp32 FMAs
 // with shuffle reductions were bound by instruction issue.
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include <mutex>
 
@@ -46,17 +47,31 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
 //   A: a0 = (row g, k 2c..2c+1)  a1 = (row g+8, k 2c..)  a2 = (row g, k 2c+8..)  a3 = (row g+8, k 2c+8..)
 //   B: b0 = (k 2c..2c+1, col g)  b1 = (k 2c+8.., col g)
 //   D: d0 = (row g, col 2c)  d1 = (row g, col 2c+1)  d2 = (row g+8, col 2c)  d3 = (row g+8, col 2c+1)
+// F16 selects fp16 operands instead of bf16 (the same fragment layout).
+template <bool F16>
 __device__ __forceinline__ void mma16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, "
-                 "{%8, %9}, {%0, %1, %2, %3};"
-                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    if constexpr (F16)
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, "
+                     "{%8, %9}, {%0, %1, %2, %3};"
+                     : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                     : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    else
+        asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, "
+                     "{%8, %9}, {%0, %1, %2, %3};"
+                     : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                     : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t*>(&v);
+template <bool F16>
+__device__ __forceinline__ uint32_t pack16x2(float lo, float hi) {
+    if constexpr (F16) {
+        __half2 v = __floats2half2_rn(lo, hi);
+        return *reinterpret_cast<uint32_t*>(&v);
+    } else {
+        __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+        return *reinterpret_cast<uint32_t*>(&v);
+    }
 }
 
 // One (batch, kv head, split) work item and its range of cached rows.
@@ -89,10 +104,10 @@ __device__ __forceinline__ Item make_item(int idx, const int32_t* lens, const in
 //   online softmax on the accumulator fragment (lane (g, c) owns head g, keys 2c, 2c+1 of each 8);
 //   O^T[dim, head] += V^T P^T  with A = pairs of V rows interleaved with byte permutes and B = the
 //                   probabilities exactly where the first MMA left them.
-template <int D, int G>
+template <int D, int G, bool F16>
 __global__ void __launch_bounds__(kThreads, 1)
 decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
-                    const __nv_bfloat16* __restrict__ q, const int32_t* __restrict__ lens,
+                    const uint16_t* __restrict__ q, const int32_t* __restrict__ lens,
                     float* __restrict__ ws_o, float* __restrict__ ws_ml,
                     int B, int Hq, int Hkv, int Smax, int num_splits, float scale_log2, int* status) {
     constexpr int NKB = D / 32;  // 32-dim blocks of the head dimension (two k16 MMAs each)
@@ -264,8 +279,8 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 s[u][0] = s[u][1] = s[u][2] = s[u][3] = 0.f;
 #pragma unroll
                 for (int kb = 0; kb < NKB; ++kb) {
-                    mma16816(s[u], qr[kb][0], 0u, qr[kb][1], 0u, kr[u][kb].x, kr[u][kb].y);
-                    mma16816(s2, qr[kb][2], 0u, qr[kb][3], 0u, kr[u][kb].z, kr[u][kb].w);
+                    mma16816<F16>(s[u], qr[kb][0], 0u, qr[kb][1], 0u, kr[u][kb].x, kr[u][kb].y);
+                    mma16816<F16>(s2, qr[kb][2], 0u, qr[kb][3], 0u, kr[u][kb].z, kr[u][kb].w);
                 }
                 s[u][0] += s2[0];
                 s[u][1] += s2[1];
@@ -307,8 +322,8 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             }
 
             // P^T as the B operand: k-slots (2c, 2c+1) = keys 2c, 2c+1; (2c+8, 2c+9) = keys 2c+8, 2c+9
-            const uint32_t pb0 = pack_bf16x2(p[0][0], p[0][1]);
-            const uint32_t pb1 = pack_bf16x2(p[1][0], p[1][1]);
+            const uint32_t pb0 = pack16x2<F16>(p[0][0], p[0][1]);
+            const uint32_t pb1 = pack16x2<F16>(p[1][0], p[1][1]);
 #pragma unroll
             for (int hb = 0; hb < NHB; ++hb) {
                 // interleave two V rows: word w of a row holds dims 2w, 2w+1 -> (row_a[d], row_b[d]) pairs
@@ -326,7 +341,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 }
                 // MMA t: row g = dim hb*64 + g*8 + t, row g+8 = dim hb*64 + g*8 + 4 + t
 #pragma unroll
-                for (int t = 0; t < 4; ++t) mma16816(acc[hb][t], ab[t], ab[4 + t], cd[t], cd[4 + t], pb0, pb1);
+                for (int t = 0; t < 4; ++t) mma16816<F16>(acc[hb][t], ab[t], ab[4 + t], cd[t], cd[4 + t], pb0, pb1);
             }
         }
 
@@ -366,10 +381,10 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 
 // grid = B * Hq, block = D threads: merges the num_splits partials of one (batch, head).  The
 // partials are read in groups of 16 with all loads of a group in flight together.
-template <int D>
+template <int D, bool F16>
 __global__ void __launch_bounds__(D)
 decode_combine_kernel(const float* __restrict__ ws_o, const float* __restrict__ ws_ml,
-                      __nv_bfloat16* __restrict__ out, int num_splits) {
+                      uint16_t* __restrict__ out, int num_splits) {
     const size_t bh = blockIdx.x;
     const int d = threadIdx.x;
     const float2* ml = reinterpret_cast<const float2*>(ws_ml) + bh * num_splits;
@@ -404,10 +419,12 @@ decode_combine_kernel(const float* __restrict__ ws_o, const float* __restrict__ 
         }
         M = Mg;
     }
-    out[bh * D + d] = __float2bfloat16_rn(L > 0.f ? O / L : 0.f);
+    const float res = L > 0.f ? O / L : 0.f;
+    if constexpr (F16) out[bh * D + d] = __half_as_ushort(__float2half_rn(res));
+    else out[bh * D + d] = __bfloat16_as_ushort(__float2bfloat16_rn(res));
 }
 
-template <int D, int G>
+template <int D, int G, bool F16>
 int launch_split(const void* q, const void* kc, const void* vc, const int32_t* lens, float* ws_o, float* ws_ml,
                  int B, int Hq, int Hkv, int Smax, int num_splits, float scale_log2, cudaStream_t s) {
     constexpr int kSmem = kWarps * kWarpRingBytes + 1024;
@@ -421,26 +438,26 @@ int launch_split(const void* q, const void* kc, const void* vc, const int32_t* l
         if (!encode_tmap_bf16_sw128(&tk, kc, 3, dims, strides, box)) return FORGE_ERR_CUDA;
         if (!encode_tmap_bf16_sw128(&tv, vc, 3, dims, strides, box)) return FORGE_ERR_CUDA;
     }
-    auto kernel = decode_split_kernel<D, G>;
+    auto kernel = decode_split_kernel<D, G, F16>;
     FORGE_SET_SMEM_ONCE(kernel, kSmem);
     const int sms = sm_count();
     if (sms <= 0) return FORGE_ERR_CUDA;
     const long long items = (long long)B * Hkv * num_splits;
     const long long ctas = (items + kWarps - 1) / kWarps;
     const int grid = ctas < sms ? (int)ctas : sms;
-    FORGE_CUDA_TRY(launch_pdl(kernel, dim3(grid), dim3(kThreads), kSmem, s, tk, tv, static_cast<const __nv_bfloat16*>(q),
+    FORGE_CUDA_TRY(launch_pdl(kernel, dim3(grid), dim3(kThreads), kSmem, s, tk, tv, static_cast<const uint16_t*>(q),
                               lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, status));
     return FORGE_OK;
 }
 
-template <int D>
+template <int D, bool F16>
 int dispatch_g(int G, const void* q, const void* kc, const void* vc, const int32_t* lens, float* ws_o,
                float* ws_ml, int B, int Hq, int Hkv, int Smax, int num_splits, float scale_log2, cudaStream_t s) {
     switch (G) {
-        case 1: return launch_split<D, 1>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
-        case 2: return launch_split<D, 2>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
-        case 4: return launch_split<D, 4>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
-        case 8: return launch_split<D, 8>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
+        case 1: return launch_split<D, 1, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
+        case 2: return launch_split<D, 2, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
+        case 4: return launch_split<D, 4, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
+        case 8: return launch_split<D, 8, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
         default: return FORGE_ERR_UNSUPPORTED;
     }
 }
@@ -454,11 +471,14 @@ extern "C" size_t forge_attn_decode_workspace_bytes(int B, int Hq, int D, int nu
     return (slots * (size_t)(D + 2) * sizeof(float) + 15) & ~(size_t)15;
 }
 
-extern "C" int forge_attn_decode_splitkv(const void* q, const void* k_cache, const void* v_cache, void* out,
-                                         int B, int Hq, int Hkv, int Smax, int D,
-                                         const int32_t* lens, int num_splits, float scale,
-                                         void* workspace, size_t workspace_bytes, void* stream) {
-    using namespace forge;
+namespace forge {
+namespace {
+
+template <bool F16>
+int decode_splitkv_impl(const void* q, const void* k_cache, const void* v_cache, void* out,
+                        int B, int Hq, int Hkv, int Smax, int D,
+                        const int32_t* lens, int num_splits, float scale,
+                        void* workspace, size_t workspace_bytes, void* stream) {
     if (!lens) return FORGE_ERR_INVALID_ARG;
     int st = check_attn_args(q, k_cache, v_cache, out, B, Hq, Hkv, 1, Smax, D, FORGE_MASK_PADDING, lens);
     if (st != FORGE_OK) return st;
@@ -473,8 +493,8 @@ extern "C" int forge_attn_decode_splitkv(const void* q, const void* k_cache, con
     const float scale_log2 = scale * 1.4426950408889634f;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int G = Hq / Hkv;
-    st = (D == 64) ? dispatch_g<64>(G, q, k_cache, v_cache, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s)
-                   : dispatch_g<128>(G, q, k_cache, v_cache, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
+    st = (D == 64) ? dispatch_g<64, F16>(G, q, k_cache, v_cache, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s)
+                   : dispatch_g<128, F16>(G, q, k_cache, v_cache, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
     if (st != FORGE_OK) return st;
     st = finish_launch(1);
     if (st != FORGE_OK) return st;
@@ -482,12 +502,31 @@ extern "C" int forge_attn_decode_splitkv(const void* q, const void* k_cache, con
     // while the split kernel drains, and block in griddepcontrol.wait until that grid has completed.
     const float* cws_o = ws_o;
     const float* cws_ml = ws_ml;
-    __nv_bfloat16* ob = static_cast<__nv_bfloat16*>(out);
+    uint16_t* ob = static_cast<uint16_t*>(out);
     if (D == 64)
-        FORGE_CUDA_TRY(launch_pdl(decode_combine_kernel<64>, dim3(B * Hq), dim3(64), 0, s, cws_o, cws_ml, ob, num_splits));
+        FORGE_CUDA_TRY(launch_pdl(decode_combine_kernel<64, F16>, dim3(B * Hq), dim3(64), 0, s, cws_o, cws_ml, ob, num_splits));
     else
-        FORGE_CUDA_TRY(launch_pdl(decode_combine_kernel<128>, dim3(B * Hq), dim3(128), 0, s, cws_o, cws_ml, ob, num_splits));
+        FORGE_CUDA_TRY(launch_pdl(decode_combine_kernel<128, F16>, dim3(B * Hq), dim3(128), 0, s, cws_o, cws_ml, ob, num_splits));
     return finish_launch(1);
+}
+
+}  // namespace
+}  // namespace forge
+
+extern "C" int forge_attn_decode_splitkv(const void* q, const void* k_cache, const void* v_cache, void* out,
+                                         int B, int Hq, int Hkv, int Smax, int D,
+                                         const int32_t* lens, int num_splits, float scale,
+                                         void* workspace, size_t workspace_bytes, void* stream) {
+    return forge::decode_splitkv_impl<false>(q, k_cache, v_cache, out, B, Hq, Hkv, Smax, D, lens, num_splits, scale,
+                                             workspace, workspace_bytes, stream);
+}
+
+extern "C" int forge_attn_decode_splitkv_f16(const void* q, const void* k_cache, const void* v_cache, void* out,
+                                             int B, int Hq, int Hkv, int Smax, int D,
+                                             const int32_t* lens, int num_splits, float scale,
+                                             void* workspace, size_t workspace_bytes, void* stream) {
+    return forge::decode_splitkv_impl<true>(q, k_cache, v_cache, out, B, Hq, Hkv, Smax, D, lens, num_splits, scale,
+                                            workspace, workspace_bytes, stream);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -14,6 +14,7 @@
 // up product in the second (the B operand of a stage is the gate tile followed by the up tile, one MMA
 // of N = 256 per k-step), and the epilogue multiplies the two halves as it reads them back.
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include "forge_common.cuh"
 #include "sm100_ptx.cuh"
@@ -64,20 +65,32 @@ __device__ __forceinline__ float activate(float z) {
     return z;
 }
 
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
-    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t*>(&v);
+// 16-bit element helpers: bf16 (F16 = false) or fp16 (F16 = true)
+template <bool F16>
+__device__ __forceinline__ uint32_t pack16(float lo, float hi) {
+    if constexpr (F16) {
+        __half2 v = __floats2half2_rn(lo, hi);
+        return *reinterpret_cast<uint32_t*>(&v);
+    } else {
+        __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+        return *reinterpret_cast<uint32_t*>(&v);
+    }
+}
+template <bool F16>
+__device__ __forceinline__ float widen16(uint16_t bits) {
+    if constexpr (F16) return __half2float(__ushort_as_half(bits));
+    else return __uint_as_float(static_cast<uint32_t>(bits) << 16);
 }
 
 // ACT: activation; W_NK: W is stored [N, K] (K-major B operand) instead of [K, N] (MN-major B operand).
 // GATED: two weight matrices (tmap_w = gate, tmap_w2 = up), output silu(gate) * up, BN / 2 output columns per tile.
 // bias and residual may be null.
-template <int BN, int STAGES, int ACT, bool W_NK, bool GATED>
+template <int BN, int STAGES, int ACT, bool W_NK, bool GATED, bool F16>
 __global__ void __launch_bounds__(kThreads, 1)
 linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                         const __grid_constant__ CUtensorMap tmap_w2,
-                        const __grid_constant__ CUtensorMap tmap_y, const __nv_bfloat16* __restrict__ bias,
-                        const __nv_bfloat16* __restrict__ residual, int M, int N, int K, int* __restrict__ status) {
+                        const __grid_constant__ CUtensorMap tmap_y, const uint16_t* __restrict__ bias,
+                        const uint16_t* __restrict__ residual, int M, int N, int K, int* __restrict__ status) {
     using L = LinearSmem<BN, STAGES>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -148,7 +161,8 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
         }
     } else if (warp == 1) {
         if (elect_one()) {
-            constexpr uint32_t idesc = make_idesc_bf16(kBM, BN, /*a_mn_major=*/false, /*b_mn_major=*/!W_NK);
+            constexpr uint32_t idesc = F16 ? make_idesc_f16(kBM, BN, /*a_mn_major=*/false, /*b_mn_major=*/!W_NK)
+                                           : make_idesc_bf16(kBM, BN, /*a_mn_major=*/false, /*b_mn_major=*/!W_NK);
             int stage = 0;
             uint32_t phase = 0;
             int it = 0;
@@ -192,7 +206,7 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
             const uint32_t acc_phase = (it >> 1) & 1;
             float* bias_s = s_bias + acc * BN;
             for (int i = etid; i < BNO; i += kEpiThreads)
-                bias_s[i] = (bias != nullptr && n0 + i < N) ? __bfloat162float(bias[n0 + i]) : 0.f;
+                bias_s[i] = (bias != nullptr && n0 + i < N) ? widen16<F16>(bias[n0 + i]) : 0.f;
             asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
             // A warp that gave up keeps taking part in the named barrier above (so the others never
             // wait for it there) but skips the work.
@@ -234,8 +248,8 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
                         const int col = c * 8 + 2 * i;
                         const float z0 = __uint_as_float(r[col]) + bias_s[blk * 64 + chalf * 32 + col];
                         const float z1 = __uint_as_float(r[col + 1]) + bias_s[blk * 64 + chalf * 32 + col + 1];
-                        w[i] = pack_bf16(activate<GATED ? FORGE_ACT_NONE : ACT>(z0) + __uint_as_float(rw[i] << 16),
-                                         activate<GATED ? FORGE_ACT_NONE : ACT>(z1) + __uint_as_float(rw[i] & 0xffff0000u));
+                        w[i] = pack16<F16>(activate<GATED ? FORGE_ACT_NONE : ACT>(z0) + widen16<F16>(static_cast<uint16_t>(rw[i] & 0xffffu)),
+                                           activate<GATED ? FORGE_ACT_NONE : ACT>(z1) + widen16<F16>(static_cast<uint16_t>(rw[i] >> 16)));
                     }
                     *reinterpret_cast<uint4*>(stage_out + row * 128 + (((chalf * 4 + c) ^ (row & 7)) << 4)) =
                         make_uint4(w[0], w[1], w[2], w[3]);
@@ -268,7 +282,7 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
     }
 }
 
-template <int BN, int STAGES, int ACT, bool W_NK, bool GATED = false>
+template <int BN, int STAGES, int ACT, bool W_NK, bool GATED = false, bool F16 = false>
 int launch_linear(const void* x, const void* w, const void* b, const void* residual, void* y, int M, int N, int K,
                   cudaStream_t s, const void* w_up = nullptr) {
     using L = LinearSmem<BN, STAGES>;
@@ -303,29 +317,26 @@ int launch_linear(const void* x, const void* w, const void* b, const void* resid
     if (!status) return FORGE_ERR_CUDA;
     const int sms = sm_count();
     if (sms <= 0) return FORGE_ERR_CUDA;
-    auto kernel = linear_bias_gelu_kernel<BN, STAGES, ACT, W_NK, GATED>;
+    auto kernel = linear_bias_gelu_kernel<BN, STAGES, ACT, W_NK, GATED, F16>;
     FORGE_SET_SMEM_ONCE(kernel, L::kAlloc);
     const int tiles = ((M + kBM - 1) / kBM) * ((N + BNO - 1) / BNO);
     const int grid = tiles < sms ? tiles : sms;
     FORGE_CUDA_TRY(launch_pdl(kernel, dim3(grid), dim3(kThreads), L::kAlloc, s, tmap_x, tmap_w, tmap_w2, tmap_y,
-                              static_cast<const __nv_bfloat16*>(b), static_cast<const __nv_bfloat16*>(residual),
+                              static_cast<const uint16_t*>(b), static_cast<const uint16_t*>(residual),
                               M, N, K, status));
     return finish_launch(1);
 }
 
-template <int ACT>
+template <int ACT, bool F16>
 int launch_layout(int w_layout, const void* x, const void* w, const void* b, const void* r, void* y, int M, int N,
                   int K, cudaStream_t s) {
-    return w_layout == FORGE_W_NK ? launch_linear<192, 4, ACT, true>(x, w, b, r, y, M, N, K, s)
-                                  : launch_linear<192, 4, ACT, false>(x, w, b, r, y, M, N, K, s);
+    return w_layout == FORGE_W_NK ? launch_linear<192, 4, ACT, true, false, F16>(x, w, b, r, y, M, N, K, s)
+                                  : launch_linear<192, 4, ACT, false, false, F16>(x, w, b, r, y, M, N, K, s);
 }
 
-}  // namespace
-}  // namespace forge
-
-extern "C" int forge_linear_act(const void* x, const void* w, const void* b, const void* residual, void* y,
-                                int M, int N, int K, int act, int w_layout, void* stream) {
-    using namespace forge;
+template <bool F16>
+int linear_act_impl(const void* x, const void* w, const void* b, const void* residual, void* y,
+                    int M, int N, int K, int act, int w_layout, void* stream) {
     if (!x || !w || !y) return FORGE_ERR_INVALID_ARG;
     if (M <= 0 || N <= 0 || K <= 0) return FORGE_ERR_INVALID_ARG;
     if (act < FORGE_ACT_GELU_TANH || act > FORGE_ACT_NONE) return FORGE_ERR_INVALID_ARG;
@@ -335,12 +346,25 @@ extern "C" int forge_linear_act(const void* x, const void* w, const void* b, con
     if ((K % 8) != 0 || (N % 8) != 0) return FORGE_ERR_UNSUPPORTED;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     switch (act) {
-        case FORGE_ACT_GELU_TANH: return launch_layout<FORGE_ACT_GELU_TANH>(w_layout, x, w, b, residual, y, M, N, K, s);
-        case FORGE_ACT_GELU_ERF: return launch_layout<FORGE_ACT_GELU_ERF>(w_layout, x, w, b, residual, y, M, N, K, s);
-        case FORGE_ACT_RELU: return launch_layout<FORGE_ACT_RELU>(w_layout, x, w, b, residual, y, M, N, K, s);
-        case FORGE_ACT_SILU: return launch_layout<FORGE_ACT_SILU>(w_layout, x, w, b, residual, y, M, N, K, s);
-        default: return launch_layout<FORGE_ACT_NONE>(w_layout, x, w, b, residual, y, M, N, K, s);
+        case FORGE_ACT_GELU_TANH: return launch_layout<FORGE_ACT_GELU_TANH, F16>(w_layout, x, w, b, residual, y, M, N, K, s);
+        case FORGE_ACT_GELU_ERF: return launch_layout<FORGE_ACT_GELU_ERF, F16>(w_layout, x, w, b, residual, y, M, N, K, s);
+        case FORGE_ACT_RELU: return launch_layout<FORGE_ACT_RELU, F16>(w_layout, x, w, b, residual, y, M, N, K, s);
+        case FORGE_ACT_SILU: return launch_layout<FORGE_ACT_SILU, F16>(w_layout, x, w, b, residual, y, M, N, K, s);
+        default: return launch_layout<FORGE_ACT_NONE, F16>(w_layout, x, w, b, residual, y, M, N, K, s);
     }
+}
+
+}  // namespace
+}  // namespace forge
+
+extern "C" int forge_linear_act(const void* x, const void* w, const void* b, const void* residual, void* y,
+                                int M, int N, int K, int act, int w_layout, void* stream) {
+    return forge::linear_act_impl<false>(x, w, b, residual, y, M, N, K, act, w_layout, stream);
+}
+
+extern "C" int forge_linear_act_f16(const void* x, const void* w, const void* b, const void* residual, void* y,
+                                    int M, int N, int K, int act, int w_layout, void* stream) {
+    return forge::linear_act_impl<true>(x, w, b, residual, y, M, N, K, act, w_layout, stream);
 }
 
 extern "C" int forge_linear_bias_gelu(const void* x, const void* w, const void* b, void* y,

@@ -205,18 +205,18 @@ def attention_workload(name, config, B, Hq, Hkv, Sq, Skv, D, mask_kind, scale, d
     return AttentionWorkload(name, B, Hq, Hkv, Sq, Skv, D, mask_kind, scale, dtype, q, k, v, lens)
 
 
-def decode_workload(name, config, B, Hq, Hkv, Smax, D, num_splits, scale, lens_range) -> DecodeWorkload:
-    q = normal_tensor(seed_for(config, "q"), (B, Hq, D), "bf16")
-    k = normal_tensor(seed_for(config, "k"), (B, Hkv, Smax, D), "bf16")
-    v = normal_tensor(seed_for(config, "v"), (B, Hkv, Smax, D), "bf16")
+def decode_workload(name, config, B, Hq, Hkv, Smax, D, num_splits, scale, lens_range, dtype="bf16") -> DecodeWorkload:
+    q = normal_tensor(seed_for(config, "q"), (B, Hq, D), dtype)
+    k = normal_tensor(seed_for(config, "k"), (B, Hkv, Smax, D), dtype)
+    v = normal_tensor(seed_for(config, "v"), (B, Hkv, Smax, D), dtype)
     lens = uniform_int(seed_for(config, "lens"), B, lens_range[0], lens_range[1])
     return DecodeWorkload(name, B, Hq, Hkv, Smax, D, num_splits, scale, q, k, v, lens)
 
 
-def linear_workload(name, config, M, N, K, w_std=0.02, b_std=0.02) -> LinearWorkload:
-    x = normal_tensor(seed_for(config, "x"), (M, K), "bf16")
-    w = normal_tensor(seed_for(config, "w"), (K, N), "bf16", std=w_std)
-    b = normal_tensor(seed_for(config, "b"), (N,), "bf16", std=b_std)
+def linear_workload(name, config, M, N, K, w_std=0.02, b_std=0.02, dtype="bf16") -> LinearWorkload:
+    x = normal_tensor(seed_for(config, "x"), (M, K), dtype)
+    w = normal_tensor(seed_for(config, "w"), (K, N), dtype, std=w_std)
+    b = normal_tensor(seed_for(config, "b"), (N,), dtype, std=b_std)
     return LinearWorkload(name, M, N, K, x, w, b)
 
 

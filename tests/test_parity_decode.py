@@ -37,6 +37,12 @@ def test_head_dims_and_group_sizes(D, Hq, Hkv):
     _run(w)
 
 
+def test_batch_larger_than_the_length_ranking_limit():
+    """More than 64 sequences: the kernel deals the items in batch order instead of by cached length."""
+    w = wl.decode_workload("t", 25, 80, 4, 2, 160, 64, 3, 0.125, (1, 160))
+    _run(w)
+
+
 def test_short_and_degenerate_lengths():
     """Fewer rows than splits (empty splits), one row, zero rows, and lens beyond Smax (clamped)."""
     w = wl.decode_workload("t", 23, 5, 8, 2, 64, 128, 16, 0.1, (1, 64))

@@ -117,7 +117,7 @@ int forge_attn_fused_f32(const void* q, const void* k, const void* v, void* out,
  * workspace: at least forge_attn_decode_workspace_bytes(...) bytes, 16-byte
  * aligned, contents need no initialisation and are overwritten.  Two calls that
  * may overlap on the GPU must not share a workspace.
- * 1 <= num_splits <= 64; D must be 64 or 128; Hq / Hkv must be 1, 2, 4 or 8.
+ * 1 <= num_splits <= 64; D must be 64 or 128; Hq / Hkv must be between 1 and 8.
  */
 int forge_attn_decode_splitkv(const void* q, const void* k_cache, const void* v_cache, void* out,
                               int B, int Hq, int Hkv, int Smax, int D,

@@ -456,7 +456,11 @@ int dispatch_g(int G, const void* q, const void* kc, const void* vc, const int32
     switch (G) {
         case 1: return launch_split<D, 1, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
         case 2: return launch_split<D, 2, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
+        case 3: return launch_split<D, 3, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
         case 4: return launch_split<D, 4, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
+        case 5: return launch_split<D, 5, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
+        case 6: return launch_split<D, 6, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
+        case 7: return launch_split<D, 7, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
         case 8: return launch_split<D, 8, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
         default: return FORGE_ERR_UNSUPPORTED;
     }

@@ -31,7 +31,8 @@ def test_result_does_not_depend_on_num_splits(num_splits):
     _run(w, num_splits)
 
 
-@pytest.mark.parametrize("D,Hq,Hkv", [(64, 12, 12), (64, 8, 4), (128, 8, 1), (128, 32, 8), (64, 16, 2)])
+@pytest.mark.parametrize("D,Hq,Hkv", [(64, 12, 12), (64, 8, 4), (128, 8, 1), (128, 32, 8), (64, 16, 2),
+                                       (128, 28, 4), (64, 6, 2), (128, 10, 2), (64, 12, 2)])
 def test_head_dims_and_group_sizes(D, Hq, Hkv):
     w = wl.decode_workload("t", 22, 3, Hq, Hkv, 333, D, 5, 1.0 / np.sqrt(D), (1, 333))
     _run(w)

@@ -88,7 +88,7 @@ def test_decode_argument_validation(lib):
     assert call(splits=65) == binding.ERR_UNSUPPORTED
     assert call(ws=None) == binding.ERR_INVALID_ARG
     assert call(wsb=need - 1) == binding.ERR_WORKSPACE
-    assert call(Hq=18, Hkv=2) == binding.ERR_UNSUPPORTED   # group size 9
+    assert call(Hq=18, Hkv=2, wsb=1 << 30) == binding.ERR_UNSUPPORTED   # group size 9
     assert call(D=96) == binding.ERR_UNSUPPORTED
 
 

@@ -194,6 +194,17 @@ int forge_linear_act_f16(const void* x, const void* w, const void* b, const void
                          int M, int N, int K, int act, int w_layout, void* stream);
 
 /*
+ * Weight-only int8 linear, the W-int8 / A-fp16 setting of the evaluation's largest model (Section 5.1):
+ * symmetric per-output-channel quantisation, W(k,n) = scale[n] * w_int8[n,k]:
+ *     y[m,n] = act(scale[n] * sum_k x[m,k] * w_int8[n,k] + b[n]) + residual[m,n]
+ * x [M,K], b [N], residual [M,N], y [M,N] fp16; w_int8 [N,K] int8; scale [N] fp32; b and residual may be
+ * NULL; act as in forge_linear_act.  The weights are widened to fp16 inside the kernel (exactly) and fed to
+ * the tensor core; the scale is applied to the fp32 accumulator.  K must be a multiple of 16, N of 8.
+ */
+int forge_linear_act_w8a16(const void* x, const void* w_int8, const float* scale, const void* b,
+                           const void* residual, void* y, int M, int N, int K, int act, void* stream);
+
+/*
  * Gated MLP input of the 1B-8B decoder models of the evaluation (SwiGLU; Section 2, model overview): the
  * linear+silu pattern of the operator-fusion pass and the element-wise product with the second
  * projection, in one kernel:

@@ -11,6 +11,7 @@ from .ref import (  # noqa: F401
     linear_bias_gelu,
     linear_act,
     linear_swiglu,
+    linear_w8,
     ACT_GELU_TANH,
     ACT_GELU_ERF,
     ACT_RELU,

@@ -280,3 +280,37 @@ int forge_ref_linear_swiglu(const double *x, const double *wg, const double *wu,
     }
     return 0;
 }
+
+/*
+ * Weight-only int8 linear (the W-int8 / A-fp16 setting of the evaluation's largest model): symmetric
+ * per-output-channel quantisation, w(k, n) = scale[n] * wq[n, k] with wq integers in [-128, 127]:
+ *     y[m, n] = act(scale[n] * sum_k x[m, k] wq[n, k] + b[n]) + r[m, n]
+ * wq is stored [N, K] (given here as doubles holding the integers); b and r may be NULL; act as in
+ * forge_ref_linear_act.
+ */
+int forge_ref_linear_w8(const double *x, const double *wq, const double *scale, const double *b, const double *r,
+                        double *y, int M, int N, int K, int act)
+{
+    if (!x || !wq || !scale || !y || M <= 0 || N <= 0 || K <= 0) return 1;
+    if (act < 0 || act > 4) return 1;
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        for (int n = 0; n < N; ++n) {
+            double z = 0.0;
+            for (int kk = 0; kk < K; ++kk) z += x[(size_t)m * K + kk] * wq[(size_t)n * K + kk];
+            z *= scale[n];
+            if (b) z += b[n];
+            double a;
+            switch (act) {
+            case 0: a = forge_ref_gelu_tanh(z); break;
+            case 1: a = 0.5 * z * (1.0 + erf(z / sqrt(2.0))); break;
+            case 2: a = z > 0.0 ? z : 0.0; break;
+            case 3: a = z / (1.0 + exp(-z)); break;
+            default: a = z; break;
+            }
+            if (r) a += r[(size_t)m * N + n];
+            y[(size_t)m * N + n] = a;
+        }
+    }
+    return 0;
+}

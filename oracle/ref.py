@@ -38,6 +38,7 @@ def _configure(lib):
     lib.forge_ref_attn_decode.argtypes = [_dp, _dp, _dp, _dp, i, i, i, i, i, _ip, ctypes.c_double]
     lib.forge_ref_linear_bias_gelu.argtypes = [_dp, _dp, _dp, _dp, i, i, i]
     lib.forge_ref_linear_act.argtypes = [_dp, _dp, _dp, _dp, _dp, i, i, i, i, i]
+    lib.forge_ref_linear_w8.argtypes = [_dp, _dp, _dp, _dp, _dp, _dp, i, i, i, i]
     lib.forge_ref_linear_swiglu.argtypes = [_dp, _dp, _dp, _dp, i, i, i, i]
     lib.forge_ref_gelu_tanh.argtypes = [ctypes.c_double]
     lib.forge_ref_gelu_tanh.restype = ctypes.c_double
@@ -161,6 +162,22 @@ def linear_act(x, w, b=None, residual=None, act=ACT_GELU_TANH, w_layout=0):
     _check(_load().forge_ref_linear_act(_ptr(x), _ptr(w), None if b is None else _ptr(b),
                                         None if residual is None else _ptr(residual), _ptr(y), M, N, K,
                                         int(act), int(w_layout)), "forge_ref_linear_act")
+    return y
+
+
+def linear_w8(x, wq, scale, b=None, residual=None, act=ACT_GELU_TANH):
+    """act(scale[n] * (x Wq^T)[m,n] + b) + residual; Wq [N,K] holds integers in [-128, 127]."""
+    x, wq, scale = _f64(x), _f64(wq), _f64(scale)
+    M, K = x.shape
+    N = wq.shape[0]
+    assert wq.shape == (N, K) and scale.shape == (N,)
+    assert np.all(wq == np.round(wq)) and wq.min() >= -128 and wq.max() <= 127
+    b = None if b is None else _f64(b)
+    residual = None if residual is None else _f64(residual)
+    y = np.empty((M, N), dtype=np.float64)
+    _check(_load().forge_ref_linear_w8(_ptr(x), _ptr(wq), _ptr(scale), None if b is None else _ptr(b),
+                                       None if residual is None else _ptr(residual), _ptr(y), M, N, K, int(act)),
+           "forge_ref_linear_w8")
     return y
 
 

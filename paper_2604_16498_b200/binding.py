@@ -34,6 +34,7 @@ SIGNATURES = {
     "forge_linear_bias_gelu": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
     "forge_linear_act": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]),
     "forge_linear_act_f16": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]),
+    "forge_linear_act_w8a16": (_i, [_vp, _vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp]),
     "forge_linear_swiglu": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _vp]),
     "forge_attn_host_scratch_bytes": (_sz, [_i, _i, _i, _i, _i, _i, _i]),
     "forge_attn_fused_host": (_i, _ATTN + [_vp, _sz, _vp]),
@@ -237,6 +238,21 @@ def linear_act(x, w, b=None, residual=None, act=ACT_GELU_TANH, w_layout=W_KN, ou
         _dev(x, bf, "x"), _dev(w, bf, "w"), None if b is None else _dev(b, bf, "b"),
         None if residual is None else _dev(residual, bf, "residual"), _dev(out, bf, "out"),
         M, N, K, int(act), int(w_layout), _stream()))
+    return out
+
+
+def linear_act_w8a16(x, w_int8, scale, b=None, residual=None, act=ACT_GELU_TANH, out=None):
+    """forge_linear_act_w8a16: fp16 x [M,K], int8 weights [N,K], fp32 per-channel scale [N]."""
+    M, K = x.shape
+    N = w_int8.shape[0]
+    if tuple(w_int8.shape) != (N, K) or tuple(scale.shape) != (N,):
+        raise ValueError("w_int8 [N,K] and scale [N] expected")
+    out = torch.empty((M, N), dtype=torch.float16, device=x.device) if out is None else out
+    h = torch.float16
+    _check("forge_linear_act_w8a16", load().forge_linear_act_w8a16(
+        _dev(x, h, "x"), _dev(w_int8, torch.int8, "w_int8"), _dev(scale, torch.float32, "scale"),
+        None if b is None else _dev(b, h, "b"), None if residual is None else _dev(residual, h, "residual"),
+        _dev(out, h, "out"), M, N, K, int(act), _stream()))
     return out
 
 

@@ -13,6 +13,11 @@
 // 128 output columns; its accumulator is 256 columns wide, the gate product in the first half and the
 // up product in the second (the B operand of a stage is the gate tile followed by the up tile, one MMA
 // of N = 256 per k-step), and the epilogue multiplies the two halves as it reads them back.
+// Weight-only int8 form (W8: fp16 activations, int8 weights [N,K] with one fp32 scale per output
+// channel, the W-int8/A-fp16 setting of the paper's largest model): the int8 tile of a stage arrives by
+// TMA next to the operand stage, eight extra warps (10-17) turn it into the swizzled fp16 B operand
+// (exact: 1024 + (w ^ 0x80) as fp16 bits, minus 1152), and the scale is applied to the accumulator in
+// the epilogue, where it factors out of the sum over K.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -29,20 +34,24 @@ constexpr int kBM = 128;
 constexpr int kBK = 64;
 constexpr int kThreads = 320;
 constexpr int kEpiThreads = 256;
+constexpr int kCvtWarps = 8;      // int8 -> fp16 converter warps of the W8 form
+constexpr int kThreadsW8 = kThreads + kCvtWarps * 32;
 constexpr int kAccStride = 256;   // TMEM columns between the two accumulators
 constexpr int kTmemCols = 512;
 
-template <int BN, int STAGES>
+template <int BN, int STAGES, bool W8 = false>
 struct LinearSmem {
     static constexpr int kABytes = kBM * kBK * 2;        // 16 KB
     static constexpr int kBBytes = kBK * BN * 2;         // 64 rows of K x BN
-    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kRawBytes = W8 ? BN * kBK : 0;  // BN rows of 64 int8 weights
+    static constexpr int kStageBytes = kABytes + kBBytes + kRawBytes;
     static constexpr int kOutBytes = kBM * 128;          // output staging: 128 rows x 64 bf16, two buffers
     static constexpr int kOutOffset = STAGES * kStageBytes;
     static constexpr int kBarOffset = kOutOffset + 2 * kOutBytes;
-    // barriers: full[S], empty[S], tmem_full[2], tmem_empty[2]; then the TMEM base, then bias[2][BN]
-    static constexpr int kBiasOffset = kBarOffset + (2 * STAGES + 4) * 8 + 16;
-    static constexpr int kTotal = kBiasOffset + 2 * BN * 4;
+    // barriers: full[S], empty[S], tmem_full[2], tmem_empty[2], raw_full[S]; then the TMEM base, then
+    // bias[2][BN] and scale[2][BN]
+    static constexpr int kBiasOffset = kBarOffset + (3 * STAGES + 4) * 8 + 16;
+    static constexpr int kTotal = kBiasOffset + 4 * BN * 4;
     static constexpr int kAlloc = kTotal + 1024;         // slack to align the base to 1024 bytes
 };
 
@@ -85,21 +94,26 @@ __device__ __forceinline__ float widen16(uint16_t bits) {
 // ACT: activation; W_NK: W is stored [N, K] (K-major B operand) instead of [K, N] (MN-major B operand).
 // GATED: two weight matrices (tmap_w = gate, tmap_w2 = up), output silu(gate) * up, BN / 2 output columns per tile.
 // bias and residual may be null.
-template <int BN, int STAGES, int ACT, bool W_NK, bool GATED, bool F16>
-__global__ void __launch_bounds__(kThreads, 1)
+// W8: tmap_w2 describes the int8 weights [N,K] (plain layout), `scale` their per-channel factors.
+template <int BN, int STAGES, int ACT, bool W_NK, bool GATED, bool F16, bool W8>
+__global__ void __launch_bounds__(W8 ? kThreadsW8 : kThreads, 1)
 linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                         const __grid_constant__ CUtensorMap tmap_w2,
                         const __grid_constant__ CUtensorMap tmap_y, const uint16_t* __restrict__ bias,
-                        const uint16_t* __restrict__ residual, int M, int N, int K, int* __restrict__ status) {
-    using L = LinearSmem<BN, STAGES>;
+                        const uint16_t* __restrict__ residual, const float* __restrict__ scale, int M, int N, int K,
+                        int* __restrict__ status) {
+    static_assert(!W8 || (W_NK && F16 && !GATED), "the int8-weight form takes [N,K] weights and fp16 activations");
+    using L = LinearSmem<BN, STAGES, W8>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::kBarOffset);
     uint64_t* empty = full + STAGES;
     uint64_t* tmem_full = empty + STAGES;
     uint64_t* tmem_empty = tmem_full + 2;
-    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(tmem_empty + 2);
+    uint64_t* raw_full = tmem_empty + 2;  // W8: the stage's int8 tile has landed
+    uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(raw_full + STAGES);
     float* s_bias = reinterpret_cast<float*>(smem + L::kBiasOffset);
+    float* s_scale = s_bias + 2 * BN;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr int BNO = GATED ? BN / 2 : BN;  // output columns per tile
@@ -108,7 +122,10 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
     const int kblocks = (K + kBK - 1) / kBK;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < STAGES; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
+        // W8: a stage is complete when X has landed and the converter warps have written the B operand
+        for (int i = 0; i < STAGES; ++i) {
+            mbar_init(&full[i], W8 ? 1 + kCvtWarps : 1); mbar_init(&empty[i], 1); mbar_init(&raw_full[i], 1);
+        }
         for (int i = 0; i < 2; ++i) { mbar_init(&tmem_full[i], 1); mbar_init(&tmem_empty[i], kEpiThreads / 32); }
         fence_mbar_init();
         prefetch_tmap(&tmap_x);
@@ -140,9 +157,12 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
                     if (!mbar_wait(&empty[stage], phase ^ 1)) { failed = true; break; }
                     uint8_t* sa = smem + stage * L::kStageBytes;
                     uint8_t* sb = sa + L::kABytes;
-                    mbar_expect_tx(&full[stage], L::kStageBytes);
+                    mbar_expect_tx(&full[stage], W8 ? L::kABytes : L::kStageBytes);
                     tma_load_2d(sa, &tmap_x, &full[stage], kb * kBK, m0);
-                    if constexpr (W_NK) {  // BN rows of W, 64 K-elements (one swizzle span) each
+                    if constexpr (W8) {  // BN rows of 64 int8 weights, plain layout, behind the operand stage
+                        mbar_expect_tx(&raw_full[stage], L::kRawBytes);
+                        tma_load_2d(sb + L::kBBytes, &tmap_w2, &raw_full[stage], kb * kBK, n0);
+                    } else if constexpr (W_NK) {  // BN rows of W, 64 K-elements (one swizzle span) each
                         tma_load_2d(sb, &tmap_w, &full[stage], kb * kBK, n0);
                         if constexpr (GATED)  // rows BN/2.. of the operand: the up weights of the same columns
                             tma_load_2d(sb + (BN / 2) * 128, &tmap_w2, &full[stage], kb * kBK, n0);
@@ -194,6 +214,45 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
                 mma_commit(&tmem_full[acc]);
             }
         }
+    } else if (W8 && warp >= 10) {
+        // ------------------------------------------------------------------ int8 -> fp16 converters
+        // Thread t of the converter warps takes 16-byte pieces t, t + 256, ... of the stage's int8 tile: piece q holds
+        // weights 16 (q % 4) .. +15 of row q / 4, which become 16-byte chunks 2 (q % 4) and 2 (q % 4) + 1 of
+        // that row's 128-byte line of the K-major, 128-byte-swizzled B operand.
+        const int ctid = (warp - 10) * 32 + lane;
+        int stage = 0;
+        uint32_t phase = 0;
+        for (int tile = blockIdx.x; tile < num_tiles && !failed; tile += gridDim.x) {
+            for (int kb = 0; kb < kblocks; ++kb) {
+                if (!warp_wait(&raw_full[stage], phase)) { failed = true; break; }
+                uint8_t* sb = smem + stage * L::kStageBytes + L::kABytes;
+                const uint8_t* raw = sb + L::kBBytes;
+#pragma unroll
+                for (int i = 0; i < BN * 4 / (kCvtWarps * 32); ++i) {
+                    const int q = i * (kCvtWarps * 32) + ctid, n = q >> 2, part = q & 3;
+                    const uint4 in = *reinterpret_cast<const uint4*>(raw + q * 16);
+                    const uint32_t wds[4] = {in.x ^ 0x80808080u, in.y ^ 0x80808080u, in.z ^ 0x80808080u, in.w ^ 0x80808080u};
+                    uint32_t o[8];
+                    const __half2 off = __floats2half2_rn(1152.f, 1152.f);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        // bytes (u, 0x64) read as fp16 are 1024 + u; u = w + 128
+                        uint32_t lo = __byte_perm(wds[j], 0x64646464u, 0x4140), hi = __byte_perm(wds[j], 0x64646464u, 0x4342);
+                        __half2 hlo = __hsub2(*reinterpret_cast<__half2*>(&lo), off);
+                        __half2 hhi = __hsub2(*reinterpret_cast<__half2*>(&hi), off);
+                        o[2 * j] = *reinterpret_cast<uint32_t*>(&hlo);
+                        o[2 * j + 1] = *reinterpret_cast<uint32_t*>(&hhi);
+                    }
+                    uint8_t* line = sb + n * 128;
+                    *reinterpret_cast<uint4*>(line + (((2 * part) ^ (n & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                    *reinterpret_cast<uint4*>(line + (((2 * part + 1) ^ (n & 7)) << 4)) = make_uint4(o[4], o[5], o[6], o[7]);
+                }
+                fence_proxy_async_smem();  // the tensor core reads what these threads wrote
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&full[stage]);
+                if (++stage == STAGES) { stage = 0; phase ^= 1; }
+            }
+        }
     } else {
         const int quarter = warp & 3;            // TMEM lane quarter this warp may access
         const int etid = (warp - 2) * 32 + lane; // 0..255
@@ -205,8 +264,11 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
             const int acc = it & 1;
             const uint32_t acc_phase = (it >> 1) & 1;
             float* bias_s = s_bias + acc * BN;
-            for (int i = etid; i < BNO; i += kEpiThreads)
+            float* scale_s = s_scale + acc * BN;
+            for (int i = etid; i < BNO; i += kEpiThreads) {
                 bias_s[i] = (bias != nullptr && n0 + i < N) ? widen16<F16>(bias[n0 + i]) : 0.f;
+                if constexpr (W8) scale_s[i] = (n0 + i < N) ? scale[n0 + i] : 0.f;
+            }
             asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
             // A warp that gave up keeps taking part in the named barrier above (so the others never
             // wait for it there) but skips the work.
@@ -246,8 +308,11 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const int col = c * 8 + 2 * i;
-                        const float z0 = __uint_as_float(r[col]) + bias_s[blk * 64 + chalf * 32 + col];
-                        const float z1 = __uint_as_float(r[col + 1]) + bias_s[blk * 64 + chalf * 32 + col + 1];
+                        const int bc = blk * 64 + chalf * 32 + col;
+                        float z0 = __uint_as_float(r[col]), z1 = __uint_as_float(r[col + 1]);
+                        if constexpr (W8) { z0 *= scale_s[bc]; z1 *= scale_s[bc + 1]; }
+                        z0 += bias_s[bc];
+                        z1 += bias_s[bc + 1];
                         w[i] = pack16<F16>(activate<GATED ? FORGE_ACT_NONE : ACT>(z0) + widen16<F16>(static_cast<uint16_t>(rw[i] & 0xffffu)),
                                            activate<GATED ? FORGE_ACT_NONE : ACT>(z1) + widen16<F16>(static_cast<uint16_t>(rw[i] >> 16)));
                     }
@@ -282,10 +347,10 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
     }
 }
 
-template <int BN, int STAGES, int ACT, bool W_NK, bool GATED = false, bool F16 = false>
+template <int BN, int STAGES, int ACT, bool W_NK, bool GATED = false, bool F16 = false, bool W8 = false>
 int launch_linear(const void* x, const void* w, const void* b, const void* residual, void* y, int M, int N, int K,
-                  cudaStream_t s, const void* w_up = nullptr) {
-    using L = LinearSmem<BN, STAGES>;
+                  cudaStream_t s, const void* w_up = nullptr, const float* scale = nullptr) {
+    using L = LinearSmem<BN, STAGES, W8>;
     constexpr int BNO = GATED ? BN / 2 : BN;
     CUtensorMap tmap_x, tmap_w, tmap_w2, tmap_y;
     {
@@ -294,7 +359,13 @@ int launch_linear(const void* x, const void* w, const void* b, const void* resid
         const uint32_t box[2] = {kBK, kBM};
         if (!encode_tmap_bf16_sw128(&tmap_x, x, 2, dims, strides, box)) return FORGE_ERR_CUDA;
     }
-    if (W_NK) {  // w[N, K]: rows of 64 K-elements
+    if (W8) {    // int8 w[N, K]: BN rows of 64 bytes per box, plain layout; no 16-bit weight map is used
+        const uint64_t dims[2] = {(uint64_t)K, (uint64_t)N};
+        const uint64_t strides[1] = {(uint64_t)K};
+        const uint32_t box[2] = {kBK, BNO};
+        if (!encode_tmap_u8_plain(&tmap_w2, w, 2, dims, strides, box)) return FORGE_ERR_CUDA;
+        tmap_w = tmap_w2;
+    } else if (W_NK) {  // w[N, K]: rows of 64 K-elements
         const uint64_t dims[2] = {(uint64_t)K, (uint64_t)N};
         const uint64_t strides[1] = {(uint64_t)K * 2};
         const uint32_t box[2] = {kBK, BNO};
@@ -317,12 +388,12 @@ int launch_linear(const void* x, const void* w, const void* b, const void* resid
     if (!status) return FORGE_ERR_CUDA;
     const int sms = sm_count();
     if (sms <= 0) return FORGE_ERR_CUDA;
-    auto kernel = linear_bias_gelu_kernel<BN, STAGES, ACT, W_NK, GATED, F16>;
+    auto kernel = linear_bias_gelu_kernel<BN, STAGES, ACT, W_NK, GATED, F16, W8>;
     FORGE_SET_SMEM_ONCE(kernel, L::kAlloc);
     const int tiles = ((M + kBM - 1) / kBM) * ((N + BNO - 1) / BNO);
     const int grid = tiles < sms ? tiles : sms;
-    FORGE_CUDA_TRY(launch_pdl(kernel, dim3(grid), dim3(kThreads), L::kAlloc, s, tmap_x, tmap_w, tmap_w2, tmap_y,
-                              static_cast<const uint16_t*>(b), static_cast<const uint16_t*>(residual),
+    FORGE_CUDA_TRY(launch_pdl(kernel, dim3(grid), dim3(W8 ? kThreadsW8 : kThreads), L::kAlloc, s, tmap_x, tmap_w, tmap_w2,
+                              tmap_y, static_cast<const uint16_t*>(b), static_cast<const uint16_t*>(residual), scale,
                               M, N, K, status));
     return finish_launch(1);
 }
@@ -385,4 +456,24 @@ extern "C" int forge_linear_swiglu(const void* x, const void* w_gate, const void
     return w_layout == FORGE_W_NK
                ? launch_linear<256, 3, FORGE_ACT_SILU, true, true>(x, w_gate, nullptr, nullptr, y, M, N, K, s, w_up)
                : launch_linear<256, 3, FORGE_ACT_SILU, false, true>(x, w_gate, nullptr, nullptr, y, M, N, K, s, w_up);
+}
+
+extern "C" int forge_linear_act_w8a16(const void* x, const void* w_int8, const float* scale, const void* b,
+                                      const void* residual, void* y, int M, int N, int K, int act, void* stream) {
+    using namespace forge;
+    if (!x || !w_int8 || !scale || !y) return FORGE_ERR_INVALID_ARG;
+    if (M <= 0 || N <= 0 || K <= 0) return FORGE_ERR_INVALID_ARG;
+    if (act < FORGE_ACT_GELU_TANH || act > FORGE_ACT_NONE) return FORGE_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(w_int8) || !aligned16(y) || (b && !aligned16(b)) || (residual && !aligned16(residual)) ||
+        (reinterpret_cast<uintptr_t>(scale) & 3u))
+        return FORGE_ERR_INVALID_ARG;
+    if ((K % 16) != 0 || (N % 8) != 0) return FORGE_ERR_UNSUPPORTED;  // 16-byte rows of int8 weights and of fp16 outputs
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    switch (act) {
+        case FORGE_ACT_GELU_TANH: return launch_linear<192, 3, FORGE_ACT_GELU_TANH, true, false, true, true>(x, w_int8, b, residual, y, M, N, K, s, nullptr, scale);
+        case FORGE_ACT_GELU_ERF: return launch_linear<192, 3, FORGE_ACT_GELU_ERF, true, false, true, true>(x, w_int8, b, residual, y, M, N, K, s, nullptr, scale);
+        case FORGE_ACT_RELU: return launch_linear<192, 3, FORGE_ACT_RELU, true, false, true, true>(x, w_int8, b, residual, y, M, N, K, s, nullptr, scale);
+        case FORGE_ACT_SILU: return launch_linear<192, 3, FORGE_ACT_SILU, true, false, true, true>(x, w_int8, b, residual, y, M, N, K, s, nullptr, scale);
+        default: return launch_linear<192, 3, FORGE_ACT_NONE, true, false, true, true>(x, w_int8, b, residual, y, M, N, K, s, nullptr, scale);
+    }
 }

@@ -163,3 +163,22 @@ def test_swiglu_against_torch_cpu(w_layout):
     # equals the already pinned linear+silu pattern times a plain matrix product
     np.testing.assert_allclose(oracle.linear_swiglu(x, g, u),
                                oracle.linear_act(x, g, None, None, oracle.ACT_SILU) * (x @ u), atol=1e-13)
+
+
+# ---- weight-only int8: y = act(scale[n] * (x Wq^T) + b) + r
+def test_w8_hand_value_and_reduction_to_the_dense_linear():
+    """One output channel, integers (3, -2), scale 0.5, x = (2, 5): 0.5 * (6 - 10) = -2, plus bias 3 = 1; relu
+    keeps 1, a negative pre-activation gives 0.  And: the quantised linear is the dense one on the
+    dequantised weights (exactly representable here), which is pinned above."""
+    x = np.array([[2.0, 5.0]]); wq = np.array([[3.0, -2.0], [1.0, 1.0]]); sc = np.array([0.5, -1.0])
+    y = oracle.linear_w8(x, wq, sc, np.array([3.0, 0.0]), None, oracle.ACT_RELU)
+    np.testing.assert_array_equal(y, [[1.0, 0.0]])
+    np.testing.assert_array_equal(oracle.linear_w8(x, wq, sc, None, np.array([[10.0, 20.0]]), oracle.ACT_NONE), [[8.0, 13.0]])
+    x = RNG.standard_normal((6, 8)); wq = RNG.integers(-128, 128, size=(5, 8)).astype(np.float64)
+    sc = 2.0 ** RNG.integers(-6, -2, size=5).astype(np.float64)   # powers of two: dequantisation is exact
+    b = RNG.standard_normal(5); r = RNG.standard_normal((6, 5))
+    for act in (oracle.ACT_GELU_TANH, oracle.ACT_SILU, oracle.ACT_NONE):
+        np.testing.assert_allclose(oracle.linear_w8(x, wq, sc, b, r, act),
+                                   oracle.linear_act(x, wq * sc[:, None], b, r, act, 1), atol=1e-13)
+    with pytest.raises(AssertionError):
+        oracle.linear_w8(x, wq + 0.5, sc)

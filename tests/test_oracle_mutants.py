@@ -37,6 +37,10 @@ MUTANTS = {
     "swiglu product dropped": ("gate / (1.0 + exp(-gate)) * up;", "gate / (1.0 + exp(-gate));"),
     "swiglu sigmoid instead of silu": ("gate / (1.0 + exp(-gate)) * up;", "1.0 / (1.0 + exp(-gate)) * up;"),
     "swiglu up weights transposed": ("up += x[(size_t)m * K + kk] * wu[wi];", "up += x[(size_t)m * K + kk] * wu[w_layout == 0 ? (size_t)n * K + kk : (size_t)kk * N + n];"),
+    "w8 scale dropped": ("            z *= scale[n];\n", ""),
+    "w8 scale after the bias": ("            z *= scale[n];\n            if (b) z += b[n];", "            if (b) z += b[n];\n            z *= scale[n];"),
+    "w8 scale indexed by row": ("z *= scale[n];", "z *= scale[m % N];"),
+    "w8 weights read as [K,N]": ("wq[(size_t)n * K + kk]", "wq[(size_t)kk * N + n]"),
     "attention bias dropped": ("        if (bias_row) s += bias_row[j];\n", ""),
     "attention bias scaled": ("        s *= scale;\n        if (bias_row) s += bias_row[j];", "        if (bias_row) s += bias_row[j];\n        s *= scale;"),
     "attention bias subtracted": ("if (bias_row) s += bias_row[j];", "if (bias_row) s -= bias_row[j];"),
@@ -90,6 +94,12 @@ def _pins():
     xs = RNG.standard_normal((4, 5)); gs = RNG.standard_normal((5, 3)); us = RNG.standard_normal((5, 3))
     np.testing.assert_allclose(oracle.linear_swiglu(xs, gs, us),
                                (torch.nn.functional.silu(torch.from_numpy(xs @ gs)) * torch.from_numpy(xs @ us)).numpy(), atol=1e-13)
+    # weight-only int8: hand value, and the dense linear on the dequantised weights (non-square)
+    np.testing.assert_array_equal(oracle.linear_w8(np.array([[2.0, 5.0]]), np.array([[3.0, -2.0], [1.0, 1.0]]),
+                                                   np.array([0.5, -1.0]), np.array([3.0, 0.0]), None, oracle.ACT_RELU), [[1.0, 0.0]])
+    xq = RNG.standard_normal((4, 6)); wq = RNG.integers(-128, 128, size=(3, 6)).astype(np.float64); sq = np.array([0.25, 0.5, 0.125])
+    np.testing.assert_allclose(oracle.linear_w8(xq, wq, sq, np.ones(3), None, oracle.ACT_NONE),
+                               xq @ (wq * sq[:, None]).T + 1.0, atol=1e-13)
     # GELU and linear
     assert abs(oracle.gelu_tanh(1.0) - 0.841192) < 5e-7
     assert abs(oracle.gelu_tanh(3.0) - oracle.gelu_tanh(-3.0) - 3.0) < 1e-14

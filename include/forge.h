@@ -60,7 +60,8 @@ enum {
  * Fused attention, bf16 in / fp32 accumulate / bf16 out:
  *     out[b,h,i,:] = sum_j softmax_j(scale * q[b,h,i,:].k[b,h/G,j,:] over visible j) * v[b,h/G,j,:]
  * (Eq. 9 with the optional scale and mask nodes of Eq. 8 folded in; scores and
- * probabilities never reach global memory).  D must be 64 or 128.  `lens` may be
+ * probabilities never reach global memory).  D: any multiple of 8 up to 128 (sizes other than 64 and
+ * 128 run on the next larger kernel: the TMA unit pads the rows with zeros on the fly).  `lens` may be
  * NULL unless mask_kind has the padding bit.  Tensor-core path (tcgen05, TMEM
  * accumulators, TMA-staged K/V).
  */
@@ -117,7 +118,7 @@ int forge_attn_fused_f32(const void* q, const void* k, const void* v, void* out,
  * workspace: at least forge_attn_decode_workspace_bytes(...) bytes, 16-byte
  * aligned, contents need no initialisation and are overwritten.  Two calls that
  * may overlap on the GPU must not share a workspace.
- * 1 <= num_splits <= 64; D must be 64 or 128; Hq / Hkv must be between 1 and 8.
+ * 1 <= num_splits <= 64; D any multiple of 8 up to 128; Hq / Hkv must be between 1 and 8.
  */
 int forge_attn_decode_splitkv(const void* q, const void* k_cache, const void* v_cache, void* out,
                               int B, int Hq, int Hkv, int Smax, int D,

@@ -157,6 +157,7 @@ struct AttnParams {
     int bias_heads;     // 1 (shared by all heads) or Hq
     float inv_scale;    // 1 / scale: the bias is added to the unscaled scores as bias / scale
     int B, Hq, Hkv, Sq, Skv;
+    int head_dim;  // elements per row in memory (<= the kernel's D; the TMA unit zero-fills the difference)
     int mask_kind;
     float scale_log2;  // > 0 (a zero scale is passed as the smallest normal number: every product flushes to 0)
     FastDiv div_heads;  // by the number of items per query step
@@ -475,9 +476,8 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             const int bh = it.b * p.Hq + pick(it.h, t);
             if (nh == 0) {  // no visible key for any row of this tile (or the tile lies beyond Sq)
                 if (qi < p.Sq) {
-                    uint16_t* orow = p.out + ((size_t)bh * p.Sq + qi) * D;
-#pragma unroll
-                    for (int c = 0; c < D / 8; ++c) reinterpret_cast<uint4*>(orow)[c] = make_uint4(0, 0, 0, 0);
+                    uint16_t* orow = p.out + ((size_t)bh * p.Sq + qi) * p.head_dim;
+                    for (int c = 0; c < p.head_dim / 8; ++c) reinterpret_cast<uint4*>(orow)[c] = make_uint4(0, 0, 0, 0);
                 }
                 if (i_next < num_items) it_next = decode(i_next);
                 it = it_next; i_cur = i_next;
@@ -704,22 +704,24 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     }
 }
 
+// D: the kernel's head dimension (64 or 128); head_dim <= D: the tensors' (a multiple of 8).  Columns beyond
+// head_dim are zero-filled on load and clipped on store by the TMA unit, so a padded head costs time, not memory.
 template <int D, bool F16, bool BIAS = false>
 int launch_attn(const void* q, const void* k, const void* v, void* out, int B, int Hq, int Hkv, int Sq, int Skv,
-                int mask_kind, const int32_t* lens, float scale, cudaStream_t s, const float* bias = nullptr,
+                int head_dim, int mask_kind, const int32_t* lens, float scale, cudaStream_t s, const float* bias = nullptr,
                 int bias_heads = 1) {
     using L = AttnSmem<D>;
     CUtensorMap tq, tk, tv;
     const uint32_t box[3] = {64, 128, 1};
     {
-        const uint64_t dims[3] = {(uint64_t)D, (uint64_t)Sq, (uint64_t)B * Hq};
-        const uint64_t strides[2] = {(uint64_t)D * 2, (uint64_t)Sq * D * 2};
+        const uint64_t dims[3] = {(uint64_t)head_dim, (uint64_t)Sq, (uint64_t)B * Hq};
+        const uint64_t strides[2] = {(uint64_t)head_dim * 2, (uint64_t)Sq * head_dim * 2};
         if (!encode_tmap_bf16_sw128(&tq, q, 3, dims, strides, box)) return FORGE_ERR_CUDA;
     }
     {
         const uint32_t box_kv[3] = {64, (uint32_t)kHalf, 1};
-        const uint64_t dims[3] = {(uint64_t)D, (uint64_t)Skv, (uint64_t)B * Hkv};
-        const uint64_t strides[2] = {(uint64_t)D * 2, (uint64_t)Skv * D * 2};
+        const uint64_t dims[3] = {(uint64_t)head_dim, (uint64_t)Skv, (uint64_t)B * Hkv};
+        const uint64_t strides[2] = {(uint64_t)head_dim * 2, (uint64_t)Skv * head_dim * 2};
         if (!encode_tmap_bf16_sw128(&tk, k, 3, dims, strides, box_kv)) return FORGE_ERR_CUDA;
         if (!encode_tmap_bf16_sw128(&tv, v, 3, dims, strides, box_kv)) return FORGE_ERR_CUDA;
     }
@@ -727,8 +729,8 @@ int launch_attn(const void* q, const void* k, const void* v, void* out, int B, i
     {
         // the output leaves in boxes of 32 rows, one per softmax warp
         const uint32_t box_o[3] = {64, 32, 1};
-        const uint64_t dims[3] = {(uint64_t)D, (uint64_t)Sq, (uint64_t)B * Hq};
-        const uint64_t strides[2] = {(uint64_t)D * 2, (uint64_t)Sq * D * 2};
+        const uint64_t dims[3] = {(uint64_t)head_dim, (uint64_t)Sq, (uint64_t)B * Hq};
+        const uint64_t strides[2] = {(uint64_t)head_dim * 2, (uint64_t)Sq * head_dim * 2};
         if (!encode_tmap_bf16_sw128(&to, out, 3, dims, strides, box_o)) return FORGE_ERR_CUDA;
     }
     AttnParams p;
@@ -737,6 +739,7 @@ int launch_attn(const void* q, const void* k, const void* v, void* out, int B, i
     p.bias = bias;
     p.bias_heads = bias_heads;
     p.inv_scale = scale > 0.f ? 1.f / scale : 0.f;
+    p.head_dim = head_dim;
     p.B = B; p.Hq = Hq; p.Hkv = Hkv; p.Sq = Sq; p.Skv = Skv;
     p.mask_kind = mask_kind;
     p.scale_log2 = scale * 1.4426950408889634f;
@@ -772,26 +775,26 @@ extern "C" int forge_attn_fused(const void* q, const void* k, const void* v, voi
                                 int B, int Hq, int Hkv, int Sq, int Skv, int D,
                                 int mask_kind, const int32_t* lens, float scale, void* stream) {
     using namespace forge;
-    int st = check_attn_args(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens);
+    int st = check_attn_args(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, /*any_head_dim=*/true);
     if (st != FORGE_OK) return st;
     if ((long long)Hq * B * ((Sq + 255) / 256) > 2147483647LL) return FORGE_ERR_UNSUPPORTED;
     if (!(scale >= 0.f)) return FORGE_ERR_UNSUPPORTED;  // the running maximum is taken on unscaled scores
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    return D == 64 ? launch_attn<64, false>(q, k, v, out, B, Hq, Hkv, Sq, Skv, mask_kind, lens, scale, s)
-                   : launch_attn<128, false>(q, k, v, out, B, Hq, Hkv, Sq, Skv, mask_kind, lens, scale, s);
+    return D <= 64 ? launch_attn<64, false>(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, s)
+                   : launch_attn<128, false>(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, s);
 }
 
 extern "C" int forge_attn_fused_f16(const void* q, const void* k, const void* v, void* out,
                                     int B, int Hq, int Hkv, int Sq, int Skv, int D,
                                     int mask_kind, const int32_t* lens, float scale, void* stream) {
     using namespace forge;
-    int st = check_attn_args(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens);
+    int st = check_attn_args(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, /*any_head_dim=*/true);
     if (st != FORGE_OK) return st;
     if ((long long)Hq * B * ((Sq + 255) / 256) > 2147483647LL) return FORGE_ERR_UNSUPPORTED;
     if (!(scale >= 0.f)) return FORGE_ERR_UNSUPPORTED;  // the running maximum is taken on unscaled scores
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    return D == 64 ? launch_attn<64, true>(q, k, v, out, B, Hq, Hkv, Sq, Skv, mask_kind, lens, scale, s)
-                   : launch_attn<128, true>(q, k, v, out, B, Hq, Hkv, Sq, Skv, mask_kind, lens, scale, s);
+    return D <= 64 ? launch_attn<64, true>(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, s)
+                   : launch_attn<128, true>(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, s);
 }
 
 extern "C" int forge_attn_fused_bias(const void* q, const void* k, const void* v, void* out,
@@ -799,13 +802,13 @@ extern "C" int forge_attn_fused_bias(const void* q, const void* k, const void* v
                                      int mask_kind, const int32_t* lens, const float* bias, int bias_heads,
                                      float scale, void* stream) {
     using namespace forge;
-    int st = check_attn_args(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens);
+    int st = check_attn_args(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, /*any_head_dim=*/true);
     if (st != FORGE_OK) return st;
     if (!bias || (reinterpret_cast<uintptr_t>(bias) & 15u)) return FORGE_ERR_INVALID_ARG;
     if (bias_heads != 1 && bias_heads != Hq) return FORGE_ERR_INVALID_ARG;
     if ((long long)Hq * B * ((Sq + 255) / 256) > 2147483647LL) return FORGE_ERR_UNSUPPORTED;
     if (!(scale > 0.f)) return FORGE_ERR_UNSUPPORTED;  // the bias enters the kernel as bias / scale
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    return D == 64 ? launch_attn<64, false, true>(q, k, v, out, B, Hq, Hkv, Sq, Skv, mask_kind, lens, scale, s, bias, bias_heads)
-                   : launch_attn<128, false, true>(q, k, v, out, B, Hq, Hkv, Sq, Skv, mask_kind, lens, scale, s, bias, bias_heads);
+    return D <= 64 ? launch_attn<64, false, true>(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, s, bias, bias_heads)
+                   : launch_attn<128, false, true>(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, s, bias, bias_heads);
 }

@@ -109,7 +109,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
                     const uint16_t* __restrict__ q, const int32_t* __restrict__ lens,
                     float* __restrict__ ws_o, float* __restrict__ ws_ml,
-                    int B, int Hq, int Hkv, int Smax, int num_splits, float scale_log2, int* status) {
+                    int B, int Hq, int Hkv, int Smax, int head_dim, int num_splits, float scale_log2, int* status) {
     constexpr int NKB = D / 32;  // 32-dim blocks of the head dimension (two k16 MMAs each)
     constexpr int NHB = D / 64;  // 64-dim blocks of the output (four 16-dim MMAs each)
     // A stage holds 16 rows of K and 16 rows of V as D / 64 tiles of 16 rows x 128 bytes each; 16-byte chunk
@@ -207,8 +207,8 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 #pragma unroll
         for (int kb = 0; kb < NKB; ++kb) {
             uint4 raw = make_uint4(0, 0, 0, 0);
-            if (g < G)
-                raw = *reinterpret_cast<const uint4*>(q + ((size_t)it.b * Hq + it.kvh * G + g) * D + kb * 32 + c * 8);
+            if (g < G && kb * 32 + c * 8 < head_dim)  // dims beyond the tensors' head size count as zeros
+                raw = *reinterpret_cast<const uint4*>(q + ((size_t)it.b * Hq + it.kvh * G + g) * head_dim + kb * 32 + c * 8);
             qr[kb][0] = raw.x; qr[kb][1] = raw.y; qr[kb][2] = raw.z; qr[kb][3] = raw.w;
         }
     };
@@ -384,7 +384,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 template <int D, bool F16>
 __global__ void __launch_bounds__(D)
 decode_combine_kernel(const float* __restrict__ ws_o, const float* __restrict__ ws_ml,
-                      uint16_t* __restrict__ out, int num_splits) {
+                      uint16_t* __restrict__ out, int num_splits, int head_dim) {
     const size_t bh = blockIdx.x;
     const int d = threadIdx.x;
     const float2* ml = reinterpret_cast<const float2*>(ws_ml) + bh * num_splits;
@@ -420,21 +420,23 @@ decode_combine_kernel(const float* __restrict__ ws_o, const float* __restrict__ 
         M = Mg;
     }
     const float res = L > 0.f ? O / L : 0.f;
-    if constexpr (F16) out[bh * D + d] = __half_as_ushort(__float2half_rn(res));
-    else out[bh * D + d] = __bfloat16_as_ushort(__float2bfloat16_rn(res));
+    if (d >= head_dim) return;  // padding columns of a head size below the kernel's
+    if constexpr (F16) out[bh * head_dim + d] = __half_as_ushort(__float2half_rn(res));
+    else out[bh * head_dim + d] = __bfloat16_as_ushort(__float2bfloat16_rn(res));
 }
 
 template <int D, int G, bool F16>
 int launch_split(const void* q, const void* kc, const void* vc, const int32_t* lens, float* ws_o, float* ws_ml,
-                 int B, int Hq, int Hkv, int Smax, int num_splits, float scale_log2, cudaStream_t s) {
+                 int B, int Hq, int Hkv, int Smax, int head_dim, int num_splits, float scale_log2, cudaStream_t s) {
     constexpr int kSmem = kWarps * kWarpRingBytes + 1024;
     int* status = device_status_word();
     if (!status) return FORGE_ERR_CUDA;
     CUtensorMap tk, tv;
     {
         const uint32_t box[3] = {64, (uint32_t)kBlockKeys, 1};
-        const uint64_t dims[3] = {(uint64_t)D, (uint64_t)Smax, (uint64_t)B * Hkv};
-        const uint64_t strides[2] = {(uint64_t)D * 2, (uint64_t)Smax * D * 2};
+        // rows of head_dim <= D elements: the TMA unit zero-fills the columns up to D
+        const uint64_t dims[3] = {(uint64_t)head_dim, (uint64_t)Smax, (uint64_t)B * Hkv};
+        const uint64_t strides[2] = {(uint64_t)head_dim * 2, (uint64_t)Smax * head_dim * 2};
         if (!encode_tmap_bf16_sw128(&tk, kc, 3, dims, strides, box)) return FORGE_ERR_CUDA;
         if (!encode_tmap_bf16_sw128(&tv, vc, 3, dims, strides, box)) return FORGE_ERR_CUDA;
     }
@@ -446,22 +448,23 @@ int launch_split(const void* q, const void* kc, const void* vc, const int32_t* l
     const long long ctas = (items + kWarps - 1) / kWarps;
     const int grid = ctas < sms ? (int)ctas : sms;
     FORGE_CUDA_TRY(launch_pdl(kernel, dim3(grid), dim3(kThreads), kSmem, s, tk, tv, static_cast<const uint16_t*>(q),
-                              lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, status));
+                              lens, ws_o, ws_ml, B, Hq, Hkv, Smax, head_dim, num_splits, scale_log2, status));
     return FORGE_OK;
 }
 
 template <int D, bool F16>
 int dispatch_g(int G, const void* q, const void* kc, const void* vc, const int32_t* lens, float* ws_o,
-               float* ws_ml, int B, int Hq, int Hkv, int Smax, int num_splits, float scale_log2, cudaStream_t s) {
+               float* ws_ml, int B, int Hq, int Hkv, int Smax, int head_dim, int num_splits, float scale_log2,
+               cudaStream_t s) {
     switch (G) {
-        case 1: return launch_split<D, 1, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
-        case 2: return launch_split<D, 2, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
-        case 3: return launch_split<D, 3, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
-        case 4: return launch_split<D, 4, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
-        case 5: return launch_split<D, 5, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
-        case 6: return launch_split<D, 6, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
-        case 7: return launch_split<D, 7, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
-        case 8: return launch_split<D, 8, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
+        case 1: return launch_split<D, 1, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, head_dim, num_splits, scale_log2, s);
+        case 2: return launch_split<D, 2, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, head_dim, num_splits, scale_log2, s);
+        case 3: return launch_split<D, 3, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, head_dim, num_splits, scale_log2, s);
+        case 4: return launch_split<D, 4, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, head_dim, num_splits, scale_log2, s);
+        case 5: return launch_split<D, 5, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, head_dim, num_splits, scale_log2, s);
+        case 6: return launch_split<D, 6, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, head_dim, num_splits, scale_log2, s);
+        case 7: return launch_split<D, 7, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, head_dim, num_splits, scale_log2, s);
+        case 8: return launch_split<D, 8, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, head_dim, num_splits, scale_log2, s);
         default: return FORGE_ERR_UNSUPPORTED;
     }
 }
@@ -472,7 +475,8 @@ int dispatch_g(int G, const void* q, const void* kc, const void* vc, const int32
 extern "C" size_t forge_attn_decode_workspace_bytes(int B, int Hq, int D, int num_splits) {
     if (B <= 0 || Hq <= 0 || D <= 0 || num_splits <= 0) return 0;
     const size_t slots = (size_t)B * Hq * num_splits;
-    return (slots * (size_t)(D + 2) * sizeof(float) + 15) & ~(size_t)15;
+    const int dp = D <= 64 ? 64 : 128;  // the partial outputs are as wide as the kernel's head dimension
+    return (slots * (size_t)(dp + 2) * sizeof(float) + 15) & ~(size_t)15;
 }
 
 namespace forge {
@@ -484,7 +488,7 @@ int decode_splitkv_impl(const void* q, const void* k_cache, const void* v_cache,
                         const int32_t* lens, int num_splits, float scale,
                         void* workspace, size_t workspace_bytes, void* stream) {
     if (!lens) return FORGE_ERR_INVALID_ARG;
-    int st = check_attn_args(q, k_cache, v_cache, out, B, Hq, Hkv, 1, Smax, D, FORGE_MASK_PADDING, lens);
+    int st = check_attn_args(q, k_cache, v_cache, out, B, Hq, Hkv, 1, Smax, D, FORGE_MASK_PADDING, lens, /*any_head_dim=*/true);
     if (st != FORGE_OK) return st;
     if (num_splits < 1) return FORGE_ERR_INVALID_ARG;
     if (num_splits > 64 || Hkv > 65535 || B > 65535) return FORGE_ERR_UNSUPPORTED;
@@ -493,12 +497,12 @@ int decode_splitkv_impl(const void* q, const void* k_cache, const void* v_cache,
 
     const size_t slots = (size_t)B * Hq * num_splits;
     float* ws_o = static_cast<float*>(workspace);
-    float* ws_ml = ws_o + slots * D;
+    float* ws_ml = ws_o + slots * (D <= 64 ? 64 : 128);
     const float scale_log2 = scale * 1.4426950408889634f;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int G = Hq / Hkv;
-    st = (D == 64) ? dispatch_g<64, F16>(G, q, k_cache, v_cache, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s)
-                   : dispatch_g<128, F16>(G, q, k_cache, v_cache, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, num_splits, scale_log2, s);
+    st = (D <= 64) ? dispatch_g<64, F16>(G, q, k_cache, v_cache, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, D, num_splits, scale_log2, s)
+                   : dispatch_g<128, F16>(G, q, k_cache, v_cache, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, D, num_splits, scale_log2, s);
     if (st != FORGE_OK) return st;
     st = finish_launch(1);
     if (st != FORGE_OK) return st;
@@ -507,10 +511,10 @@ int decode_splitkv_impl(const void* q, const void* k_cache, const void* v_cache,
     const float* cws_o = ws_o;
     const float* cws_ml = ws_ml;
     uint16_t* ob = static_cast<uint16_t*>(out);
-    if (D == 64)
-        FORGE_CUDA_TRY(launch_pdl(decode_combine_kernel<64, F16>, dim3(B * Hq), dim3(64), 0, s, cws_o, cws_ml, ob, num_splits));
+    if (D <= 64)
+        FORGE_CUDA_TRY(launch_pdl(decode_combine_kernel<64, F16>, dim3(B * Hq), dim3(64), 0, s, cws_o, cws_ml, ob, num_splits, D));
     else
-        FORGE_CUDA_TRY(launch_pdl(decode_combine_kernel<128, F16>, dim3(B * Hq), dim3(128), 0, s, cws_o, cws_ml, ob, num_splits));
+        FORGE_CUDA_TRY(launch_pdl(decode_combine_kernel<128, F16>, dim3(B * Hq), dim3(128), 0, s, cws_o, cws_ml, ob, num_splits, D));
     return finish_launch(1);
 }
 

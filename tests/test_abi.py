@@ -69,7 +69,8 @@ def test_attention_argument_validation(lib, fn):
     assert call(mask=4) == binding.ERR_INVALID_ARG
     assert call(mask=2) == binding.ERR_INVALID_ARG        # padding mask without lens
     assert call(k=P + 8) == binding.ERR_INVALID_ARG       # misaligned
-    assert call(D=80) == binding.ERR_UNSUPPORTED
+    assert call(D=256) == binding.ERR_UNSUPPORTED
+    assert call(D=100) == binding.ERR_UNSUPPORTED         # rows are not multiples of 16 bytes
 
 
 def test_decode_argument_validation(lib):
@@ -89,7 +90,8 @@ def test_decode_argument_validation(lib):
     assert call(ws=None) == binding.ERR_INVALID_ARG
     assert call(wsb=need - 1) == binding.ERR_WORKSPACE
     assert call(Hq=18, Hkv=2, wsb=1 << 30) == binding.ERR_UNSUPPORTED   # group size 9
-    assert call(D=96) == binding.ERR_UNSUPPORTED
+    assert call(D=136) == binding.ERR_UNSUPPORTED
+    assert call(D=100) == binding.ERR_UNSUPPORTED
 
 
 def test_linear_argument_validation(lib):

@@ -45,6 +45,17 @@ def test_shapes_and_masks(shape, mask_kind):
     _run(w)
 
 
+@pytest.mark.parametrize("D", [8, 32, 40, 80, 96, 120])
+@pytest.mark.parametrize("mask_kind", [1, 2])
+def test_other_head_dimensions(D, mask_kind):
+    """Head dimensions other than 64 and 128 (multiples of 8): the kernel pads them with the TMA unit's
+    zero fill; nothing is read or written beyond the rows."""
+    w = wl.attention_workload("t", 48, 2, 4, 2, 200, 333, D, mask_kind, 1.0 / np.sqrt(D), "bf16", lens_range=(1, 333))
+    q, k, v = to_device(w.q), to_device(w.k), to_device(w.v)
+    dense = binding.attn_fused(q, k, v, mask_kind, torch.from_numpy(w.lens).cuda(), w.scale)
+    assert_close_bf16(dense, oracle.attn(w.q.values, w.k.values, w.v.values, mask_kind, w.lens, w.scale))
+
+
 def test_cfg2a_gpt2_layer_full():
     _run(wl.cfg2_attention())
 

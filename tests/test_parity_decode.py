@@ -44,6 +44,13 @@ def test_batch_larger_than_the_length_ranking_limit():
     _run(w)
 
 
+@pytest.mark.parametrize("D", [32, 80, 96, 120])
+def test_other_head_dimensions(D):
+    """Head sizes other than 64 and 128 (multiples of 8) run on the next larger kernel with zero padding."""
+    w = wl.decode_workload("t", 26, 3, 8, 2, 300, D, 5, 1.0 / np.sqrt(D), (1, 300))
+    _run(w)
+
+
 def test_short_and_degenerate_lengths():
     """Fewer rows than splits (empty splits), one row, zero rows, and lens beyond Smax (clamped)."""
     w = wl.decode_workload("t", 23, 5, 8, 2, 64, 128, 16, 0.1, (1, 64))

@@ -37,7 +37,7 @@ WORKLOAD = ("GPT-2-small layer (causal attention B8 H12 S1024 D64 + c_fc GEMM 81
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (None once the kernel has changed since the capture).
-NCU_TRAFFIC_BYTES = {"attention": 38023936, "linear": 19080960, "decode": 153500000}
+NCU_TRAFFIC_BYTES = {"attention": 37918464, "linear": 18876928, "decode": 151960000}
 
 
 def load_peaks():

@@ -262,6 +262,7 @@ def run_gpu(args):
         s["do"] = torch.empty_like(s["dq"])
         s["ws"] = torch.empty(binding.attn_decode_workspace_bytes(dec.B, dec.Hq, dec.D, dec.num_splits),
                               dtype=torch.uint8, device=dev)
+        binding.attn_decode_workspace_init(s["ws"])
         sets.append(s)
     set_bytes = sum(t.numel() * t.element_size() for t in sets[0].values())
 

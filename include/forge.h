@@ -62,8 +62,10 @@ enum {
  * (Eq. 9 with the optional scale and mask nodes of Eq. 8 folded in; scores and
  * probabilities never reach global memory).  D: any multiple of 8 up to 128 (sizes other than 64 and
  * 128 run on the next larger kernel: the TMA unit pads the rows with zeros on the fly).  `lens` may be
- * NULL unless mask_kind has the padding bit.  Tensor-core path (tcgen05, TMEM
- * accumulators, TMA-staged K/V).
+ * NULL unless mask_kind has the padding bit.  scale must be >= 0 (FORGE_ERR_UNSUPPORTED otherwise: the
+ * kernel takes the running maximum on unscaled scores; forge_attn_fused_f32 accepts any sign).  Padded
+ * K and V rows (beyond lens[b]) may hold anything, including NaN and Inf: they never reach the result.
+ * Tensor-core path (tcgen05, TMEM accumulators, TMA-staged K/V).
  */
 int forge_attn_fused(const void* q, const void* k, const void* v, void* out,
                      int B, int Hq, int Hkv, int Sq, int Skv, int D,
@@ -107,17 +109,34 @@ int forge_attn_fused_f32(const void* q, const void* k, const void* v, void* out,
 
 /*
  * Decode step of the same operator (Eq. 9 with one query row per head) over a KV
- * cache, split along the cached sequence:
+ * cache, split along the cached sequence, with the combine step in the same kernel:
  *     q, out : [B, Hq, D] bf16       k_cache, v_cache : [B, Hkv, Smax, D] bf16
  * Sequence b attends rows 0 .. lens[b]-1 of its cache (lens[b] clamped to
- * [0, Smax]; 0 gives zeros).  Split s of sequence b covers rows
- * [s*c, min((s+1)*c, lens[b])) with c = ceil(lens[b] / num_splits) rounded up to a multiple of 16; each split
- * produces a partial (running max, running sum, unnormalised output) in
- * `workspace` (fp32), and a combine step merges them.  Empty splits are skipped.
- * The result does not depend on num_splits beyond rounding.
- * workspace: at least forge_attn_decode_workspace_bytes(...) bytes, 16-byte
- * aligned, contents need no initialisation and are overwritten.  Two calls that
- * may overlap on the GPU must not share a workspace.
+ * [0, Smax]; 0 gives zeros).  Rows at and beyond lens[b] may hold anything.
+ *
+ * Split rule.  Every sequence is cut into pieces of c 16-row blocks, counted from its
+ * start (the last piece may be shorter), with one c for the whole call, chosen on the
+ * device from lens: the smallest c with
+ *     c >= ceil(blocks of all sequences and kv heads / workers)   (workers = 8 per SM)
+ *     c >= ceil(blocks of the longest sequence / num_splits),
+ * raised by up to a factor of about two if that leaves no more pieces than workers.
+ * So num_splits is the largest number of pieces any sequence is cut into, and in a
+ * batch that fills the GPU every worker streams one piece of the same length.  Each
+ * piece produces a partial (running max, running sum, unnormalised output, fp32) in
+ * `workspace`; the worker that completes the last piece of a (batch, kv head) merges
+ * its partials and writes the output rows.  A sequence with a single piece never
+ * touches the workspace.  The result does not depend on num_splits beyond rounding.
+ *
+ * workspace: at least forge_attn_decode_workspace_bytes(...) bytes, 16-byte aligned.
+ * It starts with one arrival counter per (batch, kv head), which must be ZERO when a
+ * call starts: clear a new workspace once with forge_attn_decode_workspace_init (or
+ * any memset); every call that completes leaves the counters at zero, so the same
+ * workspace can be passed again and again.  The counters take the first
+ * max(64 KiB, 4 * B * Hq bytes): all shapes with B * Hq <= 16384 share that region, so
+ * a workspace cleared once also serves later calls of other such shapes; after a call
+ * with a larger B * Hq, or one that ended in FORGE_ERR_TIMEOUT, clear it again.  The
+ * rest needs no initialisation.  Two calls that may overlap on the GPU must not share
+ * a workspace.
  * 1 <= num_splits <= 64; D any multiple of 8 up to 128; Hq / Hkv must be between 1 and 8.
  */
 int forge_attn_decode_splitkv(const void* q, const void* k_cache, const void* v_cache, void* out,
@@ -135,6 +154,10 @@ int forge_attn_decode_splitkv_f16(const void* q, const void* k_cache, const void
 /* Bytes of workspace forge_attn_decode_splitkv needs; 0 for invalid arguments. */
 size_t forge_attn_decode_workspace_bytes(int B, int Hq, int D, int num_splits);
 
+/* Clears a decode workspace (a memset enqueued on `stream`): needed once after allocation, and after a
+ * call that ended in FORGE_ERR_TIMEOUT.  Belongs to the split-KV decode step above. */
+int forge_attn_decode_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+
 /*
  * forge_attn_decode_splitkv for callers that cannot provide a workspace because they cannot
  * allocate device memory at all (the paper has no counterpart to this entry point; it exists
@@ -150,14 +173,19 @@ size_t forge_attn_decode_workspace_bytes(int B, int Hq, int D, int num_splits);
  *
  *   - Problems whose partials do not fit, i.e. forge_attn_decode_workspace_bytes(B, Hq, D,
  *     num_splits) > FORGE_DECODE_STATIC_SCRATCH_BYTES, are refused with FORGE_ERR_WORKSPACE and
- *     nothing is launched (B=16, Hq=32, D=128, 16 splits needs 4.1 MiB).
+ *     nothing is launched (B=16, Hq=32, D=128, 16 splits needs 4.2 MiB).
  *   - The first call on each device looks up the array's device address (the device must be
  *     current).  Make that first call outside any stream capture; later calls do no set-up.
  *   - All calls on a device share the one array, and it keeps whatever the previous call left
- *     there.  The kernels overwrite every slot they later read, so nothing needs clearing, but
- *     two calls that may run at the same time on one GPU (different streams, threads or
- *     processes sharing the context) race on it and give wrong results: serialise them, or use
- *     forge_attn_decode_splitkv with one workspace per concurrent call.
+ *     there.  The arrival counters at its start are zero when the library is loaded and every
+ *     completed call puts them back to zero; the partial slots are overwritten before they are
+ *     read.  So nothing needs clearing between calls, but two calls that may run at the same time
+ *     on one GPU (streams or host threads of this process on the same device) race on the array
+ *     and give wrong results: serialise them, or use forge_attn_decode_splitkv with one workspace
+ *     per concurrent call.  Other processes have their own copy of the array.  A call that ended
+ *     in FORGE_ERR_TIMEOUT may leave counters behind; this entry point then stays unusable on
+ *     that device for the rest of the process.
+ *   - A slot holds (D <= 64 ? 64 : 128) + 2 floats per (batch, head, piece).
  */
 #define FORGE_DECODE_STATIC_SCRATCH_BYTES (8u << 20)
 int forge_attn_decode_splitkv_static(const void* q, const void* k_cache, const void* v_cache, void* out,
@@ -248,8 +276,33 @@ int forge_linear_bias_gelu_host(const void* x, const void* w, const void* b, voi
  * Synchronises `stream`, then reports whether any kernel launched by this library
  * since the last call gave up on a bounded wait (FORGE_ERR_TIMEOUT) and clears the
  * flag.  Returns FORGE_OK otherwise, FORGE_ERR_CUDA if the stream itself failed.
+ * The flag is one word per device, not per stream: a timeout raised by a kernel on
+ * another stream of the same device is reported to (and cleared by) whichever caller
+ * asks first, and only `stream` is synchronised.
  */
 int forge_check_status(void* stream);
+
+/*
+ * The activation of the fused linear's epilogue (Eq. 11: the `act` of matmul -> bias add -> act),
+ * applied element-wise: y[i] = act(x[i]) for i < n, fp32 device arrays (4-byte aligned), act one of
+ * FORGE_ACT_*.  The kernels of forge_linear_* call the same device function on their fp32 accumulators,
+ * so this entry point shows exactly which formula they use, at fp32 resolution (the 16-bit outputs of
+ * the fused operators cannot separate tanh-GELU from erf-GELU).  exact = 0: as in the kernels
+ * (exponential and reciprocal on the special-function unit); exact != 0: the same formulas with the
+ * accurate library routines.  Errors: FORGE_ERR_INVALID_ARG, FORGE_ERR_CUDA.
+ */
+int forge_activation_f32(const float* x, float* y, size_t n, int act, int exact, void* stream);
+
+/*
+ * Exercises the failure path of the bounded waits (every wait inside the kernels gives up after a
+ * clock budget, sets the device's status word and lets the kernel return): launches one warp that
+ * waits, with the kernels' own wait routine and a budget of `budget_clocks` SM clocks
+ * (0 .. 200,000,000), for a barrier nothing ever completes.  After the budget the warp sets the
+ * status word and exits; the next forge_check_status() returns FORGE_ERR_TIMEOUT and the one after
+ * that FORGE_OK.  Nothing else is touched; no operator kernel is involved.  The paper has no
+ * counterpart: this is a self-test of the library's error reporting.
+ */
+int forge_debug_wait_timeout(long long budget_clocks, void* stream);
 
 /* Human-readable name of a forge_status value (static storage). */
 const char* forge_status_string(int status);

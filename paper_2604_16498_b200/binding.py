@@ -30,6 +30,7 @@ SIGNATURES = {
     "forge_attn_decode_splitkv": (_i, _DEC + [_vp, _sz, _vp]),
     "forge_attn_decode_splitkv_f16": (_i, _DEC + [_vp, _sz, _vp]),
     "forge_attn_decode_workspace_bytes": (_sz, [_i, _i, _i, _i]),
+    "forge_attn_decode_workspace_init": (_i, [_vp, _sz, _vp]),
     "forge_attn_decode_splitkv_static": (_i, _DEC + [_vp]),
     "forge_linear_bias_gelu": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _vp]),
     "forge_linear_act": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp]),
@@ -44,6 +45,8 @@ SIGNATURES = {
     "forge_linear_host_scratch_bytes": (_sz, [_i, _i, _i]),
     "forge_linear_bias_gelu_host": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _vp, _sz, _vp]),
     "forge_check_status": (_i, [_vp]),
+    "forge_activation_f32": (_i, [_vp, _vp, _sz, _i, _i, _vp]),
+    "forge_debug_wait_timeout": (_i, [ctypes.c_longlong, _vp]),
     "forge_status_string": (ctypes.c_char_p, [_i]),
     "forge_last_cuda_error": (_i, []),
     "forge_launch_count": (ctypes.c_ulonglong, []),
@@ -161,9 +164,16 @@ def attn_decode_workspace_bytes(B, Hq, D, num_splits) -> int:
     return int(load().forge_attn_decode_workspace_bytes(B, Hq, D, num_splits))
 
 
+def attn_decode_workspace_init(workspace) -> None:
+    """forge_attn_decode_workspace_init: clears a new decode workspace (its arrival counters must start at zero)."""
+    _check("forge_attn_decode_workspace_init", load().forge_attn_decode_workspace_init(
+        _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream()))
+
+
 def attn_decode_splitkv(q, k_cache, v_cache, lens, num_splits, scale=None, out=None, workspace=None):
     """forge_attn_decode_splitkv (bf16 tensors) or forge_attn_decode_splitkv_f16 (fp16 tensors), chosen by
-    q.dtype: q [B,Hq,D], caches [B,Hkv,Smax,D], lens int32 [B]."""
+    q.dtype: q [B,Hq,D], caches [B,Hkv,Smax,D], lens int32 [B].  A workspace passed in must have been
+    cleared once (attn_decode_workspace_init); without one, a fresh cleared workspace is allocated."""
     B, Hq, D = q.shape
     Bk, Hkv, Smax, Dk = k_cache.shape
     if (Bk, Dk) != (B, D) or tuple(v_cache.shape) != tuple(k_cache.shape):
@@ -173,6 +183,7 @@ def attn_decode_splitkv(q, k_cache, v_cache, lens, num_splits, scale=None, out=N
     need = attn_decode_workspace_bytes(B, Hq, D, num_splits)
     if workspace is None:
         workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=q.device)
+        attn_decode_workspace_init(workspace)
     dt = torch.float16 if q.dtype == torch.float16 else torch.bfloat16
     name = "forge_attn_decode_splitkv_f16" if dt == torch.float16 else "forge_attn_decode_splitkv"
     _check(name, getattr(load(), name)(
@@ -319,6 +330,19 @@ def linear_bias_gelu_host(x, w, b, out, scratch):
         _host(x, bf, "x"), _host(w, bf, "w"), _host(b, bf, "b"), _host(out, bf, "out"), M, N, K,
         _dev(scratch, torch.uint8, "scratch"), scratch.numel(), _stream()))
     return out
+
+
+def activation_f32(x, act, exact=False, out=None):
+    """forge_activation_f32: the fused linear's epilogue activation, element-wise on an fp32 CUDA tensor."""
+    out = torch.empty_like(x) if out is None else out
+    _check("forge_activation_f32", load().forge_activation_f32(
+        _dev(x, torch.float32, "x"), _dev(out, torch.float32, "out"), x.numel(), int(act), int(bool(exact)), _stream()))
+    return out
+
+
+def debug_wait_timeout(budget_clocks: int = 1_000_000) -> None:
+    """forge_debug_wait_timeout: one warp runs the kernels' bounded wait on a barrier nothing completes."""
+    _check("forge_debug_wait_timeout", load().forge_debug_wait_timeout(int(budget_clocks), _stream()))
 
 
 def check_status() -> None:

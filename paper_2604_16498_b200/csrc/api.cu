@@ -219,7 +219,10 @@ extern "C" int forge_attn_decode_splitkv_host(const void* q, const void* k_cache
     FORGE_CUDA_TRY(cudaMemcpyAsync(dk, k_cache, kv, cudaMemcpyHostToDevice, s));
     FORGE_CUDA_TRY(cudaMemcpyAsync(dv, v_cache, kv, cudaMemcpyHostToDevice, s));
     FORGE_CUDA_TRY(cudaMemcpyAsync(dlens, lens, (size_t)B * 4, cudaMemcpyHostToDevice, s));
-    int st = forge_attn_decode_splitkv(dq, dk, dv, dout, B, Hq, Hkv, Smax, D, dlens, num_splits, scale, ws, wsb,
+    // the scratch is the caller's and may hold anything: the workspace's arrival counters must start at zero
+    int st = forge_attn_decode_workspace_init(ws, wsb, stream);
+    if (st != FORGE_OK) return st;
+    st = forge_attn_decode_splitkv(dq, dk, dv, dout, B, Hq, Hkv, Smax, D, dlens, num_splits, scale, ws, wsb,
                                        stream);
     if (st != FORGE_OK) return st;
     FORGE_CUDA_TRY(cudaMemcpyAsync(out, dout, qo, cudaMemcpyDeviceToHost, s));

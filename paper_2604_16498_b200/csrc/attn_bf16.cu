@@ -463,6 +463,9 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
         const float2 sl2v = make_float2(sl2, sl2);
         uint8_t* stage_out = smem + L::kOutOff + warp * L::kOutWarpBytes;  // this warp's 32 rows x 128 bytes per block
         int steps0 = 0, steps1 = 0;  // half-steps done so far per half (barrier phases run across items)
+        const int u = two_streams ? t : 0;  // K/V stream of this tile
+        int kvbase = 0;              // ring position of the item's first KV tile in that stream
+        const bool padding = (p.mask_kind & FORGE_MASK_PADDING) != 0;
 
         ItemInfo it;
         int i_cur = item_of_round(0);
@@ -480,6 +483,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     for (int c = 0; c < p.head_dim / 8; ++c) reinterpret_cast<uint4*>(orow)[c] = make_uint4(0, 0, 0, 0);
                 }
                 if (i_next < num_items) it_next = decode(i_next);
+                if (!two_streams) kvbase += it.n_max;  // the tiles the other query tile of the item reads
                 it = it_next; i_cur = i_next;
                 continue;
             }
@@ -636,6 +640,23 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     const float l_tile = (lsum[0].x + lsum[0].y) + (lsum[1].x + lsum[1].y);
                     l_run = l_run * alpha + l_tile;
                 }
+                // Rows of the V tile at and beyond lens[b] were copied from the caller's padding, which may hold
+                // anything; their probabilities are exactly 0, but 0 x NaN is NaN on the tensor core.  The four
+                // warps of the tile zero those rows in shared memory before the product is allowed to start (the
+                // issuer needs all four arrivals below).  Rows beyond Skv were zero-filled by the copy itself.
+                if (padding && key0 + kHalf > it.kvlen && it.kvlen < p.Skv) {
+                    const int pos = kvbase + g, st = kv_slot(u, pos);
+                    if (!warp_wait(&v_full[st], kv_phase(pos))) { failed = true; break; }
+                    const int first = max(it.kvlen - key0, 0);       // first padded row of this tile
+                    const int per_chunk = (kHalf - first) * 8;        // 16-byte pieces to clear per 64-column chunk
+                    uint8_t* vt = sV + st * L::kKVTileBytes;
+                    for (int i = quarter * 32 + lane; i < (D / 64) * per_chunk; i += 128) {
+                        const int c = i / per_chunk, rem = i - c * per_chunk;
+                        *reinterpret_cast<uint4*>(vt + c * L::kKVChunkBytes + (first + (rem >> 3)) * 128 + ((rem & 7) << 4)) =
+                            make_uint4(0, 0, 0, 0);
+                    }
+                    fence_proxy_async_smem();  // the tensor core reads what these threads wrote
+                }
                 tmem_st_wait();
                 tc_fence_before_sync();
                 __syncwarp();
@@ -687,6 +708,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     }
                 }
             }
+            kvbase += two_streams ? nh : it.n_max;
             it = it_next; i_cur = i_next;
         }
         if (lane == 0) tma_store_wait_all<0>();  // every output tile has left shared memory and is written

@@ -1,25 +1,36 @@
-// Split-KV decode attention and its combine step: Eq. 9 for a single query row per head
-// over the first lens[b] rows of a KV cache.  The cached sequence is cut into num_splits
-// ranges; each range yields a partial (running max m, running sum l, unnormalised output)
-// and the combine step merges the partials:
+// Split-KV decode attention with the combine step folded in: Eq. 9 for a single query row per head
+// over the first lens[b] rows of a KV cache.  The cached sequence of a (batch, kv head) is cut into
+// pieces; each piece yields a partial (running max m, running sum l, unnormalised output) and the
+// pieces are merged:
 //     M = max_s m_s,   L = sum_s 2^(m_s - M) l_s,   out = sum_s 2^(m_s - M) O_s / L
 // (scores are kept in log2 units: they are multiplied by scale * log2(e)).
 //
 // The work is bound by streaming K and V from HBM once, and HBM only delivers its bandwidth
 // with a deep queue of requests (pure streaming with 48 KB in flight per SM reaches 4.2 TB/s on
-// this part, with 250 KB 5.8 TB/s).  So the split kernel is persistent and every warp is an
-// independent worker: it owns whole (batch, kv head, split) items, keeps a private ring of
-// 16-row blocks in shared memory filled by TMA tile copies (16 rows x 64 columns each, 128-byte
-// swizzle, completion counted on an mbarrier per stage) that run ahead across item boundaries
-// (8 warps x 24 KB in flight per SM), and writes its partial straight from registers.  Split
-// boundaries are multiples of 16 rows, so a block never straddles two splits.  No warp ever waits for another one.  Items differ in length by up to the ratio of the
-// longest to the shortest cached sequence, so they are dealt out longest sequence first and in
-// alternating direction from round to round (a worker that got one of the longest items in one round
-// gets one of the shortest in the next), which keeps the workers' totals close together.
-// The G = Hq / Hkv query heads that share a KV
-// head are processed together, so every cached row is read exactly once.  The dot products run
-// on warp-level tensor-core MMAs (m16n8k16) with fragments read from the swizzled ring; fp32 FMAs
-// with shuffle reductions were bound by instruction issue.
+// this part, with 250 KB 5.8 TB/s).  So the kernel is persistent and every warp is an independent
+// worker: it owns whole pieces, keeps a private ring of 16-row blocks in shared memory filled by
+// TMA tile copies (16 rows x 64 columns each, 128-byte swizzle, completion counted on an mbarrier
+// per stage) that run ahead across piece boundaries (8 warps x 24 KB in flight per SM), and writes
+// its partial straight from registers.  No warp ever waits for another one.
+//
+// Pieces.  All pieces of a call are C blocks of 16 rows long (the last piece of a sequence may be
+// shorter).  Every warp works C out for itself from lens: the smallest C that is at least the even
+// share of all blocks per worker and at least ceil(longest sequence / num_splits) blocks (so no
+// sequence has more than num_splits pieces), raised further, if a modest raise achieves it, until
+// there are no more pieces than workers.  Then each worker streams at most one piece of the common
+// length, instead of num_splits pieces per sequence whose lengths differ as the sequences do.  With
+// more pieces than workers, worker w takes pieces w, w + workers, ...
+//
+// Combine.  A (batch, kv head) with one piece is normalised and written by its worker.  Otherwise
+// each worker writes its partial to the workspace, makes it visible (__threadfence) and adds one to
+// the arrival counter of its (batch, kv head); the worker that brings the counter to the number of
+// pieces merges all partials of the G heads, writes the output rows and puts the counter back to
+// zero.  Nobody waits: whoever arrives last does the merge.  The counters live at the start of the
+// workspace and must be zero when a call starts; every call leaves them at zero.
+// The G = Hq / Hkv query heads that share a KV head are processed together, so every cached row
+// is read exactly once.  The dot products run on warp-level tensor-core MMAs (m16n8k16) with
+// fragments read from the swizzled ring; fp32 FMAs with shuffle reductions were bound by
+// instruction issue.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -36,7 +47,6 @@ constexpr int kWarps = 8;
 constexpr int kThreads = kWarps * 32;
 constexpr int kBlockKeys = 16;             // cached rows per ring stage
 constexpr int kWarpRingBytes = 24 * 1024;  // per warp
-constexpr int kMaxSortedBatch = 64;        // batches up to this size are ordered by cached length
 
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 r;
@@ -74,41 +84,216 @@ __device__ __forceinline__ uint32_t pack16x2(float lo, float hi) {
     }
 }
 
-// One (batch, kv head, split) work item and its range of cached rows.
+// One piece of a (batch, kv head): rows [s0, s1) of its cache, piece number `piece` of `pieces`.
 struct Item {
-    int b, kvh, split, s0, s1;
+    int b, kvh, piece, pieces, s0, s1;
 };
-// idx counts items in dealing order: all (kv head, split) pairs of the longest sequence, then of the
-// next one, ...; order[r] is the batch entry with the r-th longest cached sequence (nullptr: identity).
-__device__ __forceinline__ Item make_item(int idx, const int32_t* lens, const int* order, int Hkv, int Smax,
-                                          int num_splits) {
+
+__device__ __forceinline__ int warp_max(int v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ long long warp_sum(long long v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// The piece schedule of a call, worked out by every warp for itself (all lanes take part and get the
+// same answer): blocks of 16 rows per piece and the number of pieces.
+struct Schedule {
+    int C;                // blocks per piece
+    long long num_items;  // pieces of all (batch, kv head) pairs
+};
+__device__ __forceinline__ int blocks_of(const int32_t* lens, int b, int Smax) {
+    return (min(max(lens[b], 0), Smax) + kBlockKeys - 1) / kBlockKeys;
+}
+// pieces of a sequence of nb blocks: at least one, so that a sequence without rows still gets its zeros
+__device__ __forceinline__ int pieces_of(int nb, int C) { return max((nb + C - 1) / C, 1); }
+
+__device__ __forceinline__ Schedule make_schedule(const int32_t* lens, int B, int Hkv, int Smax, int num_splits,
+                                                  int workers, int lane) {
+    long long total = 0;
+    int max_nb = 0;
+    for (int b0 = 0; b0 < B; b0 += 32) {
+        const int nb = (b0 + lane < B) ? blocks_of(lens, b0 + lane, Smax) : 0;
+        total += nb;
+        max_nb = max(max_nb, nb);
+    }
+    total = warp_sum(total) * Hkv;
+    max_nb = warp_max(max_nb);
+    auto count = [&](int C) {
+        long long n = 0;
+        for (int b0 = 0; b0 < B; b0 += 32)
+            if (b0 + lane < B) n += pieces_of(blocks_of(lens, b0 + lane, Smax), C);
+        return warp_sum(n) * Hkv;
+    };
+    const int c_lo = (int)max(max((total + workers - 1) / workers, (long long)((max_nb + num_splits - 1) / num_splits)), 1LL);
+    Schedule s;
+    s.C = c_lo;
+    s.num_items = count(c_lo);
+    // more pieces than workers: some worker would stream two.  Look for a slightly longer piece that leaves
+    // everyone with at most one (sixteen steps of a sixteenth cover up to twice the length).
+    if (s.num_items > workers) {
+        int C = c_lo;
+        for (int i = 0; i < 16 && C < max_nb; ++i) {
+            C += max(C >> 4, 1);
+            const long long n = count(C);
+            if (n <= workers) { s.C = C; s.num_items = n; break; }
+        }
+    }
+    return s;
+}
+
+// Piece number idx in dealing order: the kv heads of a piece of rows are consecutive (neighbouring workers
+// stream the same rows of different heads), then the next piece of the sequence, then the next sequence.
+// A warp-wide scan over lens in groups of 32 sequences finds the sequence; all lanes get the same Item.
+__device__ __forceinline__ Item make_item(long long idx, const int32_t* lens, int B, int Hkv, int Smax, int C, int lane) {
     Item it;
-    it.split = idx % num_splits;
-    const int bk = idx / num_splits;
-    it.kvh = bk % Hkv;
-    it.b = bk / Hkv;
-    if (order) it.b = order[it.b];
-    const int len = min(max(lens[it.b], 0), Smax);
-    // rows per split: the even share, rounded up to whole 16-row blocks
-    const int per = (((len + num_splits - 1) / num_splits) + kBlockKeys - 1) / kBlockKeys * kBlockKeys;
-    it.s0 = it.split * per;
-    it.s1 = min(it.s0 + per, len);
-    if (it.s1 < it.s0) it.s1 = it.s0;
+    it.kvh = (int)(idx % Hkv);
+    const long long pc = idx / Hkv;  // piece counter over the sequences
+    long long cum = 0;
+    it.b = 0; it.piece = 0; it.pieces = 1; it.s0 = it.s1 = 0;
+    for (int b0 = 0; b0 < B; b0 += 32) {
+        const int len = (b0 + lane < B) ? min(max(lens[b0 + lane], 0), Smax) : 0;
+        const int P = (b0 + lane < B) ? pieces_of((len + kBlockKeys - 1) / kBlockKeys, C) : 0;
+        int incl = P;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        const int tot = __shfl_sync(0xffffffffu, incl, 31);
+        if (pc < cum + tot) {
+            const unsigned hit = __ballot_sync(0xffffffffu, pc < cum + incl);  // first lane whose range ends beyond pc
+            const int src = __ffs(hit) - 1;
+            const int len_s = __shfl_sync(0xffffffffu, len, src);
+            const int P_s = __shfl_sync(0xffffffffu, P, src);
+            const int incl_s = __shfl_sync(0xffffffffu, incl, src);
+            it.b = b0 + src;
+            it.pieces = P_s;
+            it.piece = (int)(pc - (cum + incl_s - P_s));
+            it.s0 = min(it.piece * C * kBlockKeys, len_s);
+            it.s1 = min(it.s0 + C * kBlockKeys, len_s);
+            break;
+        }
+        cum += tot;
+    }
     return it;
 }
 
-// Worker w (= warp) takes items w, w + workers, ...; consecutive items go to different SMs.
+// Merge of the `pieces` partials of the G heads of one (batch, kv head), done by the warp that completed
+// the last piece.  Lane = D / 32 consecutive output dims.  A function of its own (not inlined): it runs once
+// per (batch, kv head) and must not take registers away from the streaming loop.
+template <int D, int G, bool F16>
+__device__ __noinline__ void merge_pieces(const float* __restrict__ ws_o, const float* __restrict__ ws_ml,
+                                          uint16_t* __restrict__ out, int head0, int pieces, int num_splits,
+                                          int head_dim, int lane) {
+    // The merge sits at the very end of the call (all pieces of a sequence end together), so it is
+    // arranged for few round trips to L2: the (m, l) pairs of all heads are requested first, then the
+    // partial outputs of two heads and sixteen pieces at a time, all before anything is used.
+    constexpr int V = D / 32;  // floats per lane
+    const int P = pieces;
+    float2 ml[G][2];  // (m, l) of pieces lane and lane + 32 (at most 64 pieces) of every head
+#pragma unroll
+    for (int h = 0; h < G; ++h) {
+        const float2* mlp = reinterpret_cast<const float2*>(ws_ml) + (size_t)(head0 + h) * num_splits;
+        ml[h][0] = (lane < P) ? __ldcg(mlp + lane) : make_float2(-INFINITY, 0.f);
+        ml[h][1] = (lane + 32 < P) ? __ldcg(mlp + lane + 32) : make_float2(-INFINITY, 0.f);
+    }
+    auto load_part = [&](int h, int sp, float (&dst)[V]) {
+        const float* src = ws_o + ((size_t)(head0 + h) * num_splits + sp) * D + lane * V;
+        if constexpr (V == 4) {
+            const float4 t4 = __ldcg(reinterpret_cast<const float4*>(src));
+            dst[0] = t4.x; dst[1] = t4.y; dst[2] = t4.z; dst[3] = t4.w;
+        } else {
+            const float2 t2 = __ldcg(reinterpret_cast<const float2*>(src));
+            dst[0] = t2.x; dst[1] = t2.y;
+        }
+    };
+#pragma unroll
+    for (int h0 = 0; h0 < G; h0 += 2) {
+        constexpr int kChunk = 16;
+        float part[2][kChunk][V];
+        auto load_chunk = [&](int s0) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e)
+#pragma unroll
+                for (int i = 0; i < kChunk; ++i) {
+                    if (h0 + e < G && s0 + i < P) load_part(h0 + e, s0 + i, part[e][i]);
+                    else {
+#pragma unroll
+                        for (int v = 0; v < V; ++v) part[e][i][v] = 0.f;
+                    }
+                }
+        };
+        load_chunk(0);
+        // weights of the two heads' pieces: w = 2^(m - M), 0 for a piece without rows
+        float w[2][2], L[2];
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const int h = (h0 + e < G) ? h0 + e : h0;
+            float M = fmaxf(ml[h][0].x, ml[h][1].x);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+            const float Mr = (M == -INFINITY) ? 0.f : M;
+            w[e][0] = exp2f(ml[h][0].x - Mr);
+            w[e][1] = exp2f(ml[h][1].x - Mr);
+            float l = w[e][0] * ml[h][0].y + w[e][1] * ml[h][1].y;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+            L[e] = l;
+        }
+        float o_acc[2][V];
+#pragma unroll
+        for (int e = 0; e < 2; ++e)
+#pragma unroll
+            for (int v = 0; v < V; ++v) o_acc[e][v] = 0.f;
+        for (int s0 = 0; s0 < P; s0 += kChunk) {
+            if (s0 > 0) load_chunk(s0);
+#pragma unroll
+            for (int e = 0; e < 2; ++e)
+#pragma unroll
+                for (int i = 0; i < kChunk; ++i) {
+                    const int sp = s0 + i;
+                    const float wgt = __shfl_sync(0xffffffffu, (sp & 32) ? w[e][1] : w[e][0], sp & 31);
+                    if (sp < P && wgt != 0.f) {
+#pragma unroll
+                        for (int v = 0; v < V; ++v) o_acc[e][v] = fmaf(wgt, part[e][i][v], o_acc[e][v]);
+                    }
+                }
+        }
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            if (h0 + e >= G) continue;
+            const float invL = L[e] > 0.f ? 1.f / L[e] : 0.f;
+            uint16_t* orow = out + (size_t)(head0 + h0 + e) * head_dim + lane * V;
+            if (lane * V < head_dim) {  // head_dim is a multiple of 8, V divides 8: all V dims are inside or none
+                if constexpr (V == 4)
+                    *reinterpret_cast<uint2*>(orow) = make_uint2(pack16x2<F16>(o_acc[e][0] * invL, o_acc[e][1] * invL),
+                                                                 pack16x2<F16>(o_acc[e][2] * invL, o_acc[e][3] * invL));
+                else
+                    *reinterpret_cast<uint32_t*>(orow) = pack16x2<F16>(o_acc[e][0] * invL, o_acc[e][1] * invL);
+            }
+        }
+    }
+}
+
+// Worker w (= warp) takes pieces w, w + workers, ...; consecutive pieces go to different SMs.
 //   S[head, key]  = Q K^T   as m16n8k16 with A = Q (rows = the G heads, padded with zero rows) and
 //                   B = K rows (the contraction runs over the head dimension in whatever order the
 //                   16-byte chunks deliver it, the same for Q and K);
 //   online softmax on the accumulator fragment (lane (g, c) owns head g, keys 2c, 2c+1 of each 8);
 //   O^T[dim, head] += V^T P^T  with A = pairs of V rows interleaved with byte permutes and B = the
 //                   probabilities exactly where the first MMA left them.
+// Workspace: counters[B * Hkv] (zero between calls), then ws_o[(b, head, piece)][D] and ws_ml[(b, head, piece)][2]
+// with num_splits piece slots per (batch, head).
 template <int D, int G, bool F16>
 __global__ void __launch_bounds__(kThreads, 1)
 decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
-                    const uint16_t* __restrict__ q, const int32_t* __restrict__ lens,
-                    float* __restrict__ ws_o, float* __restrict__ ws_ml,
+                    const uint16_t* __restrict__ q, const int32_t* __restrict__ lens, uint16_t* __restrict__ out,
+                    unsigned int* __restrict__ counters, float* __restrict__ ws_o, float* __restrict__ ws_ml,
                     int B, int Hq, int Hkv, int Smax, int head_dim, int num_splits, float scale_log2, int* status) {
     constexpr int NKB = D / 32;  // 32-dim blocks of the head dimension (two k16 MMAs each)
     constexpr int NHB = D / 64;  // 64-dim blocks of the output (four 16-dim MMAs each)
@@ -120,11 +305,6 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     constexpr int kStages = kWarpRingBytes / kStageBytes;  // 3 for D = 128, 6 for D = 64
     static_assert(kStages >= 2 && kStages <= 8, "ring size");
 
-    // Let the combine kernel (launched with programmatic stream serialisation) become resident right
-    // away: its CTAs are small, sit next to this one and block in griddepcontrol.wait until this grid
-    // has completed and its writes are visible, so the merge starts without a launch gap.
-    pdl_launch_dependents();
-    pdl_wait();  // the previous kernel in the stream has completed (this kernel may have been resident before)
     extern __shared__ __align__(128) uint8_t ring_raw[];
     __shared__ uint64_t full_bars[kWarps][8];  // [warp][stage]: the stage's rows have landed
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -140,38 +320,26 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         ptx::prefetch_tmap(&tmap_v);
     }
     __syncwarp();
+    // Set-up done: the next kernel in the stream may move in as SMs free up.  Nothing global is touched
+    // before the previous kernel has completed and its writes are visible.
+    pdl_launch_dependents();
+    pdl_wait();
 
-    const int num_items = B * Hkv * num_splits;
     const int workers = gridDim.x * kWarps;
     const int worker = warp * gridDim.x + blockIdx.x;
-
-    // ---- dealing order of the batch entries: longest cached sequence first (ties by index)
-    __shared__ int order_smem[kMaxSortedBatch];
-    const int* order = nullptr;
-    if (B <= kMaxSortedBatch) {
-        if (tid < B) {
-            const int mine = min(max(lens[tid], 0), Smax);
-            int rank = 0;
-            for (int o = 0; o < B; ++o) {
-                const int other = min(max(lens[o], 0), Smax);
-                rank += (other > mine) || (other == mine && o < tid);
-            }
-            order_smem[rank] = tid;
-        }
-        __syncthreads();
-        order = order_smem;
-    }
-    // the item of this worker in round r: rounds alternate in direction
-    auto item_of_round = [&](int r) { return r * workers + ((r & 1) ? workers - 1 - worker : worker); };
+    const Schedule sched = make_schedule(lens, B, Hkv, Smax, num_splits, workers, lane);
+    const long long num_items = sched.num_items;
+    auto item_of_round = [&](int r) { return (long long)r * workers + worker; };
 
     // ---- prefetch cursor: runs kStages blocks ahead of the compute, across item boundaries (a stage is
     // refilled as soon as its fragments are in registers, before the MMAs on them)
-    int p_round = 0, p_idx = item_of_round(0), p_j0 = 0, p_s1 = 0;
+    int p_round = 0, p_j0 = 0, p_s1 = 0;
+    long long p_idx = item_of_round(0);
     int p_bk = 0;  // batch * Hkv + kv head of the cursor's item
     int p_n = 0;  // blocks issued
     auto p_open = [&]() {  // position the cursor on the first block of the next non-empty item
         while (p_idx < num_items) {
-            const Item it = make_item(p_idx, lens, order, Hkv, Smax, num_splits);
+            const Item it = make_item(p_idx, lens, B, Hkv, Smax, sched.C, lane);
             if (it.s1 > it.s0) {
                 p_j0 = it.s0;
                 p_s1 = it.s1;
@@ -213,10 +381,10 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         }
     };
 
-    Item nxt = {0, 0, 0, 0, 0};
+    Item nxt = {0, 0, 0, 1, 0, 0};
     uint32_t qn[NKB][4];
     if (item_of_round(0) < num_items) {
-        nxt = make_item(item_of_round(0), lens, order, Hkv, Smax, num_splits);
+        nxt = make_item(item_of_round(0), lens, B, Hkv, Smax, sched.C, lane);
         load_q(nxt, qn);
     }
     int n = 0;  // blocks consumed
@@ -229,7 +397,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 #pragma unroll
             for (int i = 0; i < 4; ++i) qr[kb][i] = qn[kb][i];
         if (item_of_round(round + 1) < num_items) {  // fetch the next item's range and Q rows early
-            nxt = make_item(item_of_round(round + 1), lens, order, Hkv, Smax, num_splits);
+            nxt = make_item(item_of_round(round + 1), lens, B, Hkv, Smax, sched.C, lane);
             load_q(nxt, qn);
         }
 
@@ -346,32 +514,63 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         }
 
         if (failed) break;
-        // ---- this warp's partial is the item's partial: write it out from the fragments
+        // ---- the piece is done.  This lane holds, of heads 2c and 2c+1, dims hb*64 + g*8 + {0..7}.
         l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
         l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-        const size_t slot0 = ((size_t)it.b * Hq + it.kvh * G) * num_splits + it.split;  // head 0 of the group
+        const int head0 = it.b * Hq + it.kvh * G;  // first query head of the group, as a row of q / out
+        if (it.pieces == 1) {
+            // the only piece of its (batch, kv head): normalise and write the output rows (zeros without rows)
+            const float l_even = __shfl_sync(0xffffffffu, l_run, (2 * c) * 4);
+            const float l_odd = __shfl_sync(0xffffffffu, l_run, (2 * c + 1) * 4);
+            const float inv[2] = {l_even > 0.f ? 1.f / l_even : 0.f, l_odd > 0.f ? 1.f / l_odd : 0.f};
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                if (2 * c + e >= G) continue;
+                uint16_t* orow = out + (size_t)(head0 + 2 * c + e) * head_dim;
+#pragma unroll
+                for (int hb = 0; hb < NHB; ++hb) {
+                    const int d0 = hb * 64 + g * 8;
+                    if (d0 >= head_dim) continue;  // padding columns of a head size below the kernel's
+                    uint32_t w[4];
+#pragma unroll
+                    for (int t = 0; t < 4; t += 2) {  // dims d0 + t, t+1 (acc[.][t][e], acc[.][t+1][e]) and d0 + 4 + t, t+1
+                        w[t / 2] = pack16x2<F16>(acc[hb][t][e] * inv[e], acc[hb][t + 1][e] * inv[e]);
+                        w[2 + t / 2] = pack16x2<F16>(acc[hb][t][2 + e] * inv[e], acc[hb][t + 1][2 + e] * inv[e]);
+                    }
+                    *reinterpret_cast<uint4*>(orow + d0) = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+            }
+            continue;
+        }
+        // ---- several pieces: partial to the workspace, then the arrival count
+        const size_t slot0 = (size_t)head0 * num_splits + it.piece;  // head 0 of the group
         if (g < G && c == 0) {
             ws_ml[(slot0 + (size_t)g * num_splits) * 2] = m_run;
             ws_ml[(slot0 + (size_t)g * num_splits) * 2 + 1] = l_run;
         }
-        if (it.s1 > it.s0) {  // an empty split has m = -inf and its output slot is never read
 #pragma unroll
-            for (int hb = 0; hb < NHB; ++hb)
+        for (int e = 0; e < 2; ++e) {
+            if (2 * c + e >= G) continue;
+            float* o = ws_o + (slot0 + (size_t)(2 * c + e) * num_splits) * D;
 #pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                    const int d0 = hb * 64 + g * 8 + t;
-                    if (2 * c < G) {
-                        float* o = ws_o + (slot0 + (size_t)(2 * c) * num_splits) * D;
-                        o[d0] = acc[hb][t][0];
-                        o[d0 + 4] = acc[hb][t][2];
-                    }
-                    if (2 * c + 1 < G) {
-                        float* o = ws_o + (slot0 + (size_t)(2 * c + 1) * num_splits) * D;
-                        o[d0] = acc[hb][t][1];
-                        o[d0 + 4] = acc[hb][t][3];
-                    }
-                }
+            for (int hb = 0; hb < NHB; ++hb) {
+                const int d0 = hb * 64 + g * 8;
+                *reinterpret_cast<float4*>(o + d0) = make_float4(acc[hb][0][e], acc[hb][1][e], acc[hb][2][e], acc[hb][3][e]);
+                *reinterpret_cast<float4*>(o + d0 + 4) =
+                    make_float4(acc[hb][0][2 + e], acc[hb][1][2 + e], acc[hb][2][2 + e], acc[hb][3][2 + e]);
+            }
         }
+        __threadfence();  // the partial is visible device-wide before the arrival is counted
+        __syncwarp();
+        unsigned int arrived = 0;
+        if (lane == 0) arrived = atomicAdd(&counters[it.b * Hkv + it.kvh], 1u);
+        arrived = __shfl_sync(0xffffffffu, arrived, 0);
+        if (arrived + 1 != (unsigned)it.pieces) continue;
+
+        // ---- last to arrive: merge the pieces of the G heads
+        __threadfence();
+        if (lane == 0) counters[it.b * Hkv + it.kvh] = 0;  // as the next call expects it
+        merge_pieces<D, G, F16>(ws_o, ws_ml, out, head0, it.pieces, num_splits, head_dim, lane);
     }
     if (failed) {
         if (lane == 0) atomicExch(status, 1);
@@ -379,55 +578,10 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     }
 }
 
-// grid = B * Hq, block = D threads: merges the num_splits partials of one (batch, head).  The
-// partials are read in groups of 16 with all loads of a group in flight together.
-template <int D, bool F16>
-__global__ void __launch_bounds__(D)
-decode_combine_kernel(const float* __restrict__ ws_o, const float* __restrict__ ws_ml,
-                      uint16_t* __restrict__ out, int num_splits, int head_dim) {
-    const size_t bh = blockIdx.x;
-    const int d = threadIdx.x;
-    const float2* ml = reinterpret_cast<const float2*>(ws_ml) + bh * num_splits;
-    const float* po = ws_o + bh * num_splits * D + d;
-    pdl_launch_dependents();  // the next kernel in the stream may move in while this one runs
-    // the split kernel's writes are visible only after this returns
-    pdl_wait();
-    float M = -INFINITY, L = 0.f, O = 0.f;  // running merge over the groups
-    for (int s0 = 0; s0 < num_splits; s0 += 16) {
-        float2 mls[16];
-        float os[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const bool ok = s0 + i < num_splits;
-            mls[i] = ok ? ml[s0 + i] : make_float2(-INFINITY, 0.f);
-            // the output slot of an empty split (m = -inf) was never written: whatever is read gets weight 0
-            // through the select below
-            os[i] = ok ? po[(size_t)(s0 + i) * D] : 0.f;
-        }
-        float Mg = M;
-#pragma unroll
-        for (int i = 0; i < 16; ++i) Mg = fmaxf(Mg, mls[i].x);
-        if (Mg == -INFINITY) continue;
-        const float keep = exp2f(M - Mg);  // 0 while nothing has been merged yet
-        L *= keep;
-        O *= keep;
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const float wgt = exp2f(mls[i].x - Mg);
-            L = fmaf(wgt, mls[i].y, L);
-            O = fmaf(wgt, (mls[i].x == -INFINITY) ? 0.f : os[i], O);
-        }
-        M = Mg;
-    }
-    const float res = L > 0.f ? O / L : 0.f;
-    if (d >= head_dim) return;  // padding columns of a head size below the kernel's
-    if constexpr (F16) out[bh * head_dim + d] = __half_as_ushort(__float2half_rn(res));
-    else out[bh * head_dim + d] = __bfloat16_as_ushort(__float2bfloat16_rn(res));
-}
-
 template <int D, int G, bool F16>
-int launch_split(const void* q, const void* kc, const void* vc, const int32_t* lens, float* ws_o, float* ws_ml,
-                 int B, int Hq, int Hkv, int Smax, int head_dim, int num_splits, float scale_log2, cudaStream_t s) {
+int launch_split(const void* q, const void* kc, const void* vc, const int32_t* lens, void* out, unsigned int* counters,
+                 float* ws_o, float* ws_ml, int B, int Hq, int Hkv, int Smax, int head_dim, int num_splits,
+                 float scale_log2, cudaStream_t s) {
     constexpr int kSmem = kWarps * kWarpRingBytes + 1024;
     int* status = device_status_word();
     if (!status) return FORGE_ERR_CUDA;
@@ -444,29 +598,45 @@ int launch_split(const void* q, const void* kc, const void* vc, const int32_t* l
     FORGE_SET_SMEM_ONCE(kernel, kSmem);
     const int sms = sm_count();
     if (sms <= 0) return FORGE_ERR_CUDA;
-    const long long items = (long long)B * Hkv * num_splits;
+    // no more pieces than this can exist, whatever lens holds
+    const long long blocks_max = (Smax + kBlockKeys - 1) / kBlockKeys;
+    const long long items = (long long)B * Hkv * (blocks_max < num_splits ? blocks_max : num_splits);
     const long long ctas = (items + kWarps - 1) / kWarps;
     const int grid = ctas < sms ? (int)ctas : sms;
     FORGE_CUDA_TRY(launch_pdl(kernel, dim3(grid), dim3(kThreads), kSmem, s, tk, tv, static_cast<const uint16_t*>(q),
-                              lens, ws_o, ws_ml, B, Hq, Hkv, Smax, head_dim, num_splits, scale_log2, status));
-    return FORGE_OK;
+                              lens, static_cast<uint16_t*>(out), counters, ws_o, ws_ml, B, Hq, Hkv, Smax, head_dim,
+                              num_splits, scale_log2, status));
+    return finish_launch(1);
 }
 
 template <int D, bool F16>
-int dispatch_g(int G, const void* q, const void* kc, const void* vc, const int32_t* lens, float* ws_o,
-               float* ws_ml, int B, int Hq, int Hkv, int Smax, int head_dim, int num_splits, float scale_log2,
-               cudaStream_t s) {
+int dispatch_g(int G, const void* q, const void* kc, const void* vc, const int32_t* lens, void* out,
+               unsigned int* counters, float* ws_o, float* ws_ml, int B, int Hq, int Hkv, int Smax, int head_dim,
+               int num_splits, float scale_log2, cudaStream_t s) {
+#define FORGE_DECODE_CASE(g)                                                                                     \
+    case g:                                                                                                      \
+        return launch_split<D, g, F16>(q, kc, vc, lens, out, counters, ws_o, ws_ml, B, Hq, Hkv, Smax, head_dim, \
+                                       num_splits, scale_log2, s)
     switch (G) {
-        case 1: return launch_split<D, 1, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, head_dim, num_splits, scale_log2, s);
-        case 2: return launch_split<D, 2, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, head_dim, num_splits, scale_log2, s);
-        case 3: return launch_split<D, 3, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, head_dim, num_splits, scale_log2, s);
-        case 4: return launch_split<D, 4, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, head_dim, num_splits, scale_log2, s);
-        case 5: return launch_split<D, 5, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, head_dim, num_splits, scale_log2, s);
-        case 6: return launch_split<D, 6, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, head_dim, num_splits, scale_log2, s);
-        case 7: return launch_split<D, 7, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, head_dim, num_splits, scale_log2, s);
-        case 8: return launch_split<D, 8, F16>(q, kc, vc, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, head_dim, num_splits, scale_log2, s);
+        FORGE_DECODE_CASE(1);
+        FORGE_DECODE_CASE(2);
+        FORGE_DECODE_CASE(3);
+        FORGE_DECODE_CASE(4);
+        FORGE_DECODE_CASE(5);
+        FORGE_DECODE_CASE(6);
+        FORGE_DECODE_CASE(7);
+        FORGE_DECODE_CASE(8);
         default: return FORGE_ERR_UNSUPPORTED;
     }
+#undef FORGE_DECODE_CASE
+}
+
+// Bytes of the arrival counters at the start of the workspace: one per (batch, kv head), sized for Hkv = Hq.
+// At least 64 KiB, so that every shape with B * Hq <= 16384 keeps its counters (and only counters) in the
+// same region: a workspace cleared once then serves calls of any such shape.
+inline size_t counter_bytes(int B, int Hq) {
+    const size_t need = ((size_t)B * Hq * sizeof(unsigned int) + 255) & ~(size_t)255;
+    return need > 65536 ? need : 65536;
 }
 
 }  // namespace
@@ -476,7 +646,14 @@ extern "C" size_t forge_attn_decode_workspace_bytes(int B, int Hq, int D, int nu
     if (B <= 0 || Hq <= 0 || D <= 0 || num_splits <= 0) return 0;
     const size_t slots = (size_t)B * Hq * num_splits;
     const int dp = D <= 64 ? 64 : 128;  // the partial outputs are as wide as the kernel's head dimension
-    return (slots * (size_t)(dp + 2) * sizeof(float) + 15) & ~(size_t)15;
+    return forge::counter_bytes(B, Hq) + ((slots * (size_t)(dp + 2) * sizeof(float) + 15) & ~(size_t)15);
+}
+
+extern "C" int forge_attn_decode_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
+    using namespace forge;
+    if (!workspace || workspace_bytes == 0) return FORGE_ERR_INVALID_ARG;
+    FORGE_CUDA_TRY(cudaMemsetAsync(workspace, 0, workspace_bytes, static_cast<cudaStream_t>(stream)));
+    return FORGE_OK;
 }
 
 namespace forge {
@@ -496,26 +673,14 @@ int decode_splitkv_impl(const void* q, const void* k_cache, const void* v_cache,
     if (workspace_bytes < forge_attn_decode_workspace_bytes(B, Hq, D, num_splits)) return FORGE_ERR_WORKSPACE;
 
     const size_t slots = (size_t)B * Hq * num_splits;
-    float* ws_o = static_cast<float*>(workspace);
+    unsigned int* counters = static_cast<unsigned int*>(workspace);
+    float* ws_o = reinterpret_cast<float*>(static_cast<char*>(workspace) + counter_bytes(B, Hq));
     float* ws_ml = ws_o + slots * (D <= 64 ? 64 : 128);
     const float scale_log2 = scale * 1.4426950408889634f;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int G = Hq / Hkv;
-    st = (D <= 64) ? dispatch_g<64, F16>(G, q, k_cache, v_cache, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, D, num_splits, scale_log2, s)
-                   : dispatch_g<128, F16>(G, q, k_cache, v_cache, lens, ws_o, ws_ml, B, Hq, Hkv, Smax, D, num_splits, scale_log2, s);
-    if (st != FORGE_OK) return st;
-    st = finish_launch(1);
-    if (st != FORGE_OK) return st;
-    // The combine kernel is launched with programmatic stream serialisation: its CTAs may be placed
-    // while the split kernel drains, and block in griddepcontrol.wait until that grid has completed.
-    const float* cws_o = ws_o;
-    const float* cws_ml = ws_ml;
-    uint16_t* ob = static_cast<uint16_t*>(out);
-    if (D <= 64)
-        FORGE_CUDA_TRY(launch_pdl(decode_combine_kernel<64, F16>, dim3(B * Hq), dim3(64), 0, s, cws_o, cws_ml, ob, num_splits, D));
-    else
-        FORGE_CUDA_TRY(launch_pdl(decode_combine_kernel<128, F16>, dim3(B * Hq), dim3(128), 0, s, cws_o, cws_ml, ob, num_splits, D));
-    return finish_launch(1);
+    return (D <= 64) ? dispatch_g<64, F16>(G, q, k_cache, v_cache, lens, out, counters, ws_o, ws_ml, B, Hq, Hkv, Smax, D, num_splits, scale_log2, s)
+                     : dispatch_g<128, F16>(G, q, k_cache, v_cache, lens, out, counters, ws_o, ws_ml, B, Hq, Hkv, Smax, D, num_splits, scale_log2, s);
 }
 
 }  // namespace
@@ -583,7 +748,8 @@ extern "C" int forge_attn_decode_splitkv_static(const void* q, const void* k_cac
                                                 const int32_t* lens, int num_splits, float scale, void* stream) {
     using namespace forge;
     if (B <= 0 || Hq <= 0 || D <= 0 || num_splits <= 0) return FORGE_ERR_INVALID_ARG;
-    // the partials of this problem, B * Hq * num_splits * (D + 2) * 4 bytes, must fit the fixed array
+    // the arrival counters and the partials of this problem (num_splits slots of (D <= 64 ? 64 : 128) + 2 floats per
+    // (batch, head)) must fit the fixed array
     const size_t need = forge_attn_decode_workspace_bytes(B, Hq, D, num_splits);
     if (need > (size_t)FORGE_DECODE_STATIC_SCRATCH_BYTES) return FORGE_ERR_WORKSPACE;
     if (!q || !k_cache || !v_cache || !out || !lens) return FORGE_ERR_INVALID_ARG;

@@ -15,7 +15,7 @@ void set_last_cuda_error(cudaError_t e);
 // Counts a kernel launch (returned by forge_launch_count()).
 void count_launch(int n = 1);
 // Device-side status word, set by kernels whose bounded waits expire.
-int* device_status_word();   // device address, resolved once per process
+int* device_status_word();   // device address of the current device's word, resolved once per device
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 

@@ -21,6 +21,7 @@
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
+#include "activations.cuh"
 #include "forge_common.cuh"
 #include "sm100_ptx.cuh"
 #include "tmap.cuh"
@@ -54,25 +55,6 @@ struct LinearSmem {
     static constexpr int kTotal = kBiasOffset + 4 * BN * 4;
     static constexpr int kAlloc = kTotal + 1024;         // slack to align the base to 1024 bytes
 };
-
-__device__ __forceinline__ float gelu_tanh_f32(float z) {
-    // 0.5 z (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3)))
-    const float u = 0.7978845608028654f * z * fmaf(0.044715f * z, z, 1.0f);
-    float t;
-    asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(u));
-    const float hz = 0.5f * z;
-    return fmaf(hz, t, hz);
-}
-
-// Epilogue activations of the operator-fusion patterns (linear+gelu, linear+relu, linear+silu, mm+add).
-template <int ACT>
-__device__ __forceinline__ float activate(float z) {
-    if constexpr (ACT == FORGE_ACT_GELU_TANH) return gelu_tanh_f32(z);
-    if constexpr (ACT == FORGE_ACT_GELU_ERF) return 0.5f * z * (1.0f + erff(z * 0.70710678118654752f));
-    if constexpr (ACT == FORGE_ACT_RELU) return fmaxf(z, 0.f);
-    if constexpr (ACT == FORGE_ACT_SILU) return z / (1.0f + __expf(-z));
-    return z;
-}
 
 // 16-bit element helpers: bf16 (F16 = false) or fp16 (F16 = true)
 template <bool F16>
@@ -112,6 +94,7 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
     uint64_t* tmem_empty = tmem_full + 2;
     uint64_t* raw_full = tmem_empty + 2;  // W8: the stage's int8 tile has landed
     uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(raw_full + STAGES);
+    volatile uint32_t* epi_gave_up = tmem_base_slot + 1;  // set by an epilogue warp whose wait ran out
     float* s_bias = reinterpret_cast<float*>(smem + L::kBiasOffset);
     float* s_scale = s_bias + 2 * BN;
 
@@ -128,6 +111,7 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
         }
         for (int i = 0; i < 2; ++i) { mbar_init(&tmem_full[i], 1); mbar_init(&tmem_empty[i], kEpiThreads / 32); }
         fence_mbar_init();
+        *epi_gave_up = 0;
         prefetch_tmap(&tmap_x);
         prefetch_tmap(&tmap_w);
         if constexpr (GATED) prefetch_tmap(&tmap_w2);
@@ -269,11 +253,13 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
                 bias_s[i] = (bias != nullptr && n0 + i < N) ? widen16<F16>(bias[n0 + i]) : 0.f;
                 if constexpr (W8) scale_s[i] = (n0 + i < N) ? scale[n0 + i] : 0.f;
             }
-            asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
-            // A warp that gave up keeps taking part in the named barrier above (so the others never
-            // wait for it there) but skips the work.
-            if (!failed && !warp_wait(&tmem_full[acc], acc_phase)) failed = true;
-            if (failed) continue;
+            // The accumulator is complete.  Whether to go on is decided for the whole epilogue group: a warp
+            // whose wait ran out says so in shared memory before the barrier, and all eight warps read the
+            // flag after it, so either all of them enter the block loop below (whose barriers need all of
+            // them) or all leave.
+            if (!warp_wait(&tmem_full[acc], acc_phase) && lane == 0) *epi_gave_up = 1;
+            asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");  // also publishes bias_s / scale_s
+            if (*epi_gave_up) { failed = true; break; }
             tc_fence_after_sync();
             const int row = quarter * 32 + lane;  // row of the tile = TMEM lane
             const uint32_t taddr = tmem_base + acc * kAccStride + (static_cast<uint32_t>(quarter * 32) << 16);

@@ -53,21 +53,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // About two seconds at 2 GHz; far beyond any legitimate wait in these kernels.
 constexpr long long kWaitBudgetClocks = 4000000000LL;
 
-// Waits for the phase with the given parity.  Returns false if the budget ran out.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+// Waits for the phase with the given parity.  Returns false if the budget (in SM clocks) ran out.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, long long budget_clocks = kWaitBudgetClocks) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 0x3ffu) == 0 && clock64() - t0 > kWaitBudgetClocks) return false;
+        if ((++spins & 0x3ffu) == 0 && clock64() - t0 > budget_clocks) return false;
     }
     return true;
 }
 
 // Same for a whole converged warp: every lane gets the same answer, so that the warp-collective
 // (.sync.aligned) instructions that follow are executed by all lanes or by none.
-__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity) {
-    return __all_sync(0xffffffffu, mbar_wait(bar, parity));
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, long long budget_clocks = kWaitBudgetClocks) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, budget_clocks));
 }
 
 // ----------------------------------------------------------------- fences

@@ -64,6 +64,7 @@ def main() -> None:
         vc = randn((a.B, a.Hkv, a.S, a.D))
         out = torch.empty_like(q)
         ws = torch.empty(binding.attn_decode_workspace_bytes(a.B, a.Hq, a.D, a.splits), dtype=torch.uint8, device=dev)
+        binding.attn_decode_workspace_init(ws)
         call = lambda: binding.attn_decode_splitkv(q, kc, vc, lens, a.splits, a.D ** -0.5, out=out, workspace=ws)
 
     for _ in range(a.warmup):

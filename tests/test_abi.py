@@ -44,7 +44,10 @@ def test_status_strings(lib):
 
 
 def test_workspace_size(lib):
-    assert lib.forge_attn_decode_workspace_bytes(16, 32, 128, 16) == 16 * 32 * 16 * (128 + 2) * 4
+    # arrival counters (64 KiB, or 4 bytes per (batch, head) if that is more) + num_splits partial slots per (batch, head)
+    assert lib.forge_attn_decode_workspace_bytes(16, 32, 128, 16) == 65536 + 16 * 32 * 16 * (128 + 2) * 4
+    assert lib.forge_attn_decode_workspace_bytes(3, 8, 40, 5) == 65536 + 3 * 8 * 5 * (64 + 2) * 4
+    assert lib.forge_attn_decode_workspace_bytes(4096, 8, 64, 1) == 4096 * 8 * 4 + 4096 * 8 * (64 + 2) * 4
     assert lib.forge_attn_decode_workspace_bytes(0, 32, 128, 16) == 0
 
 

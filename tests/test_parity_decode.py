@@ -71,6 +71,37 @@ def test_rows_beyond_lens_are_never_read_into_the_result():
     assert torch.equal(a, b2)
 
 
+def test_one_workspace_serves_call_after_call_with_other_shapes():
+    """The arrival counters at the start of the workspace are cleared once; every call leaves them at zero,
+    so the same (oversized) workspace works for any later call."""
+    ws = torch.empty(binding.attn_decode_workspace_bytes(16, 32, 128, 16), dtype=torch.uint8, device="cuda")
+    ws.fill_(0xFF)
+    binding.attn_decode_workspace_init(ws)
+    for rep in range(2):
+        for (B, Hq, Hkv, Smax, D, splits, lo) in [(6, 32, 8, 1500, 128, 16, 200), (3, 8, 2, 700, 64, 9, 1),
+                                                  (16, 16, 8, 2100, 128, 4, 1800), (2, 8, 1, 4000, 128, 16, 3000)]:
+            w = wl.decode_workload("t", 27, B, Hq, Hkv, Smax, D, splits, 1.0 / np.sqrt(D), (lo, Smax))
+            out = binding.attn_decode_splitkv(to_device(w.q), to_device(w.k_cache), to_device(w.v_cache),
+                                              torch.from_numpy(w.lens).cuda(), splits, w.scale, workspace=ws)
+            binding.check_status()
+            assert_close_bf16(out, oracle.attn_decode(w.q.values, w.k_cache.values, w.v_cache.values, w.lens, w.scale))
+
+
+def test_more_pieces_than_workers():
+    """A batch whose pieces outnumber the GPU's workers (8 per SM) even at the longest allowed piece: workers
+    take several pieces each."""
+    w = wl.decode_workload("t", 28, 200, 8, 8, 48, 64, 2, 0.125, (1, 48))
+    _run(w)
+
+
+def test_run_to_run_bitwise_identical():
+    w = wl.cfg5_gqa_decode(B=8)
+    q, k, v, lens = to_device(w.q), to_device(w.k_cache), to_device(w.v_cache), torch.from_numpy(w.lens).cuda()
+    a = binding.attn_decode_splitkv(q, k, v, lens, w.num_splits, w.scale)
+    b = binding.attn_decode_splitkv(q, k, v, lens, w.num_splits, w.scale)
+    assert torch.equal(a, b)
+
+
 def test_workspace_too_small_is_rejected():
     w = wl.decode_workload("t", 25, 1, 4, 1, 32, 64, 4, 0.125, (5, 32))
     ws = torch.empty(16, dtype=torch.uint8, device="cuda")

@@ -32,18 +32,11 @@ def test_shapes(M, N, K):
     assert_close_bf16(y, ref)
 
 
-def test_cfg2b_full_size_sampled_rows():
-    """Benchmark shape and launch configuration; the oracle checks 96 whole output rows
-    (first/last rows of tiles and a seeded random sample)."""
+def test_cfg2b_full_size():
+    """Benchmark shape and launch configuration, every output element against the oracle."""
     w = wl.cfg2_linear()
     y = _run(w)
-    rng = np.random.default_rng(5)
-    rows = np.unique(np.concatenate([[0, 1, 127, 128, 4095, 4096, 8191], rng.integers(0, w.M, 89)]))
-    ref = oracle.linear_bias_gelu(w.x.values[rows], w.w.values, w.b.values)
-    assert_close_bf16(y[torch.from_numpy(rows).cuda()], ref)
-    # every output must be finite and inside GELU's range for these inputs
-    yf = to_f64(y)
-    assert np.isfinite(yf).all() and yf.min() >= -0.18
+    assert_close_bf16(y, oracle.linear_bias_gelu(w.x.values, w.w.values, w.b.values))
 
 
 def test_identity_weight_gives_gelu_of_x_plus_b():

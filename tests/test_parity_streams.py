@@ -30,11 +30,11 @@ def test_two_streams_give_the_serial_results():
             outs.append(binding.attn_decode_splitkv(dq, kc, vc, lens, dec.num_splits, dec.scale, workspace=ws))
         return outs
 
-    serial = work(torch.empty(nbytes, dtype=torch.uint8, device="cuda"))
+    serial = work(torch.zeros(nbytes, dtype=torch.uint8, device="cuda"))
     torch.cuda.synchronize()
     s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
-    ws1 = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
-    ws2 = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    ws1 = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")  # the arrival counters start at zero
+    ws2 = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
     torch.cuda.synchronize()
     with torch.cuda.stream(s1):
         a = work(ws1)

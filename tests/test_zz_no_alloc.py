@@ -11,6 +11,7 @@ has already run every other test.
 import pytest
 import torch
 
+import oracle
 from paper_2604_16498_b200 import binding, workloads as wl
 from util import assert_close_bf16, to_device, to_f64
 
@@ -31,8 +32,8 @@ def test_matches_the_workspace_entry_point_on_two_calls_in_a_row():
     lib = binding.load()
     stream = torch.cuda.current_stream().cuda_stream
     cases = [
-        # 24 and 20 splits: more than a thread-block cluster holds, so the partials really go through
-        # the fixed array (6.1 MiB of it in the first call, a small corner of it in the second)
+        # long sequences cut into many pieces, so the partials really go through the fixed array (the
+        # first call may use up to 6.2 MiB of it, the second a small corner)
         wl.decode_workload("first", 61, 16, 32, 8, 1024, 128, 24, 128 ** -0.5, (300, 1024)),
         wl.decode_workload("second", 62, 3, 8, 2, 700, 64, 20, 0.125, (1, 700)),
     ]
@@ -48,6 +49,8 @@ def test_matches_the_workspace_entry_point_on_two_calls_in_a_row():
         binding.check_status()
         assert_close_bf16(out, to_f64(expect))
         assert torch.equal(out, expect)  # same kernels, same order of operations
+        # and both are right: the oracle on the same inputs
+        assert_close_bf16(out, oracle.attn_decode(w.q.values, w.k_cache.values, w.v_cache.values, w.lens, w.scale))
 
 
 @pytest.mark.gpu
@@ -56,7 +59,7 @@ def test_too_large_problem_launches_nothing():
     q, k, v = to_device(w.q), to_device(w.k_cache), to_device(w.v_cache)
     lens = torch.from_numpy(w.lens).cuda()
     before = binding.launch_count()
-    # claim a batch whose partials (B * Hq * splits * (D + 2) * 4 bytes) exceed the 8 MiB array
+    # claim a batch whose counters and partials (4 slots of 130 floats per (batch, head)) exceed the 8 MiB array
     st = binding.load().forge_attn_decode_splitkv_static(
         q.data_ptr(), k.data_ptr(), v.data_ptr(), q.data_ptr(), 4096, 8, 2, 64, 128, lens.data_ptr(), 4, 0.1,
         torch.cuda.current_stream().cuda_stream)

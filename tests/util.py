@@ -46,3 +46,31 @@ def assert_close_bf16(got, ref):
     assert err.max() <= BF16_MAX_ABS, f"max-abs {err.max():.3e} > {BF16_MAX_ABS}"
     assert err.mean() <= BF16_MEAN_ABS, f"mean-abs {err.mean():.3e} > {BF16_MEAN_ABS}"
     return err.max(), err.mean()
+
+
+# ---- canary-guarded buffers: outputs and workspaces carved out of a larger allocation filled with a
+# sentinel, so that a write outside the buffer (a clipped TMA store that did not clip, a ragged tail
+# stored with full-width vectors) shows up even when the result itself is right.
+GUARD_BYTES = 4096
+_SENTINEL = 0x5A
+
+
+class Guarded:
+    """A CUDA tensor of `shape` / `dtype` with GUARD_BYTES of sentinel on both sides."""
+
+    def __init__(self, shape, dtype, fill_nan=True):
+        es = torch.empty((), dtype=dtype).element_size()
+        n = int(np.prod(shape)) * es
+        self.nbytes = n
+        self.raw = torch.full((GUARD_BYTES + n + GUARD_BYTES,), _SENTINEL, dtype=torch.uint8, device="cuda")
+        assert self.raw.data_ptr() % 256 == 0
+        self.tensor = self.raw[GUARD_BYTES:GUARD_BYTES + n].view(dtype).view(shape)
+        if fill_nan and dtype in (torch.bfloat16, torch.float16, torch.float32):
+            self.tensor.fill_(float("nan"))  # a position the kernel fails to write stays visible
+
+    def assert_intact(self):
+        torch.cuda.synchronize()
+        lo = self.raw[:GUARD_BYTES]
+        hi = self.raw[GUARD_BYTES + self.nbytes:]
+        assert bool((lo == _SENTINEL).all()), "bytes before the buffer were overwritten"
+        assert bool((hi == _SENTINEL).all()), "bytes after the buffer were overwritten"

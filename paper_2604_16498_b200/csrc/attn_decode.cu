@@ -94,86 +94,108 @@ __device__ __forceinline__ int warp_max(int v) {
     for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(0xffffffffu, v, o));
     return v;
 }
-__device__ __forceinline__ long long warp_sum(long long v) {
+__device__ __forceinline__ unsigned warp_sum(unsigned v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
 }
 
 // The piece schedule of a call, worked out by every warp for itself (all lanes take part and get the
-// same answer): blocks of 16 rows per piece and the number of pieces.
+// same answer): blocks of 16 rows per piece and the number of pieces.  All counts fit 32 bits (the host
+// refuses shapes whose block count does not).  Lane l also keeps what the search for a piece needs of
+// sequence l (its length, its pieces and the running total up to and including it): with B <= 32 no
+// piece lookup touches memory again, which shortens the way from the first read of lens to the first copy.
 struct Schedule {
-    int C;                // blocks per piece
-    long long num_items;  // pieces of all (batch, kv head) pairs
+    int C;               // blocks per piece
+    unsigned num_items;  // pieces of all (batch, kv head) pairs
+    int len0, P0, incl0; // of sequence `lane`: clamped length, pieces, pieces of sequences 0..lane
 };
-__device__ __forceinline__ int blocks_of(const int32_t* lens, int b, int Smax) {
-    return (min(max(lens[b], 0), Smax) + kBlockKeys - 1) / kBlockKeys;
-}
+__device__ __forceinline__ int clamped_len(const int32_t* lens, int b, int Smax) { return min(max(lens[b], 0), Smax); }
+__device__ __forceinline__ int blocks_of_len(int len) { return (len + kBlockKeys - 1) / kBlockKeys; }
 // pieces of a sequence of nb blocks: at least one, so that a sequence without rows still gets its zeros
 __device__ __forceinline__ int pieces_of(int nb, int C) { return max((nb + C - 1) / C, 1); }
+__device__ __forceinline__ int warp_incl_scan(int v, int lane) {
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += t;
+    }
+    return v;
+}
 
 __device__ __forceinline__ Schedule make_schedule(const int32_t* lens, int B, int Hkv, int Smax, int num_splits,
                                                   int workers, int lane) {
-    long long total = 0;
-    int max_nb = 0;
-    for (int b0 = 0; b0 < B; b0 += 32) {
-        const int nb = (b0 + lane < B) ? blocks_of(lens, b0 + lane, Smax) : 0;
+    Schedule s;
+    s.len0 = (lane < B) ? clamped_len(lens, lane, Smax) : 0;
+    const int nb0 = blocks_of_len(s.len0);
+    unsigned total = nb0;
+    int max_nb = nb0;
+    for (int b = 32 + lane; b < B; b += 32) {
+        const int nb = blocks_of_len(clamped_len(lens, b, Smax));
         total += nb;
         max_nb = max(max_nb, nb);
     }
     total = warp_sum(total) * Hkv;
     max_nb = warp_max(max_nb);
+    // pieces of all sequences for a piece length C; leaves group 0's scan in s
     auto count = [&](int C) {
-        long long n = 0;
-        for (int b0 = 0; b0 < B; b0 += 32)
-            if (b0 + lane < B) n += pieces_of(blocks_of(lens, b0 + lane, Smax), C);
-        return warp_sum(n) * Hkv;
+        s.P0 = (lane < B) ? pieces_of(nb0, C) : 0;
+        s.incl0 = warp_incl_scan(s.P0, lane);
+        unsigned n = (unsigned)__shfl_sync(0xffffffffu, s.incl0, 31);
+        if (B > 32) {
+            unsigned rest = 0;
+            for (int b = 32 + lane; b < B; b += 32) rest += pieces_of(blocks_of_len(clamped_len(lens, b, Smax)), C);
+            n += warp_sum(rest);
+        }
+        return n * Hkv;
     };
-    const int c_lo = (int)max(max((total + workers - 1) / workers, (long long)((max_nb + num_splits - 1) / num_splits)), 1LL);
-    Schedule s;
+    const int c_lo = max(max((int)((total + workers - 1) / (unsigned)workers), (max_nb + num_splits - 1) / num_splits), 1);
     s.C = c_lo;
     s.num_items = count(c_lo);
     // more pieces than workers: some worker would stream two.  Look for a slightly longer piece that leaves
     // everyone with at most one (sixteen steps of a sixteenth cover up to twice the length).
-    if (s.num_items > workers) {
+    if (s.num_items > (unsigned)workers) {
         int C = c_lo;
-        for (int i = 0; i < 16 && C < max_nb; ++i) {
+        bool found = false;
+        for (int i = 0; i < 16 && C < max_nb && !found; ++i) {
             C += max(C >> 4, 1);
-            const long long n = count(C);
-            if (n <= workers) { s.C = C; s.num_items = n; break; }
+            const unsigned n = count(C);
+            if (n <= (unsigned)workers) { s.C = C; s.num_items = n; found = true; }
         }
+        if (!found) s.num_items = count(c_lo);  // restores group 0's scan for c_lo
     }
     return s;
 }
 
 // Piece number idx in dealing order: the kv heads of a piece of rows are consecutive (neighbouring workers
 // stream the same rows of different heads), then the next piece of the sequence, then the next sequence.
-// A warp-wide scan over lens in groups of 32 sequences finds the sequence; all lanes get the same Item.
-__device__ __forceinline__ Item make_item(long long idx, const int32_t* lens, int B, int Hkv, int Smax, int C, int lane) {
+// A warp-wide scan over lens in groups of 32 sequences finds the sequence (the first group's scan is kept
+// in the schedule); all lanes get the same Item.
+__device__ __forceinline__ Item make_item(unsigned idx, const Schedule& sc, const int32_t* lens, int B, int Hkv, int Smax,
+                                          int lane) {
     Item it;
-    it.kvh = (int)(idx % Hkv);
-    const long long pc = idx / Hkv;  // piece counter over the sequences
-    long long cum = 0;
+    const unsigned pc = idx / (unsigned)Hkv;  // piece counter over the sequences
+    it.kvh = (int)(idx - pc * (unsigned)Hkv);
     it.b = 0; it.piece = 0; it.pieces = 1; it.s0 = it.s1 = 0;
+    const int C = sc.C;
+    unsigned cum = 0;
+    int len = sc.len0, P = sc.P0, incl = sc.incl0;
     for (int b0 = 0; b0 < B; b0 += 32) {
-        const int len = (b0 + lane < B) ? min(max(lens[b0 + lane], 0), Smax) : 0;
-        const int P = (b0 + lane < B) ? pieces_of((len + kBlockKeys - 1) / kBlockKeys, C) : 0;
-        int incl = P;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int v = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += v;
+        if (b0 > 0) {
+            len = (b0 + lane < B) ? clamped_len(lens, b0 + lane, Smax) : 0;
+            P = (b0 + lane < B) ? pieces_of(blocks_of_len(len), C) : 0;
+            incl = warp_incl_scan(P, lane);
         }
-        const int tot = __shfl_sync(0xffffffffu, incl, 31);
+        const unsigned tot = (unsigned)__shfl_sync(0xffffffffu, incl, 31);
         if (pc < cum + tot) {
-            const unsigned hit = __ballot_sync(0xffffffffu, pc < cum + incl);  // first lane whose range ends beyond pc
+            const unsigned hit = __ballot_sync(0xffffffffu, pc < cum + (unsigned)incl);  // first lane whose range ends beyond pc
             const int src = __ffs(hit) - 1;
             const int len_s = __shfl_sync(0xffffffffu, len, src);
             const int P_s = __shfl_sync(0xffffffffu, P, src);
             const int incl_s = __shfl_sync(0xffffffffu, incl, src);
             it.b = b0 + src;
             it.pieces = P_s;
-            it.piece = (int)(pc - (cum + incl_s - P_s));
+            it.piece = (int)(pc - (cum + (unsigned)(incl_s - P_s)));
             it.s0 = min(it.piece * C * kBlockKeys, len_s);
             it.s1 = min(it.s0 + C * kBlockKeys, len_s);
             break;
@@ -328,18 +350,18 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     const int workers = gridDim.x * kWarps;
     const int worker = warp * gridDim.x + blockIdx.x;
     const Schedule sched = make_schedule(lens, B, Hkv, Smax, num_splits, workers, lane);
-    const long long num_items = sched.num_items;
-    auto item_of_round = [&](int r) { return (long long)r * workers + worker; };
+    const unsigned num_items = sched.num_items;
+    auto item_of_round = [&](int r) { return (unsigned)r * (unsigned)workers + (unsigned)worker; };
 
     // ---- prefetch cursor: runs kStages blocks ahead of the compute, across item boundaries (a stage is
     // refilled as soon as its fragments are in registers, before the MMAs on them)
     int p_round = 0, p_j0 = 0, p_s1 = 0;
-    long long p_idx = item_of_round(0);
+    unsigned p_idx = item_of_round(0);
     int p_bk = 0;  // batch * Hkv + kv head of the cursor's item
     int p_n = 0;  // blocks issued
     auto p_open = [&]() {  // position the cursor on the first block of the next non-empty item
         while (p_idx < num_items) {
-            const Item it = make_item(p_idx, lens, B, Hkv, Smax, sched.C, lane);
+            const Item it = make_item(p_idx, sched, lens, B, Hkv, Smax, lane);
             if (it.s1 > it.s0) {
                 p_j0 = it.s0;
                 p_s1 = it.s1;
@@ -384,7 +406,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     Item nxt = {0, 0, 0, 1, 0, 0};
     uint32_t qn[NKB][4];
     if (item_of_round(0) < num_items) {
-        nxt = make_item(item_of_round(0), lens, B, Hkv, Smax, sched.C, lane);
+        nxt = make_item(item_of_round(0), sched, lens, B, Hkv, Smax, lane);
         load_q(nxt, qn);
     }
     int n = 0;  // blocks consumed
@@ -397,7 +419,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 #pragma unroll
             for (int i = 0; i < 4; ++i) qr[kb][i] = qn[kb][i];
         if (item_of_round(round + 1) < num_items) {  // fetch the next item's range and Q rows early
-            nxt = make_item(item_of_round(round + 1), lens, B, Hkv, Smax, sched.C, lane);
+            nxt = make_item(item_of_round(round + 1), sched, lens, B, Hkv, Smax, lane);
             load_q(nxt, qn);
         }
 
@@ -669,6 +691,8 @@ int decode_splitkv_impl(const void* q, const void* k_cache, const void* v_cache,
     if (st != FORGE_OK) return st;
     if (num_splits < 1) return FORGE_ERR_INVALID_ARG;
     if (num_splits > 64 || Hkv > 65535 || B > 65535) return FORGE_ERR_UNSUPPORTED;
+    // the kernel counts 16-row blocks and pieces in 32 bits
+    if ((long long)B * Hkv * ((Smax + kBlockKeys - 1) / kBlockKeys) >= (1LL << 31)) return FORGE_ERR_UNSUPPORTED;
     if (!workspace || !aligned16(workspace)) return FORGE_ERR_INVALID_ARG;
     if (workspace_bytes < forge_attn_decode_workspace_bytes(B, Hq, D, num_splits)) return FORGE_ERR_WORKSPACE;
 

@@ -2,23 +2,37 @@
 """Benchmark of the fused-operator hot path on B200.
 
 One step = one pass of the whole path over one batch of synthetic input:
-  1. fused c_fc GEMM + bias + tanh-GELU               (8192 x 3072 x 768, bf16)
-  2. fused causal attention, GPT-2-small layer shape  (B8 H12 S1024 D64, bf16)
-  3. split-KV GQA decode over a KV cache              (B16 32/8 heads D128, lens U[1024,4096], 16 splits)
-The headline value is the step's algorithmic FLOPs per second; the per-kernel numbers
-(TFLOP/s or GB/s and the fraction of the measured peak) are in "kernels" and "roofline".
+  1. fused c_fc GEMM + bias + tanh-GELU                        (8192 x 3072 x 768, bf16)
+  2. fused causal GQA prefill attention, 8B-class shape        (B4 32/8 heads S2048 D128, bf16)
+  3. split-KV GQA decode over a KV cache                       (B16 32/8 heads D128, lens U[1024,4096], 16 splits)
+on three rotating input sets, so that no buffer is L2-resident when it is used again.
+
+The metric has two halves.  `value` is the first: fused-attention TFLOP/s (algorithmic FLOPs of the
+prefill attention / its average launch duration); the second, split-KV decode GB/s, is in `decode_hbm`.
+`ms_per_step` is the whole step.  `kernels` holds every kernel's duration, rate and fraction of the
+measured peak; `roofline` repeats that for the kernel with the longest duration.
+
+Kernel durations: the library launches with programmatic stream serialisation, so an event between two
+kernels changes what it measures.  Each kernel is therefore timed on its own, K calls back to back on the
+rotating cold inputs with events around the K calls (`ms`); the step loop is timed the same way
+(`ms_per_step`); and a third pass puts events around every kernel inside the step (`ms_in_step`, an upper
+bound: the events take the overlap of neighbouring launches away).  Every timed region is repeated
+`--repeats` times; medians are reported with the extremes beside them.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 
-With N > 1 (torchrun, one rank per GPU) every rank runs the same step on its own data:
-the path shards by batch with no exchange, so scaling is weak and no collective is timed.
-`--impl reference` times the fp64 CPU oracle on a bounded sample of the same step.
+With N > 1 every rank runs the same step on its own data: the path shards by batch with no exchange, so
+scaling is weak and no collective is timed.  Started without a launcher (`WORLD_SIZE` unset), `--gpus N`
+starts the N ranks itself through torch.distributed.run.  `--impl reference` times the fp64 CPU oracle on
+a bounded sample of the same step.
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
+import subprocess
 import sys
 import threading
 import time
@@ -31,13 +45,14 @@ sys.path.insert(0, ROOT)
 from paper_2604_16498_b200 import workloads as wl  # noqa: E402
 
 METRIC = "fused attention TFLOP/s (% bf16 TC peak); split-KV decode HBM GB/s (% peak)"
-WORKLOAD = ("GPT-2-small layer (causal attention B8 H12 S1024 D64 + c_fc GEMM 8192x3072x768 with bias and "
-            "tanh-GELU) followed by 8B-class GQA split-KV decode (B16 32/8 heads D128, cached lengths "
+WORKLOAD = ("8B-class causal GQA prefill attention (B4 32/8 heads S2048 D128) + GPT-2-small c_fc GEMM 8192x3072x768 "
+            "with bias and tanh-GELU + 8B-class GQA split-KV decode (B16 32/8 heads D128, cached lengths "
             "U[1024,4096], 16 splits)")
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+NOMINAL_PEAKS = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (None once the kernel has changed since the capture).
-NCU_TRAFFIC_BYTES = {"attention": 37918464, "linear": 18876928, "decode": 151960000}
+NCU_TRAFFIC_BYTES = {"attention": None, "linear": None, "decode": None}
 
 
 def load_peaks():
@@ -52,10 +67,11 @@ def load_peaks():
 
 # ----------------------------------------------------------------------------- clocks
 class ClockSampler:
-    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+    """Samples SM clock and throttle reasons through NVML while the timed regions run."""
 
-    def __init__(self, index: int, period_s: float = 0.005):
+    def __init__(self, index: int, period_s: float = 0.002):
         self.samples, self.reasons = [], set()
+        self.active = True  # samples are kept only while this is set
         self.max_mhz = None
         self._stop = threading.Event()
         self._thread = None
@@ -82,11 +98,14 @@ class ClockSampler:
             getattr(nv, "nvmlDeviceGetCurrentClocksThrottleReasons")
         while not self._stop.is_set():
             try:
-                self.samples.append(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
-                mask = get_reasons(self._h)
-                for name, bit in names.items():
-                    if mask & bit:
-                        self.reasons.add(name)
+                if self.active:
+                    mhz = nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)
+                    mask = get_reasons(self._h)
+                    if self.active:
+                        self.samples.append(mhz)
+                        for name, bit in names.items():
+                            if mask & bit:
+                                self.reasons.add(name)
             except Exception:
                 pass
             time.sleep(self._period)
@@ -106,49 +125,54 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------- CPU oracle legs
-def oracle_sample_step(att, lin, dec, n_heads, n_rows, n_seqs):
-    """One pass of the step on the CPU oracle over a sample: the first n_heads (batch 0.., head)
-    slices of the attention, the first n_rows rows of the GEMM, the first n_seqs decode sequences.
-    Returns the algorithmic FLOPs it performed."""
-    import oracle
-    H = att.Hq
-    flops = 0
-    done = 0
-    b = 0
-    while done < n_heads:
-        take = min(H, n_heads - done)
-        oracle.attn(att.q.values[b:b + 1, :take], att.k.values[b:b + 1, :take], att.v.values[b:b + 1, :take],
-                    att.mask_kind, None, att.scale)
-        done += take
-        b += 1
-    flops += att.flops() // (att.B * H) * n_heads
-    oracle.linear_bias_gelu(lin.x.values[:n_rows], lin.w.values, lin.b.values)
-    flops += 2 * n_rows * lin.N * lin.K
-    oracle.attn_decode(dec.q.values[:n_seqs], dec.k_cache.values[:n_seqs], dec.v_cache.values[:n_seqs],
-                       dec.lens[:n_seqs], dec.scale)
-    flops += 4 * dec.D * dec.Hq * int(dec.lens[:n_seqs].sum())
-    return flops
-
-
 def make_host_workloads(decode_B=16):
-    att = wl.cfg2_attention()
+    att = wl.cfg4_gqa_prefill()
     lin = wl.cfg2_linear()
     dec = wl.cfg5_gqa_decode(B=decode_B)
     return att, lin, dec
 
 
+def oracle_sample_step(att, lin, dec, n_heads, n_rows, n_seqs):
+    """One pass of the step on the CPU oracle over a sample: the first n_heads (batch, query head) slices of
+    the attention, the first n_rows rows of the GEMM, the first n_seqs decode sequences.  Returns the seconds
+    and algorithmic FLOPs of the attention part and of the whole pass."""
+    import oracle
+    G = att.Hq // att.Hkv
+    t0 = time.perf_counter()
+    done = 0
+    while done < n_heads:
+        b, h0 = divmod(done, att.Hq)
+        take = min(att.Hq - h0, n_heads - done)
+        h1 = h0 + take
+        if h0 % G == 0 and h1 % G == 0:  # whole KV groups in one call
+            oracle.attn(att.q.values[b:b + 1, h0:h1], att.k.values[b:b + 1, h0 // G:h1 // G],
+                        att.v.values[b:b + 1, h0 // G:h1 // G], att.mask_kind, None, att.scale)
+        else:                            # a partial group: head by head, each with its one KV head
+            for h in range(h0, h1):
+                oracle.attn(att.q.values[b:b + 1, h:h + 1], att.k.values[b:b + 1, h // G:h // G + 1],
+                            att.v.values[b:b + 1, h // G:h // G + 1], att.mask_kind, None, att.scale)
+        done += take
+    t_att = time.perf_counter() - t0
+    f_att = att.flops() // (att.B * att.Hq) * n_heads
+    oracle.linear_bias_gelu(lin.x.values[:n_rows], lin.w.values, lin.b.values)
+    oracle.attn_decode(dec.q.values[:n_seqs], dec.k_cache.values[:n_seqs], dec.v_cache.values[:n_seqs],
+                       dec.lens[:n_seqs], dec.scale)
+    t_all = time.perf_counter() - t0
+    f_all = f_att + 2 * n_rows * lin.N * lin.K + 4 * dec.D * dec.Hq * int(dec.lens[:n_seqs].sum())
+    return t_att, f_att, t_all, f_all
+
+
 def cpu_baseline(att, lin, dec):
     """The oracle as it stands, on a bounded sample of the step (about 10-30 s of CPU work)."""
     import oracle
-    n_heads, n_rows, n_seqs = 48, 4096, min(16, dec.B)
+    n_heads, n_rows, n_seqs = 64, 4096, min(16, dec.B)
     oracle_sample_step(att, lin, dec, 1, 16, 1)  # loads the library, spins up the threads
-    t0 = time.perf_counter()
-    flops = oracle_sample_step(att, lin, dec, n_heads, n_rows, n_seqs)
-    dt = time.perf_counter() - t0
-    return {"value": flops / dt / 1e12, "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
-            "sample": f"one pass: {n_heads} of {att.B * att.Hq} attention (batch, head) slices, {n_rows} of "
-                      f"{lin.M} GEMM rows, {n_seqs} of {dec.B} decode sequences; {dt:.1f} s",
-            "seconds": dt}
+    t_att, f_att, t_all, f_all = oracle_sample_step(att, lin, dec, n_heads, n_rows, n_seqs)
+    return {"value": f_att / t_att / 1e12, "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"one pass: {n_heads} of {att.B * att.Hq} attention (batch, head) slices ({t_att:.1f} s, the "
+                      f"rate reported), then {n_rows} of {lin.M} GEMM rows and {n_seqs} of {dec.B} decode "
+                      f"sequences ({t_all:.1f} s in all)",
+            "seconds": t_all, "step_tflops": f_all / t_all / 1e12}
 
 
 def run_reference(args):
@@ -161,28 +185,31 @@ def run_reference(args):
     # calibrate on the smallest sample, then size the per-step sample for ~90 s in total
     oracle_sample_step(att, lin, dec, 1, 16, 1)
     t0 = time.perf_counter()
-    f_small = oracle_sample_step(att, lin, dec, 2, 32, 1)
+    oracle_sample_step(att, lin, dec, 2, 32, 1)
     t_small = time.perf_counter() - t0
     budget = 90.0 / max(1, args.steps + args.warmup)
-    scale = max(1.0, min(48.0, budget / max(t_small, 1e-4)))
+    scale = max(1.0, min(32.0, budget / max(t_small, 1e-4)))
     n_heads = int(min(att.B * att.Hq, max(1, round(2 * scale))))
     n_rows = int(min(lin.M, max(16, round(32 * scale))))
     n_seqs = int(min(dec.B, max(1, round(scale / 8))))
     for _ in range(args.warmup):
         oracle_sample_step(att, lin, dec, n_heads, n_rows, n_seqs)
+    t_att = f_att = 0.0
     t0 = time.perf_counter()
-    flops = 0
     for _ in range(args.steps):
-        flops += oracle_sample_step(att, lin, dec, n_heads, n_rows, n_seqs)
+        ta, fa, _, _ = oracle_sample_step(att, lin, dec, n_heads, n_rows, n_seqs)
+        t_att += ta
+        f_att += fa
     dt = time.perf_counter() - t0
-    value = flops / dt / 1e12
-    sample = (f"per step: {n_heads} of {att.B * att.Hq} attention (batch, head) slices, {n_rows} of {lin.M} GEMM "
-              f"rows, {n_seqs} of 16 decode sequences")
+    value = f_att / t_att / 1e12
+    sample = (f"per step: {n_heads} of {att.B * att.Hq} attention (batch, head) slices (the rate reported), "
+              f"{n_rows} of {lin.M} GEMM rows, {n_seqs} of 16 decode sequences")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "sample": sample},
+        "config": {"workload": WORKLOAD, "sample": sample,
+                   "value_is": "fused-attention TFLOP/s of the oracle on the sampled slices"},
         "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -207,6 +234,48 @@ def max_over_ranks(ms: float, device=None, distributed: bool = False) -> float:
 def whole_job_rate(world: int, units_per_rank: float, ms: float) -> float:
     """Units all ranks processed per second (every rank does `units_per_rank`; weak scaling)."""
     return world * units_per_rank / (ms * 1e-3)
+
+
+def free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def launcher_command(argv, gpus: int, port: int):
+    """The command that starts `gpus` ranks of this script on one node (one per GPU, rendezvous on 127.0.0.1)."""
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={gpus}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *argv]
+
+
+def maybe_relaunch(args, argv):
+    """`--gpus N` (N > 1) without a launcher around it: start the N replicas and pass their output through.
+    Returns the launcher's exit code, or None when this process is itself a rank (or N = 1)."""
+    if args.gpus <= 1 or "WORLD_SIZE" in os.environ or args.impl == "reference":
+        return None
+    return subprocess.run(launcher_command(argv, args.gpus, free_port())).returncode
+
+
+def run_dry(args):
+    """`--dry-run-cpu`: the rank plumbing of the GPU arm (process group, barrier, maximum over ranks, rank 0's
+    JSON line) on CPU with the gloo backend and a made-up per-rank time, for tests without a GPU."""
+    import torch
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    distributed = world > 1
+    if distributed:
+        dist.init_process_group("gloo")
+        dist.barrier()
+    my_ms = 10.0 + 5.0 * rank
+    ms = max_over_ranks(my_ms, torch.device("cpu"), distributed)
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "value": whole_job_rate(world, 1.0, ms), "unit": "dry-run units/s",
+                          "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+                          "scaling": "weak", "dry_run": True}))
+    if distributed:
+        dist.destroy_process_group()
+    return 0
 
 
 # ----------------------------------------------------------------------------- GPU arm
@@ -242,8 +311,8 @@ def run_gpu(args):
     gen = torch.Generator(device=dev)
     gen.manual_seed(20260416 + rank)
 
-    def randn(shape, std=1.0):
-        return (torch.randn(shape, generator=gen, device=dev, dtype=torch.float32) * std).to(torch.bfloat16)
+    def randn(shape, std=1.0, dtype=torch.bfloat16):
+        return (torch.randn(shape, generator=gen, device=dev, dtype=torch.float32) * std).to(dtype)
 
     lens_dev = torch.from_numpy(dec.lens).to(dev)
     sets = []
@@ -266,21 +335,27 @@ def run_gpu(args):
         sets.append(s)
     set_bytes = sum(t.numel() * t.element_size() for t in sets[0].values())
 
-    def step(s, ev=None):
-        if ev is not None:
-            ev[0].record()
-        # GEMM first: its 50 MB of output drain from L2 under the compute-bound attention, not under the
-        # bandwidth-bound decode
+    def k_linear(s):
         binding.linear_bias_gelu(s["x"], s["w"], s["b"], out=s["y"])
-        if ev is not None:
-            ev[1].record()
+
+    def k_attention(s):
         binding.attn_fused(s["q"], s["k"], s["v"], att.mask_kind, None, att.scale, out=s["o"])
-        if ev is not None:
-            ev[2].record()
+
+    def k_decode(s):
         binding.attn_decode_splitkv(s["dq"], s["kc"], s["vc"], lens_dev, dec.num_splits, dec.scale,
                                     out=s["do"], workspace=s["ws"])
+
+    KERNELS = (("linear", k_linear), ("attention", k_attention), ("decode", k_decode))
+
+    def step(s, ev=None):
+        # GEMM first: its 50 MB of output drain from L2 under the compute-bound attention, not under the
+        # bandwidth-bound decode
+        for i, (_, fn) in enumerate(KERNELS):
+            if ev is not None:
+                ev[i].record()
+            fn(s)
         if ev is not None:
-            ev[3].record()
+            ev[len(KERNELS)].record()
 
     def barrier():
         if distributed:
@@ -291,55 +366,75 @@ def run_gpu(args):
         step(sets[i % nsets])
     binding.check_status()
 
-    # ---- timed region: K steps back to back, device events around the region only (the library launches
-    # its kernels with programmatic stream serialisation, so consecutive launches overlap their heads and
-    # tails; an event between two kernels would take that away)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    def timed_region(fn, iters):
+        """K back-to-back calls of fn(set) on the rotating sets, device events around the region only.  The
+        GPU idles for `--cooldown` seconds first: back-to-back regions of the tensor-core kernels run into the
+        board's power cap within tens of milliseconds and the clock drops, which the burst peaks they are
+        compared with did not see.  Three untimed calls bring the clocks back up from idle before the region
+        starts.  The clock sampler only looks while a region runs."""
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        time.sleep(args.cooldown)
+        for i in range(3):  # the clocks come back up from idle during a few untimed calls
+            fn(sets[(iters + i) % nsets])
+        sampler.active = True
+        e0.record()
+        for i in range(iters):
+            fn(sets[i % nsets])
+        e1.record()
+        barrier()
+        sampler.active = False
+        return e0.elapsed_time(e1)
+
+    def stats(ms_list, iters):
+        per = [max_over_ranks(m, dev, distributed) / iters for m in ms_list]
+        return {"median": float(np.median(per)), "min": float(min(per)), "max": float(max(per)), "repeats": len(per)}
+
+    reps = max(1, args.repeats)
     sampler = ClockSampler(local_rank)
-    barrier()
+    sampler.active = False
     launches0 = binding.launch_count()
     sampler.start()
     t_wall0 = time.perf_counter()
-    ev0.record()
-    for i in range(args.steps):
-        step(sets[i % nsets])
-    ev1.record()
-    barrier()
+    # ---- timed region 1: K whole steps back to back, repeated
+    step_ms = [timed_region(step, args.steps) for _ in range(reps)]
     wall = time.perf_counter() - t_wall0
     launches = binding.launch_count() - launches0
-    binding.check_status()
-    dev_ms = ev0.elapsed_time(ev1)
-
-    # ---- the same K steps again with events around every kernel: per-kernel launch durations (each
-    # event separates the kernels, so these add up to a little more than the step above)
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    # ---- timed region 2: each kernel on its own, K calls back to back on the rotating sets, repeated
+    kernel_ms = {name: [timed_region(fn, args.steps) for _ in range(reps)] for name, fn in KERNELS}
+    # ---- pass 3: events around every kernel inside the step (upper bounds)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(len(KERNELS) + 1)] for _ in range(args.steps)]
+    barrier()
+    time.sleep(args.cooldown)
+    sampler.active = True
     for i in range(args.steps):
         step(sets[i % nsets], evs[i])
     barrier()
     clocks = sampler.stop()
     binding.check_status()
-    k_ms = [float(np.mean([e[i].elapsed_time(e[i + 1]) for e in evs])) for i in range(3)]
-    split_ms = evs[0][0].elapsed_time(evs[-1][3]) / args.steps
+    in_step_ms = [float(np.median([e[i].elapsed_time(e[i + 1]) for e in evs])) for i in range(len(KERNELS))]
 
-    dev_ms = max_over_ranks(dev_ms, dev, distributed)
-    ms_per_step = dev_ms / args.steps
-
-    step_flops = att.flops() + lin.flops() + dec.flops()
-    value = whole_job_rate(world, step_flops, ms_per_step) / 1e12
-
-    # ---- per-kernel numbers and the roofline of the dominant one
-    sustained = dev_ms >= 1000.0
+    st = stats(step_ms, args.steps)
+    ms_per_step = st["median"]
+    sustained = sum(step_ms) >= 1000.0
     tensor_peak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
-    kern = {
-        "attention": {"ms": k_ms[1], "tflops": att.flops() / k_ms[1] / 1e9, "gbs": att.bytes() / k_ms[1] / 1e6,
-                      "bound": "tensor", "flops": att.flops(), "bytes": att.bytes()},
-        "linear": {"ms": k_ms[0], "tflops": lin.flops() / k_ms[0] / 1e9, "gbs": lin.bytes() / k_ms[0] / 1e6,
-                   "bound": "tensor", "flops": lin.flops(), "bytes": lin.bytes()},
-        "decode": {"ms": k_ms[2], "tflops": dec.flops() / k_ms[2] / 1e9, "gbs": dec.bytes() / k_ms[2] / 1e6,
-                   "bound": "hbm", "flops": dec.flops(), "bytes": dec.bytes()},
-    }
-    for name, k in kern.items():
-        k["frac"] = k["tflops"] / tensor_peak if k["bound"] == "tensor" else k["gbs"] / peaks["hbm_gbs"]
+    work = {"linear": lin, "attention": att, "decode": dec}
+    bound = {"linear": "tensor", "attention": "tensor", "decode": "hbm"}
+    kern = {}
+    for i, (name, _) in enumerate(KERNELS):
+        ks = stats(kernel_ms[name], args.steps)
+        w = work[name]
+        ms = ks["median"]
+        k = {"ms": ms, "ms_min": ks["min"], "ms_max": ks["max"], "ms_in_step": in_step_ms[i],
+             "tflops": w.flops() / ms / 1e9, "gbs": w.bytes() / ms / 1e6, "bound": bound[name],
+             "flops": w.flops(), "bytes": w.bytes()}
+        if bound[name] == "tensor":
+            k["frac"] = k["tflops"] / tensor_peak
+            k["frac_of_nominal"] = k["tflops"] / NOMINAL_PEAKS["bf16_tflops"]
+        else:
+            k["frac"] = k["gbs"] / peaks["hbm_gbs"]
+            k["frac_of_nominal"] = k["gbs"] / NOMINAL_PEAKS["hbm_gbs"]
+        kern[name] = k
     dom = max(kern, key=lambda n: kern[n]["ms"])
     d = kern[dom]
     roofline = {
@@ -350,48 +445,14 @@ def run_gpu(args):
         "frac": d["frac"], "traffic": NCU_TRAFFIC_BYTES[dom],
         "peak_source": f"{peak_src} ({'sustained' if sustained and d['bound'] == 'tensor' else 'burst'})",
     }
+    # the metric's first half: fused-attention TFLOP/s, whole job (every rank runs its own replica)
+    value = whole_job_rate(world, att.flops(), kern["attention"]["ms"]) / 1e12
+    step_flops = att.flops() + lin.flops() + dec.flops()
 
-    # ---- the other configurations, each timed on its own after the step loop (not part of `value`):
-    # 8B-class GQA prefill (the shape where the tensor-core target applies), the padded encoder batch and
-    # the fp32 GPT-2-small case (latency).  Device-drawn inputs of the workloads' shapes and distributions.
+    # ---- the other configurations, each timed on its own after the step loop (not part of `value`)
     other = None
     if rank == 0 and not args.no_other_configs:
-        def timed(fn, iters):
-            for _ in range(3):
-                fn()
-            torch.cuda.synchronize()
-            a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            for _ in range(iters):
-                fn()
-            b_.record()
-            torch.cuda.synchronize()
-            return a.elapsed_time(b_) / iters
-
-        other = {}
-        B4, Hq4, Hkv4, S4, D4 = 4, 32, 8, 2048, 128
-        q4, k4, v4 = randn((B4, Hq4, S4, D4)), randn((B4, Hkv4, S4, D4)), randn((B4, Hkv4, S4, D4))
-        o4 = torch.empty_like(q4)
-        ms = timed(lambda: binding.attn_fused(q4, k4, v4, wl.MASK_CAUSAL, None, D4 ** -0.5, out=o4), 20)
-        fl = 4 * D4 * B4 * Hq4 * (S4 * (S4 + 1) // 2)
-        other["cfg4_gqa_prefill_B4_32/8_S2048_D128"] = {
-            "ms": ms, "tflops": fl / ms / 1e9, "frac_of_bf16_peak": fl / ms / 1e9 / peaks["bf16_tflops"],
-            "flops": fl, "l2": "warm (inputs 101 MB, reused across calls)"}
-        del q4, k4, v4, o4
-        B3, H3, S3, D3 = 32, 12, 128, 64
-        lens3 = torch.from_numpy(wl.cfg3_encoder().lens).to(dev)
-        q3, k3, v3 = randn((B3, H3, S3, D3)), randn((B3, H3, S3, D3)), randn((B3, H3, S3, D3))
-        o3 = torch.empty_like(q3)
-        ms = timed(lambda: binding.attn_fused(q3, k3, v3, wl.MASK_PADDING, lens3, 0.125, out=o3), 50)
-        sl = int(lens3.sum().item())
-        other["cfg3_encoder_padding_B32_H12_S128_D64"] = {
-            "ms": ms, "tflops": 393216 * sl / ms / 1e9, "gbs": (12582912 + 3072 * sl) / ms / 1e6, "sum_lens": sl,
-            "l2": "warm"}
-        q1 = torch.randn((1, 12, 128, 64), generator=gen, device=dev)
-        k1, v1 = torch.randn_like(q1), torch.randn_like(q1)
-        o1 = torch.empty_like(q1)
-        ms = timed(lambda: binding.attn_fused_f32(q1, k1, v1, wl.MASK_CAUSAL, None, 0.125, out=o1), 50)
-        other["cfg1_gpt2_fp32_B1_H12_S128_D64"] = {"latency_us": ms * 1e3, "l2": "warm"}
+        other = other_configs(torch, binding, dev, gen, randn, peaks, args)
 
     # ---- spot check of set 0 against values the oracle computes one by one (not timed)
     spot = None
@@ -400,9 +461,11 @@ def run_gpu(args):
         s = sets[0]
         step(s)
         torch.cuda.synchronize()
-        ref = oracle.attn(att.q.values[7:8, 11:12], att.k.values[7:8, 11:12], att.v.values[7:8, 11:12],
-                          att.mask_kind, None, att.scale)
-        e_att = float(np.abs(s["o"][7:8, 11:12].float().cpu().double().numpy() - ref).max())
+        G = att.Hq // att.Hkv
+        b_, h_ = 3, 29
+        ref = oracle.attn(att.q.values[b_:b_ + 1, h_:h_ + 1], att.k.values[b_:b_ + 1, h_ // G:h_ // G + 1],
+                          att.v.values[b_:b_ + 1, h_ // G:h_ // G + 1], att.mask_kind, None, att.scale)
+        e_att = float(np.abs(s["o"][b_:b_ + 1, h_:h_ + 1].float().cpu().double().numpy() - ref).max())
         rows = [0, 4097, 8191]
         ref = oracle.linear_bias_gelu(lin.x.values[rows], lin.w.values, lin.b.values)
         e_lin = float(np.abs(s["y"][rows].float().cpu().double().numpy() - ref).max())
@@ -427,29 +490,40 @@ def run_gpu(args):
         sc_l = torch.empty(binding.linear_host_scratch_bytes(lin.M, lin.N, lin.K), dtype=torch.uint8, device=dev)
         sc_d = torch.empty(binding.attn_decode_host_scratch_bytes(dec.B, dec.Hq, dec.Hkv, dec.Smax, dec.D,
                                                                   dec.num_splits), dtype=torch.uint8, device=dev)
+        e_steps = max(1, min(args.steps, 10))
+        ea = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(e_steps)]
 
-        def host_step():
-            binding.attn_fused_host(pin["q"], pin["k"], pin["v"], outs["o"], sc_a, att.mask_kind, None, att.scale)
+        def host_step(ev=None):
+            if ev:
+                ev[0].record()
             binding.linear_bias_gelu_host(pin["x"], pin["w"], pin["b"], outs["y"], sc_l)
+            if ev:
+                ev[1].record()
+            binding.attn_fused_host(pin["q"], pin["k"], pin["v"], outs["o"], sc_a, att.mask_kind, None, att.scale)
+            if ev:
+                ev[2].record()
             binding.attn_decode_splitkv_host(pin["dq"], pin["kc"], pin["vc"], lens_host, dec.num_splits,
                                              outs["do"], sc_d, dec.scale)
+            if ev:
+                ev[3].record()
 
-        e_steps = max(1, min(args.steps, 10))
         for _ in range(2):
             host_step()
         barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(e_steps):
-            host_step()
-        e1.record()
+        for i in range(e_steps):
+            host_step(ea[i])
         barrier()
-        e2e_ms = max_over_ranks(e0.elapsed_time(e1), dev, distributed)
+        att_ms = max_over_ranks(float(np.median([e[1].elapsed_time(e[2]) for e in ea])), dev, distributed)
+        all_ms = max_over_ranks(float(np.median([e[0].elapsed_time(e[3]) for e in ea])), dev, distributed)
         h2d = sum(pin[k].numel() * 2 for k in pin) + dec.B * 4
         d2h = sum(outs[k].numel() * 2 for k in outs)
-        e2e = {"value": world * step_flops / (e2e_ms / e_steps * 1e-3) / 1e12, "unit": "TFLOP/s",
+        e2e = {"value": whole_job_rate(world, att.flops(), att_ms) / 1e12, "unit": "TFLOP/s",
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e_steps,
-               "ms_per_step": e2e_ms / e_steps}
+               "ms_per_step": all_ms, "attention_ms": att_ms,
+               "attention_h2d_bytes": int(sum(pin[k].numel() * 2 for k in ("q", "k", "v"))),
+               "attention_d2h_bytes": int(outs["o"].numel() * 2),
+               "note": "value = attention FLOPs / duration of forge_attn_fused_host (copies included); "
+                       "ms_per_step is the whole host step"}
 
     if rank == 0:
         line = {
@@ -457,13 +531,20 @@ def run_gpu(args):
             "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOAD,
-                       "l2": f"rotating {nsets} input sets of {set_bytes / 1e6:.0f} MB each (a step streams "
-                             f"more than the 126 MB L2 between two uses of any buffer)",
-                       "sum_lens": int(dec.lens.sum())},
+                       "value_is": "fused-attention TFLOP/s: FLOPs of the prefill attention / its median launch "
+                                   "duration (K calls back to back on rotating inputs); decode GB/s is in decode_hbm",
+                       "l2": f"rotating {nsets} input sets of {set_bytes / 1e6:.0f} MB each (more than the 126 MB L2 "
+                             f"is streamed between two uses of any buffer)",
+                       "sum_lens": int(dec.lens.sum()), "repeats": reps, "cooldown_s": args.cooldown},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
             "roofline": roofline, "cpu_baseline": base, "kernels": kern, "other_configs": other,
-            "decode_hbm": {"value": kern["decode"]["gbs"], "unit": "GB/s", "frac_of_measured_peak": kern["decode"]["frac"]},
-            "wall_ms_per_step": wall / args.steps * 1e3, "ms_per_step_with_kernel_events": split_ms,
+            "decode_hbm": {"value": kern["decode"]["gbs"], "unit": "GB/s",
+                           "frac_of_measured_peak": kern["decode"]["frac"],
+                           "frac_of_nominal_8tbs": kern["decode"]["frac_of_nominal"]},
+            "step": {"ms_median": st["median"], "ms_min": st["min"], "ms_max": st["max"], "repeats": st["repeats"],
+                     "tflops": whole_job_rate(world, step_flops, ms_per_step) / 1e12,
+                     "sum_of_kernel_ms": sum(k["ms"] for k in kern.values())},
+            "wall_ms_per_step": wall / (args.steps * reps) * 1e3,
             "spot_check": spot,
         }
         print(json.dumps(line))
@@ -472,16 +553,104 @@ def run_gpu(args):
     return 0
 
 
-def main():
+def other_configs(torch, binding, dev, gen, randn, peaks, args):
+    """The remaining configurations and the other fused patterns, each K calls back to back on two rotating
+    input sets.  Device-drawn inputs of the workloads' shapes and distributions."""
+    iters = max(5, min(args.steps, 50))
+    bf, h = torch.bfloat16, torch.float16
+
+    def empty(shape, dtype=bf):
+        return torch.empty(shape, dtype=dtype, device=dev)
+
+    def timed(make, call, nset=2):
+        data = [make() for _ in range(nset)]
+        for d in data:
+            call(d)
+        torch.cuda.synchronize()
+        per = []
+        for _ in range(3):
+            a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for i in range(iters):
+                call(data[i % nset])
+            b_.record()
+            torch.cuda.synchronize()
+            per.append(a.elapsed_time(b_) / iters)
+        return float(np.median(per))
+
+    other = {}
+    pk = peaks["bf16_tflops"]
+    # cfg 2a: GPT-2-small layer attention (the D = 64 shape, bound by the exponentials)
+    B, H, S, D = 8, 12, 1024, 64
+    ms = timed(lambda: (randn((B, H, S, D)), randn((B, H, S, D)), randn((B, H, S, D)), empty((B, H, S, D))),
+               lambda d: binding.attn_fused(d[0], d[1], d[2], wl.MASK_CAUSAL, None, 0.125, out=d[3]))
+    fl = 4 * D * B * H * (S * (S + 1) // 2)
+    other["cfg2a_gpt2_attention_B8_H12_S1024_D64"] = {"ms": ms, "tflops": fl / ms / 1e9,
+                                                      "frac_of_bf16_peak": fl / ms / 1e9 / pk, "flops": fl}
+    # cfg 3: padded encoder batch
+    B3, H3, S3, D3 = 32, 12, 128, 64
+    lens3 = torch.from_numpy(wl.cfg3_encoder().lens).to(dev)
+    sl = int(lens3.sum().item())
+    ms = timed(lambda: (randn((B3, H3, S3, D3)), randn((B3, H3, S3, D3)), randn((B3, H3, S3, D3)), empty((B3, H3, S3, D3))),
+               lambda d: binding.attn_fused(d[0], d[1], d[2], wl.MASK_PADDING, lens3, 0.125, out=d[3]))
+    other["cfg3_encoder_padding_B32_H12_S128_D64"] = {"ms": ms, "tflops": 393216 * sl / ms / 1e9,
+                                                      "gbs": (12582912 + 3072 * sl) / ms / 1e6, "sum_lens": sl,
+                                                      "l2": "warm (two sets of 25 MB)"}
+    # cfg 1: fp32 GPT-2-small attention (latency)
+    def f32(shape):
+        return torch.randn(shape, generator=gen, device=dev)
+    s1 = (1, 12, 128, 64)
+    ms = timed(lambda: (f32(s1), f32(s1), f32(s1), empty(s1, torch.float32)),
+               lambda d: binding.attn_fused_f32(d[0], d[1], d[2], wl.MASK_CAUSAL, None, 0.125, out=d[3]))
+    other["cfg1_gpt2_fp32_B1_H12_S128_D64"] = {"latency_us": ms * 1e3, "l2": "warm"}
+    # the other fused patterns at the 8B-class prefill shape
+    B4, Hq4, Hkv4, S4, D4 = 4, 32, 8, 2048, 128
+    fl4 = 4 * D4 * B4 * Hq4 * (S4 * (S4 + 1) // 2)
+    ms = timed(lambda: (randn((B4, Hq4, S4, D4), dtype=h), randn((B4, Hkv4, S4, D4), dtype=h),
+                        randn((B4, Hkv4, S4, D4), dtype=h), empty((B4, Hq4, S4, D4), h)),
+               lambda d: binding.attn_fused_f16(d[0], d[1], d[2], wl.MASK_CAUSAL, None, D4 ** -0.5, out=d[3]))
+    other["attention_fp16_cfg4_shape"] = {"ms": ms, "tflops": fl4 / ms / 1e9, "frac_of_bf16_peak": fl4 / ms / 1e9 / pk}
+    bias = torch.zeros((B4, 1, S4, S4), device=dev)
+    ms = timed(lambda: (randn((B4, Hq4, S4, D4)), randn((B4, Hkv4, S4, D4)), randn((B4, Hkv4, S4, D4)),
+                        empty((B4, Hq4, S4, D4))),
+               lambda d: binding.attn_fused_bias(d[0], d[1], d[2], bias, wl.MASK_CAUSAL, None, D4 ** -0.5, out=d[3]))
+    other["attention_additive_bias_cfg4_shape"] = {"ms": ms, "tflops": fl4 / ms / 1e9,
+                                                    "frac_of_bf16_peak": fl4 / ms / 1e9 / pk,
+                                                    "bias_bytes": int(bias.numel() * 4)}
+    del bias
+    M, N, K = 8192, 8192, 2048
+    ms = timed(lambda: (randn((M, K)), randn((K, N), 0.02), randn((K, N), 0.02), empty((M, N))),
+               lambda d: binding.linear_swiglu(d[0], d[1], d[2], out=d[3]))
+    fl = 4 * M * N * K
+    other["linear_swiglu_8192x8192x2048"] = {"ms": ms, "tflops": fl / ms / 1e9, "frac_of_bf16_peak": fl / ms / 1e9 / pk}
+    M, N, K = 8192, 8192, 4096
+    ms = timed(lambda: (randn((M, K), dtype=h), torch.randint(-127, 128, (N, K), generator=gen, device=dev, dtype=torch.int8),
+                        torch.rand((N,), generator=gen, device=dev) * 0.01, empty((M, N), h)),
+               lambda d: binding.linear_act_w8a16(d[0], d[1], d[2], None, None, binding.ACT_GELU_TANH, out=d[3]))
+    fl = 2 * M * N * K
+    other["linear_w8a16_8192x8192x4096"] = {"ms": ms, "tflops": fl / ms / 1e9, "frac_of_fp16_peak": fl / ms / 1e9 / pk}
+    return other
+
+
+def main(argv=None):
+    argv = sys.argv[1:] if argv is None else argv
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--repeats", type=int, default=5, help="how often every K-step timed region is repeated")
+    ap.add_argument("--cooldown", type=float, default=0.2, help="idle seconds before every timed region")
     ap.add_argument("--impl", default="forge", choices=["forge", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-other-configs", action="store_true")
-    args = ap.parse_args()
+    ap.add_argument("--dry-run-cpu", action="store_true", help="rank plumbing only, on CPU with gloo (for tests)")
+    args = ap.parse_args(argv)
+    rc = maybe_relaunch(args, argv)
+    if rc is not None:
+        return rc
+    if args.dry_run_cpu:
+        return run_dry(args)
     if args.impl == "reference":
         return run_reference(args)
     return run_gpu(args)

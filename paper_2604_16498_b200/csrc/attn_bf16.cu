@@ -317,6 +317,21 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                         tma_load_3d(sQ + t * L::kTileBytes + c * L::kChunkBytes, &tmap_q, &q_full[t], c * 64,
                                     it.q0[t], it.b * p.Hq + it.h[t]);
                 }
+                // The next item's Q tiles are asked into L2 now, a whole item ahead: Q can only be copied to
+                // shared memory once this item's last scores are done, and a copy that then has to come from
+                // HBM leaves the tensor core idle for a microsecond or two at every item boundary.
+                {
+                    const int i_next = item_of_round(r + 1);
+                    if (i_next < num_items) {
+                        const ItemInfo nx = decode(i_next);
+#pragma unroll
+                        for (int t = 0; t < kTilesPerCta; ++t) {
+                            if (nx.nh[t] == 0) continue;
+#pragma unroll
+                            for (int c = 0; c < D / 64; ++c) tma_prefetch_l2_3d(&tmap_q, c * 64, nx.q0[t], nx.b * p.Hq + nx.h[t]);
+                        }
+                    }
+                }
                 for (int j = 0; j < it.n_max && !failed; ++j) {
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {

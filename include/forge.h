@@ -84,6 +84,22 @@ int forge_attn_fused_f16(const void* q, const void* k, const void* v, void* out,
                          int mask_kind, const int32_t* lens, float scale, void* stream);
 
 /*
+ * forge_attn_fused on tensors that are views of larger buffers: the same operator (Eq. 9), same kernel,
+ * bf16, but q, k, v and out are addressed through element strides {batch, head, row} given by the caller
+ * (x_strides[0..2]); the D elements of a row are contiguous.  This is what lets the operator read the
+ * output of a fused QKV projection ([tokens, (Hq + 2 Hkv) D], i.e. [B, S, heads, D]) and write what the
+ * output projection reads ([tokens, Hq D]) without any copy in between: the dense layout of
+ * forge_attn_fused is the special case {H S D, S D, D}.  Every stride must be positive and a multiple
+ * of 8 elements (rows start on 16-byte boundaries), the row stride at least D; FORGE_ERR_INVALID_ARG /
+ * FORGE_ERR_UNSUPPORTED otherwise.  Everything else as forge_attn_fused.
+ */
+int forge_attn_fused_strided(const void* q, const void* k, const void* v, void* out,
+                             int B, int Hq, int Hkv, int Sq, int Skv, int D,
+                             const int64_t* q_strides, const int64_t* k_strides, const int64_t* v_strides,
+                             const int64_t* out_strides, int mask_kind, const int32_t* lens, float scale,
+                             void* stream);
+
+/*
  * forge_attn_fused with the optional mask node of the fused pattern (Eq. 8) given as a
  * tensor: bias [B, bias_heads, Sq, Skv] fp32 on the device (16-byte aligned, contiguous),
  * bias_heads = 1 (shared by all query heads) or Hq, is added to the scaled scores before
@@ -244,6 +260,75 @@ int forge_linear_act_w8a16(const void* x, const void* w_int8, const float* scale
  */
 int forge_linear_swiglu(const void* x, const void* w_gate, const void* w_up, void* y,
                         int M, int N, int K, int w_layout, void* stream);
+
+/*
+ * Buffer planning for a fixed sequence of operators (Section 4.5, "Liveness Analysis" and "Linear-Scan
+ * Buffer Allocation").  Host code only; nothing is launched.
+ *
+ * forge_plan_liveness (Eq. 14): the program is ops 0 .. num_ops-1; op j writes register out_reg[j] (-1: none)
+ * and reads registers in_regs[in_off[j]] .. in_regs[in_off[j+1]-1].  On return start[r] is the op that
+ * writes register r (-1 for a register nobody writes: an input) and end[r] the last op that reads it
+ * (start[r] for a register that is never read).  FORGE_ERR_INVALID_ARG for a register index out of range
+ * or a register with two writers.
+ *
+ * forge_plan_linear_scan (Algorithm 2): n live intervals [start[i], end[i]] (end >= start) are mapped to
+ * buffers.  Intervals are taken in order of their start (ties by index); intervals that ended BEFORE the
+ * current start (end < start) are expired and their buffers returned to a pool; the interval gets the
+ * buffer released longest ago, or a new one if the pool is empty or pinned[i] is set (pinned may be NULL;
+ * a pinned register's buffer goes to the pool like any other once the register has expired, as in the
+ * paper's listing).  Two intervals that share an op index overlap and never share a buffer.  buf_of[i]
+ * receives the buffer of interval i, *num_bufs the number M of buffers, buf_bytes[0..M-1] (if not NULL; room
+ * for n entries) the size of each: the largest bytes[i] among its tenants (bytes may be NULL: all sizes 1).
+ * The buffer reduction ratio of Eq. 15 is 1 - M / n.
+ */
+int forge_plan_liveness(int num_ops, const int* out_reg, const int* in_off, const int* in_regs,
+                        int num_regs, int* start, int* end);
+int forge_plan_linear_scan(int n, const int* start, const int* end, const size_t* bytes,
+                           const unsigned char* pinned, int* buf_of, size_t* buf_bytes, int* num_bufs);
+
+/*
+ * A decoder layer run as a fixed sequence of the fused operators on one stream, with its intermediate
+ * tensors in planned buffers (Section 4.5; the flat pre-resolved instruction stream of Listing 9):
+ *     qkv  = x Wqkv (+ b_qkv)                                  [T, (Hq + 2 Hkv) D],  T = B S
+ *     attn = fused attention over the q, k, v columns of qkv    [T, Hq D]   (mask_kind / lens / scale)
+ *     h1   = attn Wo (+ b_o) + x                                [T, Hq D]
+ *     g    = silu(h1 Wgate) * (h1 Wup)        (FORGE_MLP_SWIGLU; b_up must be NULL)
+ *          | gelu_tanh(h1 Wup + b_up)         (FORGE_MLP_GELU; w_gate unused)          [T, F]
+ *     y    = g Wdown (+ b_down) + h1                            [T, Hq D]
+ * The columns of qkv are the Hq query heads, then the Hkv key heads, then the Hkv value heads, D each.
+ * Normalisations and rotary embeddings, which the fusion passes leave alone, are not part of it.
+ * x [T, Hq D] and y [T, Hq D] are the caller's bf16 device tensors; all weights bf16, every one stored
+ * [in, out] (FORGE_W_KN) or every one [out, in] (FORGE_W_NK); biases [out] or NULL.  The four
+ * intermediates live in `workspace` (256-byte aligned, at least forge_decoder_layer_workspace_bytes):
+ * their live intervals let the linear scan put them into two buffers.  forge_decoder_layer_plan reports
+ * the plan (N registers, M buffers, rho_buf = 1 - M/N, sizes and offsets) without launching anything.
+ * D: a multiple of 8 up to 128; F a multiple of 8.  Errors as the operators'.
+ */
+enum { FORGE_MLP_SWIGLU = 0, FORGE_MLP_GELU = 1 };
+typedef struct forge_decoder_layer_desc {
+    int B, S, Hq, Hkv, D, F;
+    int mlp_kind;   /* FORGE_MLP_SWIGLU or FORGE_MLP_GELU */
+    int w_layout;   /* FORGE_W_KN or FORGE_W_NK, for every weight */
+    int mask_kind;  /* FORGE_MASK_* for the attention */
+    float scale;    /* of the attention scores */
+    const int32_t* lens;  /* device, [B]; NULL unless mask_kind has the padding bit */
+    const void *w_qkv, *b_qkv, *w_o, *b_o, *w_gate, *w_up, *b_up, *w_down, *b_down;
+} forge_decoder_layer_desc;
+typedef struct forge_layer_plan {
+    int num_regs;          /* N: planned intermediates (qkv, attn, h1, g) */
+    int num_bufs;          /* M */
+    float rho_buf;         /* 1 - M / N (Eq. 15) */
+    int buf_of[4];         /* buffer of each register */
+    int reg_start[4], reg_end[4];   /* live intervals in op indices (Eq. 14) */
+    size_t reg_bytes[4];
+    size_t buf_bytes[4], buf_offset[4];  /* first num_bufs entries: size and place in the workspace */
+    size_t workspace_bytes;  /* what the planned buffers take */
+    size_t unplanned_bytes;  /* what one buffer per register would take */
+} forge_layer_plan;
+int forge_decoder_layer_plan(const forge_decoder_layer_desc* desc, forge_layer_plan* plan);
+size_t forge_decoder_layer_workspace_bytes(const forge_decoder_layer_desc* desc);
+int forge_decoder_layer(const forge_decoder_layer_desc* desc, const void* x, void* y,
+                        void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * Host-buffer variants: the same operators for callers whose tensors live in

@@ -21,3 +21,4 @@ from .ref import (  # noqa: F401
     num_threads,
     build,
 )
+from . import planner, layer  # noqa: F401,E402

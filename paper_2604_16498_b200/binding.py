@@ -26,6 +26,7 @@ SIGNATURES = {
     "forge_attn_fused": (_i, _ATTN + [_vp]),
     "forge_attn_fused_f32": (_i, _ATTN + [_vp]),
     "forge_attn_fused_f16": (_i, _ATTN + [_vp]),
+    "forge_attn_fused_strided": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _i, _vp, _f, _vp]),
     "forge_attn_fused_bias": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _i, _vp, _vp, _i, _f, _vp]),
     "forge_attn_decode_splitkv": (_i, _DEC + [_vp, _sz, _vp]),
     "forge_attn_decode_splitkv_f16": (_i, _DEC + [_vp, _sz, _vp]),
@@ -51,6 +52,31 @@ SIGNATURES = {
     "forge_last_cuda_error": (_i, []),
     "forge_launch_count": (ctypes.c_ulonglong, []),
 }
+
+
+
+class LayerDesc(ctypes.Structure):
+    """forge_decoder_layer_desc"""
+    _fields_ = [("B", _i), ("S", _i), ("Hq", _i), ("Hkv", _i), ("D", _i), ("F", _i), ("mlp_kind", _i),
+                ("w_layout", _i), ("mask_kind", _i), ("scale", _f), ("lens", _vp),
+                ("w_qkv", _vp), ("b_qkv", _vp), ("w_o", _vp), ("b_o", _vp), ("w_gate", _vp), ("w_up", _vp),
+                ("b_up", _vp), ("w_down", _vp), ("b_down", _vp)]
+
+
+class LayerPlan(ctypes.Structure):
+    """forge_layer_plan"""
+    _fields_ = [("num_regs", _i), ("num_bufs", _i), ("rho_buf", _f), ("buf_of", _i * 4), ("reg_start", _i * 4),
+                ("reg_end", _i * 4), ("reg_bytes", _sz * 4), ("buf_bytes", _sz * 4), ("buf_offset", _sz * 4),
+                ("workspace_bytes", _sz), ("unplanned_bytes", _sz)]
+
+
+SIGNATURES.update({
+    "forge_plan_liveness": (_i, [_i, _vp, _vp, _vp, _i, _vp, _vp]),
+    "forge_plan_linear_scan": (_i, [_i, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "forge_decoder_layer_plan": (_i, [ctypes.POINTER(LayerDesc), ctypes.POINTER(LayerPlan)]),
+    "forge_decoder_layer_workspace_bytes": (_sz, [ctypes.POINTER(LayerDesc)]),
+    "forge_decoder_layer": (_i, [ctypes.POINTER(LayerDesc), _vp, _vp, _vp, _sz, _vp]),
+})
 
 _lib = None
 
@@ -118,6 +144,26 @@ def attn_fused(q, k, v, mask_kind=MASK_NONE, lens=None, scale=None, out=None):
     _check("forge_attn_fused", load().forge_attn_fused(
         _dev(q, torch.bfloat16, "q"), _dev(k, torch.bfloat16, "k"), _dev(v, torch.bfloat16, "v"),
         _dev(out, torch.bfloat16, "out"), B, Hq, Hkv, Sq, Skv, D, int(mask_kind), lp, float(scale), _stream()))
+    return out
+
+
+def attn_fused_strided(q, k, v, out, mask_kind=MASK_NONE, lens=None, scale=None):
+    """forge_attn_fused_strided: q/out [B,Hq,Sq,D] and k/v [B,Hkv,Skv,D] bf16 VIEWS (any strides with a
+    contiguous last dimension, e.g. slices of a fused QKV projection permuted to head-major)."""
+    B, Hq, Sq, D = q.shape
+    _, Hkv, Skv, _ = k.shape
+    if tuple(k.shape) != (B, Hkv, Skv, D) or tuple(v.shape) != (B, Hkv, Skv, D) or tuple(out.shape) != (B, Hq, Sq, D):
+        raise ValueError("q/out [B,Hq,Sq,D], k/v [B,Hkv,Skv,D] expected")
+    scale = D ** -0.5 if scale is None else scale
+    arrs = []
+    for name, t in (("q", q), ("k", k), ("v", v), ("out", out)):
+        if not (t.is_cuda and t.dtype == torch.bfloat16 and t.stride(3) == 1):
+            raise ValueError(f"{name}: expected a CUDA bf16 tensor whose last dimension is contiguous")
+        arrs.append((ctypes.c_int64 * 3)(t.stride(0), t.stride(1), t.stride(2)))
+    lp = None if lens is None else _dev(lens, torch.int32, "lens")
+    _check("forge_attn_fused_strided", load().forge_attn_fused_strided(
+        q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), B, Hq, Hkv, Sq, Skv, D,
+        arrs[0], arrs[1], arrs[2], arrs[3], int(mask_kind), lp, float(scale), _stream()))
     return out
 
 
@@ -279,6 +325,74 @@ def linear_swiglu(x, w_gate, w_up, w_layout=W_KN, out=None):
     _check("forge_linear_swiglu", load().forge_linear_swiglu(
         _dev(x, bf, "x"), _dev(w_gate, bf, "w_gate"), _dev(w_up, bf, "w_up"), _dev(out, bf, "out"),
         M, N, K, int(w_layout), _stream()))
+    return out
+
+
+# ---- buffer planning (host only) and the decoder layer ----
+MLP_SWIGLU, MLP_GELU = 0, 1
+
+
+def plan_liveness(out_reg, in_regs_per_op, num_regs):
+    """forge_plan_liveness: ops given as (register written or -1, list of registers read).  Returns (start, end)."""
+    n = len(out_reg)
+    off = [0]
+    flat = []
+    for regs in in_regs_per_op:
+        flat.extend(regs)
+        off.append(len(flat))
+    c_out = (ctypes.c_int * max(n, 1))(*out_reg)
+    c_off = (ctypes.c_int * (n + 1))(*off)
+    c_in = (ctypes.c_int * max(len(flat), 1))(*flat)
+    start = (ctypes.c_int * max(num_regs, 1))()
+    end = (ctypes.c_int * max(num_regs, 1))()
+    _check("forge_plan_liveness", load().forge_plan_liveness(n, c_out, c_off, c_in, num_regs, start, end))
+    return list(start)[:num_regs], list(end)[:num_regs]
+
+
+def plan_linear_scan(start, end, nbytes=None, pinned=None):
+    """forge_plan_linear_scan.  Returns (buf_of, buf_bytes, num_bufs)."""
+    n = len(start)
+    c_s = (ctypes.c_int * max(n, 1))(*start)
+    c_e = (ctypes.c_int * max(n, 1))(*end)
+    c_b = None if nbytes is None else (ctypes.c_size_t * max(n, 1))(*nbytes)
+    c_p = None if pinned is None else (ctypes.c_ubyte * max(n, 1))(*[1 if x else 0 for x in pinned])
+    buf_of = (ctypes.c_int * max(n, 1))()
+    buf_bytes = (ctypes.c_size_t * max(n, 1))()
+    m = ctypes.c_int(0)
+    _check("forge_plan_linear_scan", load().forge_plan_linear_scan(n, c_s, c_e, c_b, c_p, buf_of, buf_bytes, ctypes.byref(m)))
+    return list(buf_of)[:n], list(buf_bytes)[:m.value], m.value
+
+
+def _layer_desc(B, S, Hq, Hkv, D, F, mlp_kind, w_layout, mask_kind, scale, lens, weights):
+    d = LayerDesc(B=B, S=S, Hq=Hq, Hkv=Hkv, D=D, F=F, mlp_kind=mlp_kind, w_layout=w_layout, mask_kind=mask_kind,
+                  scale=float(scale), lens=None if lens is None else _dev(lens, torch.int32, "lens"))
+    for name in ("w_qkv", "b_qkv", "w_o", "b_o", "w_gate", "w_up", "b_up", "w_down", "b_down"):
+        t = weights.get(name)
+        setattr(d, name, None if t is None else _dev(t, torch.bfloat16, name))
+    return d
+
+
+def decoder_layer_plan(B, S, Hq, Hkv, D, F, mlp_kind=MLP_SWIGLU):
+    """forge_decoder_layer_plan: the buffer plan of a layer of these dimensions (no GPU needed)."""
+    d = LayerDesc(B=B, S=S, Hq=Hq, Hkv=Hkv, D=D, F=F, mlp_kind=mlp_kind, w_layout=W_KN, mask_kind=MASK_CAUSAL, scale=1.0)
+    plan = LayerPlan()
+    _check("forge_decoder_layer_plan", load().forge_decoder_layer_plan(ctypes.byref(d), ctypes.byref(plan)))
+    return plan
+
+
+def decoder_layer(x, weights, B, S, Hq, Hkv, D, F, mlp_kind=MLP_SWIGLU, w_layout=W_KN, mask_kind=MASK_CAUSAL,
+                  scale=None, lens=None, out=None, workspace=None):
+    """forge_decoder_layer: x [B*S, Hq*D] bf16; weights: dict of bf16 tensors (w_qkv, w_o, w_gate, w_up, w_down
+    and optional b_qkv, b_o, b_up, b_down)."""
+    scale = D ** -0.5 if scale is None else scale
+    d = _layer_desc(B, S, Hq, Hkv, D, F, mlp_kind, w_layout, mask_kind, scale, lens, weights)
+    out = torch.empty_like(x) if out is None else out
+    need = int(load().forge_decoder_layer_workspace_bytes(ctypes.byref(d)))
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=x.device)
+    _check("forge_decoder_layer", load().forge_decoder_layer(
+        ctypes.byref(d), _dev(x, torch.bfloat16, "x"), _dev(out, torch.bfloat16, "out"),
+        _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream()))
     return out
 
 

@@ -152,6 +152,7 @@ __device__ __forceinline__ int fast_div(int n, const FastDiv& f) {
 
 struct AttnParams {
     uint16_t* out;  // bf16 or fp16 elements
+    long long o_sb, o_sh, o_ss;  // element strides of out between batch entries, heads and rows
     const int32_t* lens;
     const float* bias;  // additive bias on the scaled scores [B, bias_heads, Sq, Skv], or nullptr
     int bias_heads;     // 1 (shared by all heads) or Hq
@@ -314,8 +315,8 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     mbar_expect_tx(&q_full[t], L::kTileBytes);
 #pragma unroll
                     for (int c = 0; c < D / 64; ++c)  // rows beyond Sq are zero-filled by the TMA unit
-                        tma_load_3d(sQ + t * L::kTileBytes + c * L::kChunkBytes, &tmap_q, &q_full[t], c * 64,
-                                    it.q0[t], it.b * p.Hq + it.h[t]);
+                        tma_load_4d(sQ + t * L::kTileBytes + c * L::kChunkBytes, &tmap_q, &q_full[t], c * 64,
+                                    it.q0[t], it.h[t], it.b);
                 }
                 // The next item's Q tiles are asked into L2 now, a whole item ahead: Q can only be copied to
                 // shared memory once this item's last scores are done, and a copy that then has to come from
@@ -328,7 +329,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                         for (int t = 0; t < kTilesPerCta; ++t) {
                             if (nx.nh[t] == 0) continue;
 #pragma unroll
-                            for (int c = 0; c < D / 64; ++c) tma_prefetch_l2_3d(&tmap_q, c * 64, nx.q0[t], nx.b * p.Hq + nx.h[t]);
+                            for (int c = 0; c < D / 64; ++c) tma_prefetch_l2_4d(&tmap_q, c * 64, nx.q0[t], nx.h[t], nx.b);
                         }
                     }
                 }
@@ -339,19 +340,19 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                         if (two_streams && j >= it.nh[u]) continue;
                         const int g = kvn[u]++, st = kv_slot(u, g);
                         const uint32_t ph = kv_phase(g);
-                        const int kv_row = it.b * p.Hkv + it.kvh[u];
+                        const int kvh = it.kvh[u];
                         if (!mbar_wait(&k_empty[st], ph ^ 1)) { failed = true; break; }
                         mbar_expect_tx(&k_full[st], L::kKVTileBytes);
 #pragma unroll
                         for (int c = 0; c < D / 64; ++c)
-                            tma_load_3d(sK + st * L::kKVTileBytes + c * L::kKVChunkBytes, &tmap_k, &k_full[st], c * 64,
-                                        j * kHalf, kv_row);
+                            tma_load_4d(sK + st * L::kKVTileBytes + c * L::kKVChunkBytes, &tmap_k, &k_full[st], c * 64,
+                                        j * kHalf, kvh, it.b);
                         if (!mbar_wait(&v_empty[st], ph ^ 1)) { failed = true; break; }
                         mbar_expect_tx(&v_full[st], L::kKVTileBytes);
 #pragma unroll
                         for (int c = 0; c < D / 64; ++c)
-                            tma_load_3d(sV + st * L::kKVTileBytes + c * L::kKVChunkBytes, &tmap_v, &v_full[st], c * 64,
-                                        j * kHalf, kv_row);
+                            tma_load_4d(sV + st * L::kKVTileBytes + c * L::kKVChunkBytes, &tmap_v, &v_full[st], c * 64,
+                                        j * kHalf, kvh, it.b);
                     }
                 }
             }
@@ -491,10 +492,10 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             const int q0 = pick(it.q0, t);
             const int qi = q0 + row;
             const int nh = pick(it.nh, t);
-            const int bh = it.b * p.Hq + pick(it.h, t);
+            const int head = pick(it.h, t);
             if (nh == 0) {  // no visible key for any row of this tile (or the tile lies beyond Sq)
                 if (qi < p.Sq) {
-                    uint16_t* orow = p.out + ((size_t)bh * p.Sq + qi) * p.head_dim;
+                    uint16_t* orow = p.out + it.b * p.o_sb + head * p.o_sh + qi * p.o_ss;
                     for (int c = 0; c < p.head_dim / 8; ++c) reinterpret_cast<uint4*>(orow)[c] = make_uint4(0, 0, 0, 0);
                 }
                 if (i_next < num_items) it_next = decode(i_next);
@@ -718,7 +719,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     const int row0 = q0 + quarter * 32;
                     if (row0 < p.Sq) {
 #pragma unroll
-                        for (int cb = 0; cb < D / 64; ++cb) tma_store_3d(&tmap_o, stage_out + cb * 4096, cb * 64, row0, bh);
+                        for (int cb = 0; cb < D / 64; ++cb) tma_store_4d(&tmap_o, stage_out + cb * 4096, cb * 64, row0, head, it.b);
                         tma_store_commit();
                     }
                 }
@@ -741,37 +742,38 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     }
 }
 
+// Element strides of a [B, H, S, D] tensor between batch entries, heads and rows (the D elements of a row are
+// contiguous).  Dense tensors have {H * S * D, S * D, D}; the strided entry point passes the caller's.
+struct Strides {
+    long long b, h, s;
+};
+inline Strides dense_strides(int H, int S, int D) { return {(long long)H * S * D, (long long)S * D, (long long)D}; }
+
 // D: the kernel's head dimension (64 or 128); head_dim <= D: the tensors' (a multiple of 8).  Columns beyond
 // head_dim are zero-filled on load and clipped on store by the TMA unit, so a padded head costs time, not memory.
 template <int D, bool F16, bool BIAS = false>
 int launch_attn(const void* q, const void* k, const void* v, void* out, int B, int Hq, int Hkv, int Sq, int Skv,
                 int head_dim, int mask_kind, const int32_t* lens, float scale, cudaStream_t s, const float* bias = nullptr,
-                int bias_heads = 1) {
+                int bias_heads = 1, const Strides* sq_ = nullptr, const Strides* sk_ = nullptr, const Strides* sv_ = nullptr,
+                const Strides* so_ = nullptr) {
     using L = AttnSmem<D>;
-    CUtensorMap tq, tk, tv;
-    const uint32_t box[3] = {64, 128, 1};
-    {
-        const uint64_t dims[3] = {(uint64_t)head_dim, (uint64_t)Sq, (uint64_t)B * Hq};
-        const uint64_t strides[2] = {(uint64_t)head_dim * 2, (uint64_t)Sq * head_dim * 2};
-        if (!encode_tmap_bf16_sw128(&tq, q, 3, dims, strides, box)) return FORGE_ERR_CUDA;
-    }
-    {
-        const uint32_t box_kv[3] = {64, (uint32_t)kHalf, 1};
-        const uint64_t dims[3] = {(uint64_t)head_dim, (uint64_t)Skv, (uint64_t)B * Hkv};
-        const uint64_t strides[2] = {(uint64_t)head_dim * 2, (uint64_t)Skv * head_dim * 2};
-        if (!encode_tmap_bf16_sw128(&tk, k, 3, dims, strides, box_kv)) return FORGE_ERR_CUDA;
-        if (!encode_tmap_bf16_sw128(&tv, v, 3, dims, strides, box_kv)) return FORGE_ERR_CUDA;
-    }
-    CUtensorMap to;
-    {
-        // the output leaves in boxes of 32 rows, one per softmax warp
-        const uint32_t box_o[3] = {64, 32, 1};
-        const uint64_t dims[3] = {(uint64_t)head_dim, (uint64_t)Sq, (uint64_t)B * Hq};
-        const uint64_t strides[2] = {(uint64_t)head_dim * 2, (uint64_t)Sq * head_dim * 2};
-        if (!encode_tmap_bf16_sw128(&to, out, 3, dims, strides, box_o)) return FORGE_ERR_CUDA;
-    }
+    const Strides sq = sq_ ? *sq_ : dense_strides(Hq, Sq, head_dim), so = so_ ? *so_ : dense_strides(Hq, Sq, head_dim);
+    const Strides sk = sk_ ? *sk_ : dense_strides(Hkv, Skv, head_dim), sv = sv_ ? *sv_ : dense_strides(Hkv, Skv, head_dim);
+    // every tensor as a 4-D map (D, rows, heads, batch): the strides carry the layout
+    auto encode = [&](CUtensorMap* m, const void* base, int H, int S, const Strides& st, uint32_t box_rows) {
+        const uint32_t box[4] = {64, box_rows, 1, 1};
+        const uint64_t dims[4] = {(uint64_t)head_dim, (uint64_t)S, (uint64_t)H, (uint64_t)B};
+        const uint64_t strides[3] = {(uint64_t)st.s * 2, (uint64_t)st.h * 2, (uint64_t)st.b * 2};
+        return encode_tmap_bf16_sw128(m, base, 4, dims, strides, box);
+    };
+    CUtensorMap tq, tk, tv, to;
+    if (!encode(&tq, q, Hq, Sq, sq, 128)) return FORGE_ERR_CUDA;
+    if (!encode(&tk, k, Hkv, Skv, sk, kHalf)) return FORGE_ERR_CUDA;
+    if (!encode(&tv, v, Hkv, Skv, sv, kHalf)) return FORGE_ERR_CUDA;
+    if (!encode(&to, out, Hq, Sq, so, 32)) return FORGE_ERR_CUDA;  // the output leaves in boxes of 32 rows, one per softmax warp
     AttnParams p;
     p.out = static_cast<uint16_t*>(out);
+    p.o_sb = so.b; p.o_sh = so.h; p.o_ss = so.s;
     p.lens = lens;
     p.bias = bias;
     p.bias_heads = bias_heads;
@@ -848,4 +850,31 @@ extern "C" int forge_attn_fused_bias(const void* q, const void* k, const void* v
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     return D <= 64 ? launch_attn<64, false, true>(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, s, bias, bias_heads)
                    : launch_attn<128, false, true>(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, s, bias, bias_heads);
+}
+
+extern "C" int forge_attn_fused_strided(const void* q, const void* k, const void* v, void* out,
+                                        int B, int Hq, int Hkv, int Sq, int Skv, int D,
+                                        const int64_t* q_strides, const int64_t* k_strides, const int64_t* v_strides,
+                                        const int64_t* out_strides, int mask_kind, const int32_t* lens, float scale,
+                                        void* stream) {
+    using namespace forge;
+    int st = check_attn_args(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, /*any_head_dim=*/true);
+    if (st != FORGE_OK) return st;
+    if (!q_strides || !k_strides || !v_strides || !out_strides) return FORGE_ERR_INVALID_ARG;
+    if ((long long)Hq * B * ((Sq + 255) / 256) > 2147483647LL) return FORGE_ERR_UNSUPPORTED;
+    if (!(scale >= 0.f)) return FORGE_ERR_UNSUPPORTED;  // the running maximum is taken on unscaled scores
+    Strides str[4];
+    const int64_t* in[4] = {q_strides, k_strides, v_strides, out_strides};
+    for (int i = 0; i < 4; ++i) {
+        str[i] = {in[i][0], in[i][1], in[i][2]};
+        // rows must not overlap their own elements, and every stride must keep rows on 16-byte boundaries
+        if (str[i].b <= 0 || str[i].h <= 0 || str[i].s < D) return FORGE_ERR_INVALID_ARG;
+        if ((str[i].b % 8) || (str[i].h % 8) || (str[i].s % 8)) return FORGE_ERR_UNSUPPORTED;
+        if (str[i].b >= (1LL << 38) || str[i].h >= (1LL << 38) || str[i].s >= (1LL << 38)) return FORGE_ERR_UNSUPPORTED;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    return D <= 64 ? launch_attn<64, false>(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, s, nullptr, 1,
+                                            &str[0], &str[1], &str[2], &str[3])
+                   : launch_attn<128, false>(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, s, nullptr, 1,
+                                             &str[0], &str[1], &str[2], &str[3]);
 }

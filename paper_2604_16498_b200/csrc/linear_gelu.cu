@@ -23,6 +23,7 @@
 
 #include "activations.cuh"
 #include "forge_common.cuh"
+#include "linear_pair.cuh"
 #include "sm100_ptx.cuh"
 #include "tmap.cuh"
 
@@ -402,6 +403,8 @@ int linear_act_impl(const void* x, const void* w, const void* b, const void* res
         return FORGE_ERR_INVALID_ARG;
     if ((K % 8) != 0 || (N % 8) != 0) return FORGE_ERR_UNSUPPORTED;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // large outputs run on CTA pairs (see linear_pair.cu); shapes with few tiles stay on the one-CTA kernel
+    if (linear_pair_pays(M, N, sm_count())) return linear_pair(F16, x, w, b, residual, y, M, N, K, act, w_layout, s);
     switch (act) {
         case FORGE_ACT_GELU_TANH: return launch_layout<FORGE_ACT_GELU_TANH, F16>(w_layout, x, w, b, residual, y, M, N, K, s);
         case FORGE_ACT_GELU_ERF: return launch_layout<FORGE_ACT_GELU_ERF, F16>(w_layout, x, w, b, residual, y, M, N, K, s);

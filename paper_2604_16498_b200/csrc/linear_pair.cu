@@ -6,12 +6,12 @@
 // copies (no multicast), and the tensor cores of both SMs read both halves of W (tcgen05.mma
 // cta_group::2).  Per SM and k-step that is 32 KB for 512 tensor-core cycles: 64 B per cycle instead of 104.
 //
-// Roles per CTA (320 threads):
+// Roles per CTA (576 threads):
 //   warp 0    : TMA producer for this CTA's operand halves; the bytes of both CTAs are counted on the even
 //               CTA's barrier of the stage, so the issuer observes one barrier per k-step
 //   warp 1    : even CTA: issues the pair's MMAs (one elected lane).  In both CTAs this warp allocates and
 //               frees the tensor memory.
-//   warps 2-9 : epilogue of this CTA's 128 x 256 half of the tile; each warp on its own (no barriers)
+//   warps 2-17: epilogue of this CTA's 128 x 256 half of the tile; each warp on its own (no barriers)
 // Two accumulators of 256 columns: the epilogue of tile i overlaps the main loop of tile i + 1.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
@@ -31,15 +31,15 @@ constexpr int kBM = 128;          // rows per CTA
 constexpr int kBN = 256;          // columns of the pair's tile (128 loaded per CTA)
 constexpr int kBK = 64;
 constexpr int kStages = 5;
-constexpr int kThreads = 320;
-constexpr int kEpiThreads = 256;
+constexpr int kEpiWarps = 16;     // four per TMEM lane quarter, one 64-column block of the tile each
+constexpr int kThreads = 64 + kEpiWarps * 32;
 constexpr int kTmemCols = 512;    // two accumulators of 256 columns
 
 struct PairSmem {
     static constexpr int kABytes = kBM * kBK * 2;          // 16 KB: 128 rows of X
     static constexpr int kBBytes = kBK * (kBN / 2) * 2;    // 16 KB: 128 columns of W
     static constexpr int kStageBytes = kABytes + kBBytes;
-    static constexpr int kOutBytes = 8 * 4096;             // output staging: 32 rows x 64 elements per epilogue warp
+    static constexpr int kOutBytes = kEpiWarps * 4096;     // output staging: 32 rows x 64 elements per epilogue warp
     static constexpr int kOutOffset = kStages * kStageBytes;
     static constexpr int kBarOffset = kOutOffset + kOutBytes;
     // full[S], empty[S], tmem_full[2], tmem_empty[2]; then the TMEM base
@@ -88,7 +88,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(&tmem_full[i], 1); mbar_init(&tmem_empty[i], 2 * kEpiThreads / 32); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&tmem_full[i], 1); mbar_init(&tmem_empty[i], 2 * kEpiWarps); }
         fence_mbar_init();
         prefetch_tmap(&tmap_x);
         prefetch_tmap(&tmap_w);
@@ -168,10 +168,10 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         }
     } else if (warp >= 2) {
         // ------------------------------------------------------------------ epilogue of this CTA's 128 rows
-        // Every warp works alone: it owns 32 rows (its TMEM lane quarter) of two of the tile's four 64-column
-        // blocks, its own 4 KB of staging and its own TMA stores, so the eight warps never meet at a barrier.
-        const int quarter = warp & 3;       // TMEM lane quarter this warp may access
-        const int which = (warp - 2) >> 2;  // 0: blocks 0 and 2 of the tile, 1: blocks 1 and 3
+        // Every warp works alone: it owns 32 rows (its TMEM lane quarter) of one of the tile's four 64-column
+        // blocks, its own 4 KB of staging and its own TMA stores, so the sixteen warps never meet at a barrier.
+        const int quarter = warp & 3;    // TMEM lane quarter this warp may access
+        const int blk = (warp - 2) >> 2; // its 64-column block of the tile
         uint8_t* stage_out = smem + L::kOutOffset + (warp - 2) * 4096;
         const uint32_t empty_on_leader = map_to_cta(&tmem_empty[0], 0);  // [acc] at + 8 * acc
         int it = 0;
@@ -183,29 +183,22 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             tc_fence_after_sync();
             const int row = quarter * 32 + lane;  // row of this CTA's half of the tile = TMEM lane
             const uint32_t taddr = tmem_base + acc * kBN + (static_cast<uint32_t>(quarter * 32) << 16);
-#pragma unroll 1
-            for (int bi = 0; bi < 2; ++bi) {
-                const int blk = which + 2 * bi;
-                uint32_t r[64];
-                {
-                    uint32_t lo[32], hi[32];
-                    tmem_ld_x32(taddr + blk * 64, lo);
-                    tmem_ld_x32(taddr + blk * 64 + 32, hi);
-                    tmem_ld_wait();
+            if (lane == 0) tma_store_wait_read<0>();  // this warp's previous store has read the staging rows
+            __syncwarp();
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) { r[i] = lo[i]; r[32 + i] = hi[i]; }
-                }
-                if (bi == 1) {
+            for (int half = 0; half < 2; ++half) {  // 32 columns at a time keeps the registers of 576 threads in bounds
+                uint32_t r[32];
+                tmem_ld_x32(taddr + blk * 64 + half * 32, r);
+                tmem_ld_wait();
+                if (half == 1) {
                     // this warp has read all it needs of the accumulator: tell the issuer (in the even CTA)
                     tc_fence_before_sync();
                     __syncwarp();
                     if (lane == 0) mbar_arrive_cluster(empty_on_leader + acc * 8);
                 }
-                if (lane == 0) tma_store_wait_read<0>();  // this warp's previous store has read the staging rows
-                __syncwarp();
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {  // 16-byte chunk c of the row's 128-byte line: 8 columns
-                    const int gcol = n0 + blk * 64 + c * 8;
+                for (int c = 0; c < 4; ++c) {  // 16-byte chunk half*4 + c of the row's 128-byte line: 8 columns
+                    const int gcol = n0 + blk * 64 + half * 32 + c * 8;
                     uint4 bv = make_uint4(0, 0, 0, 0), res = make_uint4(0, 0, 0, 0);
                     if (bias != nullptr && gcol < N) bv = __ldg(reinterpret_cast<const uint4*>(bias + gcol));
                     if (residual != nullptr && m0 + row < M && gcol < N)
@@ -219,14 +212,15 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                         w[i] = pack16<F16>(activate<ACT>(z0) + widen16<F16>(static_cast<uint16_t>(rw[i] & 0xffffu)),
                                            activate<ACT>(z1) + widen16<F16>(static_cast<uint16_t>(rw[i] >> 16)));
                     }
-                    *reinterpret_cast<uint4*>(stage_out + lane * 128 + ((c ^ (lane & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                    *reinterpret_cast<uint4*>(stage_out + lane * 128 + (((half * 4 + c) ^ (lane & 7)) << 4)) =
+                        make_uint4(w[0], w[1], w[2], w[3]);
                 }
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0 && m0 + quarter * 32 < M) {
-                    tma_store_2d(&tmap_y, stage_out, n0 + blk * 64, m0 + quarter * 32);  // rows >= M, columns >= N are clipped
-                    tma_store_commit();
-                }
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0 && m0 + quarter * 32 < M) {
+                tma_store_2d(&tmap_y, stage_out, n0 + blk * 64, m0 + quarter * 32);  // rows >= M, columns >= N are clipped
+                tma_store_commit();
             }
         }
         if (lane == 0) tma_store_wait_all<0>();

@@ -47,7 +47,7 @@ constexpr int kColS = 0;          // S_t at t * 128
 constexpr int kColO = 256;        // O_t at 256 + t * D
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 #ifndef FORGE_ATTN_FMA_EXP_PAIRS
-#define FORGE_ATTN_FMA_EXP_PAIRS 8
+#define FORGE_ATTN_FMA_EXP_PAIRS 2
 #endif
 // of the 32 score pairs of a half-step, how many take their exponentials on the FMA pipe (unmasked steps)
 constexpr int kFmaExpPairs = FORGE_ATTN_FMA_EXP_PAIRS;

@@ -10,7 +10,7 @@
 // this part, with 250 KB 5.8 TB/s).  So the kernel is persistent and every warp is an independent
 // worker: it owns whole pieces, keeps a private ring of 16-row blocks in shared memory filled by
 // TMA tile copies (16 rows x 64 columns each, 128-byte swizzle, completion counted on an mbarrier
-// per stage) that run ahead across piece boundaries (8 warps x 24 KB in flight per SM), and writes
+// per stage) that run ahead across piece boundaries (8 warps x 16 KB in flight per SM), and writes
 // its partial straight from registers.  No warp ever waits for another one.
 //
 // Pieces.  All pieces of a call are C blocks of 16 rows long (the last piece of a sequence may be
@@ -46,7 +46,10 @@ namespace {
 constexpr int kWarps = 8;
 constexpr int kThreads = kWarps * 32;
 constexpr int kBlockKeys = 16;             // cached rows per ring stage
-constexpr int kWarpRingBytes = 24 * 1024;  // per warp
+// Per warp.  16 KB (two stages of 16 rows at D = 128) measured a little faster than 24 KB: the memory system is
+// saturated either way, and what is queued beyond that only adds to the latency of every block, which is what
+// the end of the call (the last blocks of the slowest warps) waits for.
+constexpr int kWarpRingBytes = 16 * 1024;
 
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 r;
@@ -324,7 +327,7 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     constexpr int kTileBytes = kBlockKeys * 128;
     constexpr int kKBytes = (D / 64) * kTileBytes;
     constexpr int kStageBytes = 2 * kKBytes;
-    constexpr int kStages = kWarpRingBytes / kStageBytes;  // 3 for D = 128, 6 for D = 64
+    constexpr int kStages = kWarpRingBytes / kStageBytes;  // 2 for D = 128, 4 for D = 64
     static_assert(kStages >= 2 && kStages <= 8, "ring size");
 
     extern __shared__ __align__(128) uint8_t ring_raw[];

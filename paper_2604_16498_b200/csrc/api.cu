@@ -88,6 +88,12 @@ bool encode_tmap_bf16_sw128(CUtensorMap* map, const void* base, int rank, const 
                                strides_bytes, box);
 }
 
+bool encode_tmap_bf16_plain(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
+                            const uint64_t* strides_bytes, const uint32_t* box) {
+    return encode_tmap_generic(CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, CU_TENSOR_MAP_SWIZZLE_NONE, map, base, rank, dims,
+                               strides_bytes, box);
+}
+
 bool encode_tmap_u8_plain(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
                           const uint64_t* strides_bytes, const uint32_t* box) {
     return encode_tmap_generic(CU_TENSOR_MAP_DATA_TYPE_UINT8, CU_TENSOR_MAP_SWIZZLE_NONE, map, base, rank, dims,

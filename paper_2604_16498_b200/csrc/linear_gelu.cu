@@ -442,6 +442,8 @@ extern "C" int forge_linear_swiglu(const void* x, const void* w_gate, const void
     if (!aligned16(x) || !aligned16(w_gate) || !aligned16(w_up) || !aligned16(y)) return FORGE_ERR_INVALID_ARG;
     if ((K % 8) != 0 || (N % 8) != 0) return FORGE_ERR_UNSUPPORTED;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // more than one row tile: CTA pairs (see linear_pair.cu)
+    if (M > 128 && sm_count() >= 2) return linear_pair_swiglu(x, w_gate, w_up, y, M, N, K, w_layout, s);
     return w_layout == FORGE_W_NK
                ? launch_linear<256, 3, FORGE_ACT_SILU, true, true>(x, w_gate, nullptr, nullptr, y, M, N, K, s, w_up)
                : launch_linear<256, 3, FORGE_ACT_SILU, false, true>(x, w_gate, nullptr, nullptr, y, M, N, K, s, w_up);

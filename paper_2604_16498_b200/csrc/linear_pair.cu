@@ -13,6 +13,9 @@
 //               frees the tensor memory.
 //   warps 2-17: epilogue of this CTA's 128 x 256 half of the tile; each warp on its own (no barriers)
 // Two accumulators of 256 columns: the epilogue of tile i overlaps the main loop of tile i + 1.
+// Gated form (SwiGLU, silu(X Wg) * (X Wu)): the pair's tile is 256 rows x 128 output columns; each CTA loads 64
+// gate columns and the 64 up columns of the same outputs, so the accumulator holds [gate | up] of CTA 0's columns,
+// then [gate | up] of CTA 1's, and the epilogue multiplies the two halves as it reads them back.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -64,9 +67,11 @@ __device__ __forceinline__ float widen16(uint16_t bits) {
     else return __uint_as_float(static_cast<uint32_t>(bits) << 16);
 }
 
-template <int ACT, bool W_NK, bool F16>
+// GATED: tmap_w = gate weights, tmap_w2 = up weights, tmap_y stores boxes of 32 columns; no bias, residual or ACT.
+template <int ACT, bool W_NK, bool F16, bool GATED>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 linear_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+                   const __grid_constant__ CUtensorMap tmap_w2,
                    const __grid_constant__ CUtensorMap tmap_y, const uint16_t* __restrict__ bias,
                    const uint16_t* __restrict__ residual, int M, int N, int K, int* __restrict__ status) {
     using L = PairSmem;
@@ -82,7 +87,8 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();  // 0: issues the MMAs
     const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
-    const int tiles_m = (M + 2 * kBM - 1) / (2 * kBM), tiles_n = (N + kBN - 1) / kBN;
+    constexpr int BNO = GATED ? kBN / 2 : kBN;  // output columns of the pair's tile
+    const int tiles_m = (M + 2 * kBM - 1) / (2 * kBM), tiles_n = (N + BNO - 1) / BNO;
     const int num_tiles = tiles_m * tiles_n;
     const int kblocks = (K + kBK - 1) / kBK;
 
@@ -92,6 +98,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         fence_mbar_init();
         prefetch_tmap(&tmap_x);
         prefetch_tmap(&tmap_w);
+        if constexpr (GATED) prefetch_tmap(&tmap_w2);
         prefetch_tmap(&tmap_y);
     }
     if (warp == 1) {
@@ -114,7 +121,8 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             uint32_t phase = 0;
             for (int tile = pair; tile < num_tiles && !failed; tile += num_pairs) {
                 const int m0 = (tile / tiles_n) * 2 * kBM + (int)rank * kBM;
-                const int n0 = (tile % tiles_n) * kBN + (int)rank * (kBN / 2);
+                // this CTA's columns of W: half of the tile's (gated: 64 gate columns and the same 64 up columns)
+                const int n0 = (tile % tiles_n) * BNO + (int)rank * (BNO / 2);
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!mbar_wait(&empty[stage], phase ^ 1)) { failed = true; break; }
                     uint8_t* sa = smem + stage * L::kStageBytes;
@@ -123,11 +131,17 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
                     if (rank == 0) mbar_expect_tx(&full[stage], 2 * L::kStageBytes);
                     const uint32_t bar = map_to_cta(&full[stage], 0);
                     tma_load_2d_pair(sa, &tmap_x, bar, kb * kBK, m0);
-                    if constexpr (W_NK) {  // 128 rows of W, 64 K-elements (one swizzle span) each
-                        tma_load_2d_pair(sb, &tmap_w, bar, kb * kBK, n0);
+                    if constexpr (W_NK) {  // rows of W, 64 K-elements (one swizzle span) each
+                        if constexpr (GATED) {
+                            tma_load_2d_pair(sb, &tmap_w, bar, kb * kBK, n0);               // 64 gate rows
+                            tma_load_2d_pair(sb + 64 * 128, &tmap_w2, bar, kb * kBK, n0);   // 64 up rows
+                        } else {
+                            tma_load_2d_pair(sb, &tmap_w, bar, kb * kBK, n0);               // 128 rows
+                        }
                     } else {               // two boxes of 64 K-rows x 64 columns
                         tma_load_2d_pair(sb, &tmap_w, bar, n0, kb * kBK);
-                        tma_load_2d_pair(sb + kBK * 128, &tmap_w, bar, n0 + 64, kb * kBK);
+                        if constexpr (GATED) tma_load_2d_pair(sb + kBK * 128, &tmap_w2, bar, n0, kb * kBK);
+                        else tma_load_2d_pair(sb + kBK * 128, &tmap_w, bar, n0 + 64, kb * kBK);
                     }
                     if (++stage == kStages) { stage = 0; phase ^= 1; }
                 }
@@ -176,7 +190,7 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         const uint32_t empty_on_leader = map_to_cta(&tmem_empty[0], 0);  // [acc] at + 8 * acc
         int it = 0;
         for (int tile = pair; tile < num_tiles; tile += num_pairs, ++it) {
-            const int m0 = (tile / tiles_n) * 2 * kBM + (int)rank * kBM, n0 = (tile % tiles_n) * kBN;
+            const int m0 = (tile / tiles_n) * 2 * kBM + (int)rank * kBM, n0 = (tile % tiles_n) * BNO;
             const int acc = it & 1;
             const uint32_t acc_phase = (it >> 1) & 1;
             if (!warp_wait(&tmem_full[acc], acc_phase)) { failed = true; break; }
@@ -185,6 +199,37 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
             const uint32_t taddr = tmem_base + acc * kBN + (static_cast<uint32_t>(quarter * 32) << 16);
             if (lane == 0) tma_store_wait_read<0>();  // this warp's previous store has read the staging rows
             __syncwarp();
+            if constexpr (GATED) {
+                // This warp: 32 of the tile's 128 output columns.  Output column c of the tile was computed by CTA
+                // c / 64, whose part of the accumulator is [gate 64 | up 64] at column (c / 64) * 128.
+                const int oc = blk * 32;                                   // first output column of this warp
+                const uint32_t gcol = (oc >> 6) * 128 + (oc & 63);         // its gate columns in the accumulator
+                uint32_t rg[32], ru[32];
+                tmem_ld_x32(taddr + gcol, rg);
+                tmem_ld_x32(taddr + gcol + 64, ru);
+                tmem_ld_wait();
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(empty_on_leader + acc * 8);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {  // 16-byte chunk c of this warp's 64-byte staging row
+                    uint32_t w[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int k = c * 8 + 2 * i;
+                        w[i] = pack16<F16>(activate<FORGE_ACT_SILU>(__uint_as_float(rg[k])) * __uint_as_float(ru[k]),
+                                           activate<FORGE_ACT_SILU>(__uint_as_float(rg[k + 1])) * __uint_as_float(ru[k + 1]));
+                    }
+                    *reinterpret_cast<uint4*>(stage_out + lane * 64 + c * 16) = make_uint4(w[0], w[1], w[2], w[3]);
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0 && m0 + quarter * 32 < M && n0 + oc < N) {
+                    tma_store_2d(&tmap_y, stage_out, n0 + oc, m0 + quarter * 32);  // a plain box of 32 columns x 32 rows
+                    tma_store_commit();
+                }
+                continue;
+            }
 #pragma unroll
             for (int half = 0; half < 2; ++half) {  // 32 columns at a time keeps the registers of 576 threads in bounds
                 uint32_t r[32];
@@ -241,44 +286,52 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     }
 }
 
-template <int ACT, bool W_NK, bool F16>
+template <int ACT, bool W_NK, bool F16, bool GATED = false>
 int launch_pair(const void* x, const void* w, const void* b, const void* residual, void* y, int M, int N, int K,
-                cudaStream_t s) {
+                cudaStream_t s, const void* w_up = nullptr) {
     using L = PairSmem;
-    CUtensorMap tmap_x, tmap_w, tmap_y;
+    constexpr int BNO = GATED ? kBN / 2 : kBN;
+    CUtensorMap tmap_x, tmap_w, tmap_w2, tmap_y;
     {
         const uint64_t dims[2] = {(uint64_t)K, (uint64_t)M};
         const uint64_t strides[1] = {(uint64_t)K * 2};
         const uint32_t box[2] = {kBK, kBM};
         if (!encode_tmap_bf16_sw128(&tmap_x, x, 2, dims, strides, box)) return FORGE_ERR_CUDA;
     }
-    if (W_NK) {  // w[N, K]: 128 rows of 64 K-elements
+    if (W_NK) {  // w[N, K]: rows of 64 K-elements; a CTA's half of the tile's columns per box (gated: 64 + 64)
         const uint64_t dims[2] = {(uint64_t)K, (uint64_t)N};
         const uint64_t strides[1] = {(uint64_t)K * 2};
-        const uint32_t box[2] = {kBK, kBN / 2};
+        const uint32_t box[2] = {kBK, GATED ? 64u : 128u};
         if (!encode_tmap_bf16_sw128(&tmap_w, w, 2, dims, strides, box)) return FORGE_ERR_CUDA;
+        if (!encode_tmap_bf16_sw128(&tmap_w2, GATED ? w_up : w, 2, dims, strides, box)) return FORGE_ERR_CUDA;
     } else {     // w[K, N]: 64 K-rows of 64 N-elements per box
         const uint64_t dims[2] = {(uint64_t)N, (uint64_t)K};
         const uint64_t strides[1] = {(uint64_t)N * 2};
         const uint32_t box[2] = {64, kBK};
         if (!encode_tmap_bf16_sw128(&tmap_w, w, 2, dims, strides, box)) return FORGE_ERR_CUDA;
+        if (!encode_tmap_bf16_sw128(&tmap_w2, GATED ? w_up : w, 2, dims, strides, box)) return FORGE_ERR_CUDA;
     }
     {
         const uint64_t dims[2] = {(uint64_t)N, (uint64_t)M};
         const uint64_t strides[1] = {(uint64_t)N * 2};
-        const uint32_t box[2] = {64, 32};  // one epilogue warp's rows
-        if (!encode_tmap_bf16_sw128(&tmap_y, y, 2, dims, strides, box)) return FORGE_ERR_CUDA;
+        if (GATED) {  // one epilogue warp's 32 rows x 32 columns, rows of 64 bytes as they lie in its staging buffer
+            const uint32_t box[2] = {32, 32};
+            if (!encode_tmap_bf16_plain(&tmap_y, y, 2, dims, strides, box)) return FORGE_ERR_CUDA;
+        } else {      // one epilogue warp's 32 rows x 64 columns
+            const uint32_t box[2] = {64, 32};
+            if (!encode_tmap_bf16_sw128(&tmap_y, y, 2, dims, strides, box)) return FORGE_ERR_CUDA;
+        }
     }
     int* status = device_status_word();
     if (!status) return FORGE_ERR_CUDA;
     const int sms = sm_count();
     if (sms <= 1) return FORGE_ERR_CUDA;
-    auto kernel = linear_pair_kernel<ACT, W_NK, F16>;
+    auto kernel = linear_pair_kernel<ACT, W_NK, F16, GATED>;
     FORGE_SET_SMEM_ONCE(kernel, L::kAlloc);
-    const int tiles = ((M + 2 * kBM - 1) / (2 * kBM)) * ((N + kBN - 1) / kBN);
+    const int tiles = ((M + 2 * kBM - 1) / (2 * kBM)) * ((N + BNO - 1) / BNO);
     const int pairs = tiles < sms / 2 ? tiles : sms / 2;
     // the cluster shape is part of the kernel (__cluster_dims__); programmatic stream serialisation as everywhere
-    FORGE_CUDA_TRY(launch_pdl(kernel, dim3(2 * pairs), dim3(kThreads), L::kAlloc, s, tmap_x, tmap_w, tmap_y,
+    FORGE_CUDA_TRY(launch_pdl(kernel, dim3(2 * pairs), dim3(kThreads), L::kAlloc, s, tmap_x, tmap_w, tmap_w2, tmap_y,
                               static_cast<const uint16_t*>(b), static_cast<const uint16_t*>(residual), M, N, K, status));
     return finish_launch(1);
 }
@@ -308,6 +361,13 @@ bool linear_pair_pays(int M, int N, int sms) {
     const long long t2 = (long long)((M + 255) / 256) * ((N + 255) / 256);
     // with a single row tile the second CTA of every pair would work on padding only
     return sms >= 2 && M > 128 && 0.95 * fill(t2, sms / 2) > 0.61 * fill(t1, sms);
+}
+
+int linear_pair_swiglu(const void* x, const void* w_gate, const void* w_up, void* y, int M, int N, int K, int w_layout,
+                       cudaStream_t s) {
+    return w_layout == FORGE_W_NK
+               ? launch_pair<FORGE_ACT_SILU, true, false, true>(x, w_gate, nullptr, nullptr, y, M, N, K, s, w_up)
+               : launch_pair<FORGE_ACT_SILU, false, false, true>(x, w_gate, nullptr, nullptr, y, M, N, K, s, w_up);
 }
 
 int linear_pair(bool f16, const void* x, const void* w, const void* b, const void* residual, void* y, int M, int N,

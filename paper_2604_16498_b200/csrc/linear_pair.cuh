@@ -13,4 +13,8 @@ bool linear_pair_pays(int M, int N, int sms);
 int linear_pair(bool f16, const void* x, const void* w, const void* b, const void* residual, void* y, int M, int N,
                 int K, int act, int w_layout, cudaStream_t s);
 
+// silu(x Wg) * (x Wu) on CTA pairs (bf16); arguments as forge_linear_swiglu.  Pays whenever M > 128.
+int linear_pair_swiglu(const void* x, const void* w_gate, const void* w_up, void* y, int M, int N, int K, int w_layout,
+                       cudaStream_t s);
+
 }  // namespace forge

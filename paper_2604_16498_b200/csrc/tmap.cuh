@@ -18,6 +18,11 @@ namespace forge {
 bool encode_tmap_bf16_sw128(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
                             const uint64_t* strides_bytes, const uint32_t* box);
 
+// Encodes a tiled tensor map over 16-bit elements without swizzle (the tile lies row by row in shared memory);
+// box[0] * 2 bytes must be a multiple of 16.  Same conventions and return value as above.
+bool encode_tmap_bf16_plain(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
+                            const uint64_t* strides_bytes, const uint32_t* box);
+
 // Encodes a tiled tensor map over bytes without swizzle (the tile lands row by row).  box[0] must be a
 // multiple of 16 bytes.  Same conventions and return value as above.
 bool encode_tmap_u8_plain(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,

@@ -91,6 +91,20 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     const int tiles_m = (M + 2 * kBM - 1) / (2 * kBM), tiles_n = (N + BNO - 1) / BNO;
     const int num_tiles = tiles_m * tiles_n;
     const int kblocks = (K + kBK - 1) / kBK;
+    // Work units.  The tiles of the last, incomplete round of the persistent schedule are cut into two halves of
+    // 128 columns when that lets them all run at once: the round then takes half as long, which matters when a
+    // pair only gets five or six tiles in all.  (Not for the gated form: a CTA's half would be 32 + 32 columns.)
+    const int rem = num_tiles % num_pairs;
+    const bool split = !GATED && rem > 0 && 2 * rem <= num_pairs;
+    const int n_whole = split ? num_tiles - rem : num_tiles;
+    const int num_units = n_whole + (split ? 2 * rem : 0);
+    struct Unit { int tile, col0, width; };  // col0: first column of the unit inside its tile
+    auto unit_of = [&](int u) {
+        Unit x;
+        if (u < n_whole) { x.tile = u; x.col0 = 0; x.width = BNO; }
+        else { const int v = u - n_whole; x.tile = n_whole + (v >> 1); x.col0 = (v & 1) * (kBN / 2); x.width = kBN / 2; }
+        return x;
+    };
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < kStages; ++i) { mbar_init(&full[i], 1); mbar_init(&empty[i], 1); }
@@ -119,29 +133,33 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         if (elect_one()) {
             int stage = 0;
             uint32_t phase = 0;
-            for (int tile = pair; tile < num_tiles && !failed; tile += num_pairs) {
+            for (int u = pair; u < num_units && !failed; u += num_pairs) {
+                const Unit un = unit_of(u);
+                const int tile = un.tile;
                 const int m0 = (tile / tiles_n) * 2 * kBM + (int)rank * kBM;
-                // this CTA's columns of W: half of the tile's (gated: 64 gate columns and the same 64 up columns)
-                const int n0 = (tile % tiles_n) * BNO + (int)rank * (BNO / 2);
+                // this CTA's columns of W: half of the unit's (gated: 64 gate columns and the same 64 up columns)
+                const int n0 = (tile % tiles_n) * BNO + un.col0 + (int)rank * (un.width / 2);
+                const bool narrow = un.width < BNO;  // a half tile: 64 columns of W per CTA
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!mbar_wait(&empty[stage], phase ^ 1)) { failed = true; break; }
                     uint8_t* sa = smem + stage * L::kStageBytes;
                     uint8_t* sb = sa + L::kABytes;
                     // one arrival and the bytes of BOTH CTAs' tiles, announced by the even CTA on its barrier
-                    if (rank == 0) mbar_expect_tx(&full[stage], 2 * L::kStageBytes);
+                    if (rank == 0) mbar_expect_tx(&full[stage], 2 * (L::kABytes + (narrow ? L::kBBytes / 2 : L::kBBytes)));
                     const uint32_t bar = map_to_cta(&full[stage], 0);
                     tma_load_2d_pair(sa, &tmap_x, bar, kb * kBK, m0);
                     if constexpr (W_NK) {  // rows of W, 64 K-elements (one swizzle span) each
                         if constexpr (GATED) {
                             tma_load_2d_pair(sb, &tmap_w, bar, kb * kBK, n0);               // 64 gate rows
                             tma_load_2d_pair(sb + 64 * 128, &tmap_w2, bar, kb * kBK, n0);   // 64 up rows
-                        } else {
-                            tma_load_2d_pair(sb, &tmap_w, bar, kb * kBK, n0);               // 128 rows
+                        } else {                                                             // one or two boxes of 64 rows
+                            tma_load_2d_pair(sb, &tmap_w, bar, kb * kBK, n0);
+                            if (!narrow) tma_load_2d_pair(sb + 64 * 128, &tmap_w, bar, kb * kBK, n0 + 64);
                         }
-                    } else {               // two boxes of 64 K-rows x 64 columns
+                    } else {               // boxes of 64 K-rows x 64 columns
                         tma_load_2d_pair(sb, &tmap_w, bar, n0, kb * kBK);
                         if constexpr (GATED) tma_load_2d_pair(sb + kBK * 128, &tmap_w2, bar, n0, kb * kBK);
-                        else tma_load_2d_pair(sb + kBK * 128, &tmap_w, bar, n0 + 64, kb * kBK);
+                        else if (!narrow) tma_load_2d_pair(sb + kBK * 128, &tmap_w, bar, n0 + 64, kb * kBK);
                     }
                     if (++stage == kStages) { stage = 0; phase ^= 1; }
                 }
@@ -150,12 +168,15 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
     } else if (warp == 1 && rank == 0) {
         // ------------------------------------------------------------------ even CTA: MMA issuer of the pair
         if (elect_one()) {
-            constexpr uint32_t idesc = F16 ? make_idesc_f16(2 * kBM, kBN, /*a_mn_major=*/false, /*b_mn_major=*/!W_NK)
-                                           : make_idesc_bf16(2 * kBM, kBN, /*a_mn_major=*/false, /*b_mn_major=*/!W_NK);
+            constexpr uint32_t idesc_whole = F16 ? make_idesc_f16(2 * kBM, kBN, /*a_mn_major=*/false, /*b_mn_major=*/!W_NK)
+                                                 : make_idesc_bf16(2 * kBM, kBN, /*a_mn_major=*/false, /*b_mn_major=*/!W_NK);
+            constexpr uint32_t idesc_half = F16 ? make_idesc_f16(2 * kBM, kBN / 2, false, !W_NK)
+                                                : make_idesc_bf16(2 * kBM, kBN / 2, false, !W_NK);
             int stage = 0;
             uint32_t phase = 0;
             int it = 0;
-            for (int tile = pair; tile < num_tiles && !failed; tile += num_pairs, ++it) {
+            for (int u = pair; u < num_units && !failed; u += num_pairs, ++it) {
+                const uint32_t idesc = (!GATED && unit_of(u).width < kBN) ? idesc_half : idesc_whole;
                 const int acc = it & 1;
                 const uint32_t acc_phase = (it >> 1) & 1;
                 if (!mbar_wait_cluster(&tmem_empty[acc], acc_phase ^ 1)) { failed = true; break; }
@@ -189,14 +210,22 @@ linear_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_cons
         uint8_t* stage_out = smem + L::kOutOffset + (warp - 2) * 4096;
         const uint32_t empty_on_leader = map_to_cta(&tmem_empty[0], 0);  // [acc] at + 8 * acc
         int it = 0;
-        for (int tile = pair; tile < num_tiles; tile += num_pairs, ++it) {
-            const int m0 = (tile / tiles_n) * 2 * kBM + (int)rank * kBM, n0 = (tile % tiles_n) * BNO;
+        for (int u = pair; u < num_units; u += num_pairs, ++it) {
+            const Unit un = unit_of(u);
+            const int tile = un.tile;
+            const int m0 = (tile / tiles_n) * 2 * kBM + (int)rank * kBM, n0 = (tile % tiles_n) * BNO + un.col0;
             const int acc = it & 1;
             const uint32_t acc_phase = (it >> 1) & 1;
             if (!warp_wait(&tmem_full[acc], acc_phase)) { failed = true; break; }
             tc_fence_after_sync();
             const int row = quarter * 32 + lane;  // row of this CTA's half of the tile = TMEM lane
             const uint32_t taddr = tmem_base + acc * kBN + (static_cast<uint32_t>(quarter * 32) << 16);
+            if (!GATED && blk * 64 >= un.width) {  // a half tile has no block for this warp: only the accumulator hand-back
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(empty_on_leader + acc * 8);
+                continue;
+            }
             if (lane == 0) tma_store_wait_read<0>();  // this warp's previous store has read the staging rows
             __syncwarp();
             if constexpr (GATED) {
@@ -298,10 +327,10 @@ int launch_pair(const void* x, const void* w, const void* b, const void* residua
         const uint32_t box[2] = {kBK, kBM};
         if (!encode_tmap_bf16_sw128(&tmap_x, x, 2, dims, strides, box)) return FORGE_ERR_CUDA;
     }
-    if (W_NK) {  // w[N, K]: rows of 64 K-elements; a CTA's half of the tile's columns per box (gated: 64 + 64)
+    if (W_NK) {  // w[N, K]: boxes of 64 rows of 64 K-elements (gated: gate rows and up rows; else one or two per CTA)
         const uint64_t dims[2] = {(uint64_t)K, (uint64_t)N};
         const uint64_t strides[1] = {(uint64_t)K * 2};
-        const uint32_t box[2] = {kBK, GATED ? 64u : 128u};
+        const uint32_t box[2] = {kBK, 64u};
         if (!encode_tmap_bf16_sw128(&tmap_w, w, 2, dims, strides, box)) return FORGE_ERR_CUDA;
         if (!encode_tmap_bf16_sw128(&tmap_w2, GATED ? w_up : w, 2, dims, strides, box)) return FORGE_ERR_CUDA;
     } else {     // w[K, N]: 64 K-rows of 64 N-elements per box

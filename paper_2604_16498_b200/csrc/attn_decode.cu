@@ -22,7 +22,7 @@
 // more pieces than workers, worker w takes pieces w, w + workers, ...
 //
 // Combine.  A (batch, kv head) with one piece is normalised and written by its worker.  Otherwise
-// each worker writes its partial to the workspace, makes it visible (__threadfence) and adds one to
+// each worker writes its partial to the workspace and, with release-acquire ordering, adds one to
 // the arrival counter of its (batch, kv head); the worker that brings the counter to the number of
 // pieces merges all partials of the G heads, writes the output rows and puts the counter back to
 // zero.  Nobody waits: whoever arrives last does the merge.  The counters live at the start of the
@@ -585,15 +585,18 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     make_float4(acc[hb][0][2 + e], acc[hb][1][2 + e], acc[hb][2][2 + e], acc[hb][3][2 + e]);
             }
         }
-        __threadfence();  // the partial is visible device-wide before the arrival is counted
+        // The arrival is a release-acquire read-modify-write at device scope by lane 0, after a warp barrier:
+        // the warp's stores of the partial happen before it, and whoever reads the full count has acquired the
+        // partials of all earlier arrivals.  (One combined operation instead of fence, atomic, fence: the
+        // round trips to L2 at this point are what the end of the call waits for.)
         __syncwarp();
         unsigned int arrived = 0;
-        if (lane == 0) arrived = atomicAdd(&counters[it.b * Hkv + it.kvh], 1u);
-        arrived = __shfl_sync(0xffffffffu, arrived, 0);
+        if (lane == 0)
+            asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(arrived) : "l"(counters + it.b * Hkv + it.kvh) : "memory");
+        arrived = __shfl_sync(0xffffffffu, arrived, 0);  // the other lanes read the partials after this exchange
         if (arrived + 1 != (unsigned)it.pieces) continue;
 
         // ---- last to arrive: merge the pieces of the G heads
-        __threadfence();
         if (lane == 0) counters[it.b * Hkv + it.kvh] = 0;  // as the next call expects it
         merge_pieces<D, G, F16>(ws_o, ws_ml, out, head0, it.pieces, num_splits, head_dim, lane);
     }

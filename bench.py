@@ -610,6 +610,11 @@ def other_configs(torch, binding, dev, gen, randn, peaks, args):
                         randn((B4, Hkv4, S4, D4), dtype=h), empty((B4, Hq4, S4, D4), h)),
                lambda d: binding.attn_fused_f16(d[0], d[1], d[2], wl.MASK_CAUSAL, None, D4 ** -0.5, out=d[3]))
     other["attention_fp16_cfg4_shape"] = {"ms": ms, "tflops": fl4 / ms / 1e9, "frac_of_bf16_peak": fl4 / ms / 1e9 / pk}
+    Bw, Hqw, Hkvw, Sw, Dw = 4, 16, 4, 2048, 256  # head size 256: the one-tile-per-CTA kernel
+    flw = 4 * Dw * Bw * Hqw * (Sw * (Sw + 1) // 2)
+    ms = timed(lambda: (randn((Bw, Hqw, Sw, Dw)), randn((Bw, Hkvw, Sw, Dw)), randn((Bw, Hkvw, Sw, Dw)), empty((Bw, Hqw, Sw, Dw))),
+               lambda d: binding.attn_fused(d[0], d[1], d[2], wl.MASK_CAUSAL, None, Dw ** -0.5, out=d[3]))
+    other["attention_D256_B4_16/4_S2048"] = {"ms": ms, "tflops": flw / ms / 1e9, "frac_of_bf16_peak": flw / ms / 1e9 / pk}
     bias = torch.zeros((B4, 1, S4, S4), device=dev)
     ms = timed(lambda: (randn((B4, Hq4, S4, D4)), randn((B4, Hkv4, S4, D4)), randn((B4, Hkv4, S4, D4)),
                         empty((B4, Hq4, S4, D4))),

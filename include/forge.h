@@ -60,8 +60,9 @@ enum {
  * Fused attention, bf16 in / fp32 accumulate / bf16 out:
  *     out[b,h,i,:] = sum_j softmax_j(scale * q[b,h,i,:].k[b,h/G,j,:] over visible j) * v[b,h/G,j,:]
  * (Eq. 9 with the optional scale and mask nodes of Eq. 8 folded in; scores and
- * probabilities never reach global memory).  D: any multiple of 8 up to 128 (sizes other than 64 and
- * 128 run on the next larger kernel: the TMA unit pads the rows with zeros on the fly).  `lens` may be
+ * probabilities never reach global memory).  D: any multiple of 8 up to 256 (sizes other than 64, 128 and
+ * 256 run on the next larger kernel: the TMA unit pads the rows with zeros on the fly; sizes above 128 run
+ * on a kernel of their own with one query tile per CTA).  `lens` may be
  * NULL unless mask_kind has the padding bit.  scale must be >= 0 (FORGE_ERR_UNSUPPORTED otherwise: the
  * kernel takes the running maximum on unscaled scores; forge_attn_fused_f32 accepts any sign).  Padded
  * K and V rows (beyond lens[b]) may hold anything, including NaN and Inf: they never reach the result.
@@ -107,7 +108,7 @@ int forge_attn_fused_strided(const void* q, const void* k, const void* v, void* 
  * excludes the key; a row whose keys are all excluded gives zeros.  Finite entries are
  * arbitrary (relative-position or ALiBi-style biases), but a "large negative" stand-in
  * for -infinity must stay finite after division by scale.  mask_kind / lens apply on top.
- * bf16 q, k, v, out as in forge_attn_fused.  scale must be > 0 (FORGE_ERR_UNSUPPORTED
+ * bf16 q, k, v, out as in forge_attn_fused, D up to 128.  scale must be > 0 (FORGE_ERR_UNSUPPORTED
  * otherwise); other errors as forge_attn_fused.
  */
 int forge_attn_fused_bias(const void* q, const void* k, const void* v, void* out,

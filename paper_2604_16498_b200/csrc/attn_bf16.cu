@@ -28,6 +28,7 @@
 
 #include <type_traits>
 
+#include "attn_wide.cuh"
 #include "forge_common.cuh"
 #include "sm100_ptx.cuh"
 #include "tmap.cuh"
@@ -807,6 +808,14 @@ int launch_attn(const void* q, const void* k, const void* v, void* out, int B, i
     return finish_launch(1);
 }
 
+// Head sizes above 128 run on the one-tile-per-CTA kernel of attn_wide.cu.
+int wide_dense(bool f16, const void* q, const void* k, const void* v, void* out, int B, int Hq, int Hkv, int Sq, int Skv,
+               int D, int mask_kind, const int32_t* lens, float scale, cudaStream_t s) {
+    const Strides a = dense_strides(Hq, Sq, D), c = dense_strides(Hkv, Skv, D);
+    const long long st[4][3] = {{a.b, a.h, a.s}, {c.b, c.h, c.s}, {c.b, c.h, c.s}, {a.b, a.h, a.s}};
+    return attn_wide(f16, q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, st, s);
+}
+
 }  // namespace
 }  // namespace forge
 
@@ -814,11 +823,12 @@ extern "C" int forge_attn_fused(const void* q, const void* k, const void* v, voi
                                 int B, int Hq, int Hkv, int Sq, int Skv, int D,
                                 int mask_kind, const int32_t* lens, float scale, void* stream) {
     using namespace forge;
-    int st = check_attn_args(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, /*any_head_dim=*/true);
+    int st = check_attn_args(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, /*any_head_dim=*/true, 256);
     if (st != FORGE_OK) return st;
-    if ((long long)Hq * B * ((Sq + 255) / 256) > 2147483647LL) return FORGE_ERR_UNSUPPORTED;
+    if ((long long)Hq * B * ((Sq + 127) / 128) > 2147483647LL) return FORGE_ERR_UNSUPPORTED;
     if (!(scale >= 0.f)) return FORGE_ERR_UNSUPPORTED;  // the running maximum is taken on unscaled scores
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (D > 128) return wide_dense(false, q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, s);
     return D <= 64 ? launch_attn<64, false>(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, s)
                    : launch_attn<128, false>(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, s);
 }
@@ -827,11 +837,12 @@ extern "C" int forge_attn_fused_f16(const void* q, const void* k, const void* v,
                                     int B, int Hq, int Hkv, int Sq, int Skv, int D,
                                     int mask_kind, const int32_t* lens, float scale, void* stream) {
     using namespace forge;
-    int st = check_attn_args(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, /*any_head_dim=*/true);
+    int st = check_attn_args(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, /*any_head_dim=*/true, 256);
     if (st != FORGE_OK) return st;
-    if ((long long)Hq * B * ((Sq + 255) / 256) > 2147483647LL) return FORGE_ERR_UNSUPPORTED;
+    if ((long long)Hq * B * ((Sq + 127) / 128) > 2147483647LL) return FORGE_ERR_UNSUPPORTED;
     if (!(scale >= 0.f)) return FORGE_ERR_UNSUPPORTED;  // the running maximum is taken on unscaled scores
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (D > 128) return wide_dense(true, q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, s);
     return D <= 64 ? launch_attn<64, true>(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, s)
                    : launch_attn<128, true>(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, s);
 }
@@ -858,10 +869,10 @@ extern "C" int forge_attn_fused_strided(const void* q, const void* k, const void
                                         const int64_t* out_strides, int mask_kind, const int32_t* lens, float scale,
                                         void* stream) {
     using namespace forge;
-    int st = check_attn_args(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, /*any_head_dim=*/true);
+    int st = check_attn_args(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, /*any_head_dim=*/true, 256);
     if (st != FORGE_OK) return st;
     if (!q_strides || !k_strides || !v_strides || !out_strides) return FORGE_ERR_INVALID_ARG;
-    if ((long long)Hq * B * ((Sq + 255) / 256) > 2147483647LL) return FORGE_ERR_UNSUPPORTED;
+    if ((long long)Hq * B * ((Sq + 127) / 128) > 2147483647LL) return FORGE_ERR_UNSUPPORTED;
     if (!(scale >= 0.f)) return FORGE_ERR_UNSUPPORTED;  // the running maximum is taken on unscaled scores
     Strides str[4];
     const int64_t* in[4] = {q_strides, k_strides, v_strides, out_strides};
@@ -873,6 +884,11 @@ extern "C" int forge_attn_fused_strided(const void* q, const void* k, const void
         if (str[i].b >= (1LL << 38) || str[i].h >= (1LL << 38) || str[i].s >= (1LL << 38)) return FORGE_ERR_UNSUPPORTED;
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (D > 128) {
+        long long w[4][3];
+        for (int i = 0; i < 4; ++i) { w[i][0] = str[i].b; w[i][1] = str[i].h; w[i][2] = str[i].s; }
+        return attn_wide(false, q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, w, s);
+    }
     return D <= 64 ? launch_attn<64, false>(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, s, nullptr, 1,
                                             &str[0], &str[1], &str[2], &str[3])
                    : launch_attn<128, false>(q, k, v, out, B, Hq, Hkv, Sq, Skv, D, mask_kind, lens, scale, s, nullptr, 1,

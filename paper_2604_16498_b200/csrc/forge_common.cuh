@@ -84,7 +84,7 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 // Common validation of the attention entry points' scalar arguments and pointers.
 inline int check_attn_args(const void* q, const void* k, const void* v, const void* out,
                            int B, int Hq, int Hkv, int Sq, int Skv, int D,
-                           int mask_kind, const int32_t* lens, bool any_head_dim = false) {
+                           int mask_kind, const int32_t* lens, bool any_head_dim = false, int max_head_dim = 128) {
     if (!q || !k || !v || !out) return FORGE_ERR_INVALID_ARG;
     if (B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Skv <= 0 || D <= 0) return FORGE_ERR_INVALID_ARG;
     if (Hq % Hkv != 0) return FORGE_ERR_INVALID_ARG;
@@ -92,8 +92,8 @@ inline int check_attn_args(const void* q, const void* k, const void* v, const vo
     if ((mask_kind & FORGE_MASK_PADDING) && !lens) return FORGE_ERR_INVALID_ARG;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out)) return FORGE_ERR_INVALID_ARG;
     if (lens && (reinterpret_cast<uintptr_t>(lens) & 3u)) return FORGE_ERR_INVALID_ARG;
-    // any_head_dim: every multiple of 8 up to 128 (16-byte rows); otherwise the two sizes with their own kernels
-    if (any_head_dim ? (D > 128 || (D % 8) != 0) : (D != 64 && D != 128)) return FORGE_ERR_UNSUPPORTED;
+    // any_head_dim: every multiple of 8 (16-byte rows) up to max_head_dim; otherwise the two sizes with their own kernels
+    if (any_head_dim ? (D > max_head_dim || (D % 8) != 0) : (D != 64 && D != 128)) return FORGE_ERR_UNSUPPORTED;
     return FORGE_OK;
 }
 

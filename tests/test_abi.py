@@ -72,7 +72,9 @@ def test_attention_argument_validation(lib, fn):
     assert call(mask=4) == binding.ERR_INVALID_ARG
     assert call(mask=2) == binding.ERR_INVALID_ARG        # padding mask without lens
     assert call(k=P + 8) == binding.ERR_INVALID_ARG       # misaligned
-    assert call(D=256) == binding.ERR_UNSUPPORTED
+    assert call(D=264) == binding.ERR_UNSUPPORTED         # beyond the largest head size
+    if fn == "forge_attn_fused_f32":
+        assert call(D=256) == binding.ERR_UNSUPPORTED     # the fp32 kernel has 64 and 128 only
     assert call(D=100) == binding.ERR_UNSUPPORTED         # rows are not multiples of 16 bytes
 
 

@@ -9,7 +9,9 @@
 // Warp roles:
 //   warps 0-3 : softmax / rescale / epilogue of tile 0; thread = one query row (TMEM lane), so row
 //   warps 4-7 : the same for tile 1                    maxima and sums need no cross-thread reduction
-//   warp 8    : TMA producer: Q tiles, then K and V tiles (64 keys, one per half-step) through rings
+//   warp 8    : TMA producer: Q tiles, then K and V tiles (64 keys, one per half-step) through rings;
+//               it sleeps between barrier polls (a spinning thread takes issue slots from the softmax
+//               warp of its scheduler: 1.2 % of the kernel)
 //   warp 9    : tcgen05.mma issuer of tile 0 (one elected lane), owns the TMEM allocation
 //   warp 10   : tcgen05.mma issuer of tile 1
 //   warp 11 only completes the third warpgroup, which hands registers to the other two
@@ -311,7 +313,7 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 for (int t = 0; t < kTilesPerCta; ++t) {
                     if (it.nh[t] == 0) continue;
                     // the tile's last S = Q K^T of its previous item has completed: Q may be replaced
-                    if (!mbar_wait(&q_empty[t], (q_loads[t] & 1) ^ 1)) { failed = true; break; }
+                    if (!mbar_wait_relaxed(&q_empty[t], (q_loads[t] & 1) ^ 1)) { failed = true; break; }
                     ++q_loads[t];
                     mbar_expect_tx(&q_full[t], L::kTileBytes);
 #pragma unroll
@@ -342,13 +344,13 @@ attn_bf16_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                         const int g = kvn[u]++, st = kv_slot(u, g);
                         const uint32_t ph = kv_phase(g);
                         const int kvh = it.kvh[u];
-                        if (!mbar_wait(&k_empty[st], ph ^ 1)) { failed = true; break; }
+                        if (!mbar_wait_relaxed(&k_empty[st], ph ^ 1)) { failed = true; break; }
                         mbar_expect_tx(&k_full[st], L::kKVTileBytes);
 #pragma unroll
                         for (int c = 0; c < D / 64; ++c)
                             tma_load_4d(sK + st * L::kKVTileBytes + c * L::kKVChunkBytes, &tmap_k, &k_full[st], c * 64,
                                         j * kHalf, kvh, it.b);
-                        if (!mbar_wait(&v_empty[st], ph ^ 1)) { failed = true; break; }
+                        if (!mbar_wait_relaxed(&v_empty[st], ph ^ 1)) { failed = true; break; }
                         mbar_expect_tx(&v_full[st], L::kKVTileBytes);
 #pragma unroll
                         for (int c = 0; c < D / 64; ++c)

@@ -64,6 +64,19 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, long l
     return true;
 }
 
+// Same, for a thread whose wait is not on the critical path (a producer that runs ahead of its consumers):
+// it sleeps between polls, which leaves the issue slots and the shared-memory queue of its scheduler to
+// the warps that compute.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint64_t* bar, uint32_t parity, long long budget_clocks = kWaitBudgetClocks) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        __nanosleep(100);
+        if (clock64() - t0 > budget_clocks) return false;
+    }
+    return true;
+}
+
 // Same for a whole converged warp: every lane gets the same answer, so that the warp-collective
 // (.sync.aligned) instructions that follow are executed by all lanes or by none.
 __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, long long budget_clocks = kWaitBudgetClocks) {

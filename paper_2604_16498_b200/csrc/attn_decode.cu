@@ -10,7 +10,7 @@
 // this part, with 250 KB 5.8 TB/s).  So the kernel is persistent and every warp is an independent
 // worker: it owns whole pieces, keeps a private ring of 16-row blocks in shared memory filled by
 // TMA tile copies (16 rows x 64 columns each, 128-byte swizzle, completion counted on an mbarrier
-// per stage) that run ahead across piece boundaries (8 warps x 16 KB in flight per SM), and writes
+// per stage) that run ahead across piece boundaries (7 warps x 16 KB in flight per SM), and writes
 // its partial straight from registers.  No warp ever waits for another one.
 //
 // Pieces.  All pieces of a call are C blocks of 16 rows long (the last piece of a sequence may be
@@ -43,7 +43,11 @@
 namespace forge {
 namespace {
 
-constexpr int kWarps = 8;
+// Workers per CTA.  Each keeps its ring full, so the warp count sets how many bytes the SM has in flight; beyond
+// what saturates the memory system, more only queue: every block arrives later, the first ones spread over a
+// longer start-up burst, and the call ends one loaded latency after its last request.  Measured at B 16,
+// 32/8 heads, lengths 1024..4096, D = 128 (148 MB): 5 / 6 / 7 / 8 warps give 33.1 / 31.5 / 31.0 / 33.4 us.
+constexpr int kWarps = 7;
 constexpr int kThreads = kWarps * 32;
 constexpr int kBlockKeys = 16;             // cached rows per ring stage
 // Per warp.  16 KB (two stages of 16 rows at D = 128) measured a little faster than 24 KB: the memory system is

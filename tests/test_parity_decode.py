@@ -88,7 +88,7 @@ def test_one_workspace_serves_call_after_call_with_other_shapes():
 
 
 def test_more_pieces_than_workers():
-    """A batch whose pieces outnumber the GPU's workers (8 per SM) even at the longest allowed piece: workers
+    """A batch whose pieces outnumber the GPU's workers (7 per SM) even at the longest allowed piece: workers
     take several pieces each."""
     w = wl.decode_workload("t", 28, 200, 8, 8, 48, 64, 2, 0.125, (1, 48))
     _run(w)

@@ -46,7 +46,8 @@ namespace {
 // Workers per CTA.  Each keeps its ring full, so the warp count sets how many bytes the SM has in flight; beyond
 // what saturates the memory system, more only queue: every block arrives later, the first ones spread over a
 // longer start-up burst, and the call ends one loaded latency after its last request.  Measured at B 16,
-// 32/8 heads, lengths 1024..4096, D = 128 (148 MB): 5 / 6 / 7 / 8 warps give 33.1 / 31.5 / 31.0 / 33.4 us.
+// 32/8 heads, lengths 1024..4096, D = 128 (148 MB): 5 / 6 / 7 / 8 warps give 33.1 / 31.5 / 31.0 / 33.4 us
+// (30.1 / 28.9 / 31.4 us for 6 / 7 / 8 warps once the rows are loaded with the evict-first policy).
 constexpr int kWarps = 7;
 constexpr int kThreads = kWarps * 32;
 constexpr int kBlockKeys = 16;             // cached rows per ring stage
@@ -378,6 +379,9 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             p_idx = item_of_round(++p_round);
         }
     };
+    // Every cached row is read once per call: its lines are marked first to go, so that they do not push the
+    // partials, the queries and whatever the caller keeps in L2 out of it (2 us of 31 at B 16, lengths 1024..4096).
+    const uint64_t stream_policy = ptx::l2_policy_evict_first();
     auto issue = [&]() {  // one lane starts the block's tile copies (rows past the cache's end are zero-filled)
         if (p_idx < num_items) {
             if (lane == 0) {
@@ -386,8 +390,8 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 ptx::mbar_expect_tx(&full[st], kStageBytes);
 #pragma unroll
                 for (int cb = 0; cb < D / 64; ++cb) {
-                    ptx::tma_load_3d_addr(dst + cb * kTileBytes, &tmap_k, &full[st], cb * 64, p_j0, p_bk);
-                    ptx::tma_load_3d_addr(dst + kKBytes + cb * kTileBytes, &tmap_v, &full[st], cb * 64, p_j0, p_bk);
+                    ptx::tma_load_3d_addr_hint(dst + cb * kTileBytes, &tmap_k, &full[st], cb * 64, p_j0, p_bk, stream_policy);
+                    ptx::tma_load_3d_addr_hint(dst + kKBytes + cb * kTileBytes, &tmap_v, &full[st], cb * 64, p_j0, p_bk, stream_policy);
                 }
             }
             ++p_n;

@@ -35,9 +35,10 @@ def test_shapes_and_activations(shape, act):
     assert_close_bf16(y, ref)
 
 
-def test_extreme_weights_are_widened_exactly():
+@pytest.mark.parametrize("M", [128, 384])  # one row tile (one-CTA kernel) and several (CTA pairs)
+def test_extreme_weights_are_widened_exactly(M):
     """-128, 127 and 0 only, identity-like activations: the result is an exact small integer combination."""
-    M, N, K = 128, 64, 64
+    N, K = 64, 64
     x = torch.zeros((M, K), dtype=torch.float16, device="cuda"); x[:, 0] = 1.0; x[:, 1] = 2.0
     wq = torch.zeros((N, K), dtype=torch.int8, device="cuda"); wq[:, 0] = -128; wq[:, 1] = 127; wq[5, 1] = -128
     y = binding.linear_act_w8a16(x, wq, torch.ones(N, device="cuda"), None, None, binding.ACT_NONE)

@@ -634,6 +634,23 @@ def other_configs(torch, binding, dev, gen, randn, peaks, args):
                lambda d: binding.linear_act_w8a16(d[0], d[1], d[2], None, None, binding.ACT_GELU_TANH, out=d[3]))
     fl = 2 * M * N * K
     other["linear_w8a16_8192x8192x4096"] = {"ms": ms, "tflops": fl / ms / 1e9, "frac_of_fp16_peak": fl / ms / 1e9 / pk}
+    # a whole decoder layer of the 8B-class shape (QKV projection, causal GQA attention, output projection with
+    # residual, SwiGLU MLP, down projection with residual) into its two planned buffers; one set of weights
+    # (436 MB, larger than L2), rotating activations
+    B, S, Hq, Hkv, D, F = 4, 2048, 32, 8, 128, 14336
+    Hd, Nqkv, T = Hq * D, (Hq + 2 * Hkv) * D, B * S
+    weights = {"w_qkv": randn((Hd, Nqkv), 0.02), "w_o": randn((Hd, Hd), 0.02), "w_gate": randn((Hd, F), 0.02),
+               "w_up": randn((Hd, F), 0.02), "w_down": randn((F, Hd), 0.02)}
+    plan = binding.decoder_layer_plan(B, S, Hq, Hkv, D, F)
+    ws = torch.empty(max(int(plan.workspace_bytes), 256), dtype=torch.uint8, device=dev)
+    ms = timed(lambda: (randn((T, Hd)), empty((T, Hd))),
+               lambda d: binding.decoder_layer(d[0], weights, B, S, Hq, Hkv, D, F, out=d[1], workspace=ws))
+    fl = 2 * T * Hd * (Nqkv + Hd + 3 * F) + 4 * D * B * Hq * (S * (S + 1) // 2)
+    other["decoder_layer_8b_shape_B4_S2048"] = {
+        "ms": ms, "tflops": fl / ms / 1e9, "frac_of_bf16_peak_sustained": fl / ms / 1e9 / peaks.get("bf16_tflops_sustained", pk),
+        "flops": fl, "launches": 5, "intermediates": int(plan.num_regs), "buffers": int(plan.num_bufs), "rho_buf": float(plan.rho_buf),
+        "workspace_bytes": int(plan.workspace_bytes), "unplanned_bytes": int(plan.unplanned_bytes)}
+    del weights, ws
     return other
 
 

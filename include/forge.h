@@ -335,7 +335,10 @@ int forge_decoder_layer(const forge_decoder_layer_desc* desc, const void* x, voi
  * Host-buffer variants: the same operators for callers whose tensors live in
  * HOST memory (pinned memory makes the copies asynchronous).  Inputs are copied
  * to `dev_scratch`, the operator runs there, and the result is copied back to the
- * host pointer, all on `stream`; the call returns without synchronising.
+ * host pointer, all ordered after what `stream` held before the call and before
+ * what it is given afterwards; the call returns without synchronising.  (The
+ * 16-bit attention with several batch entries moves entry by entry on two streams
+ * of the library's own, so that copies in, kernels and copies out overlap.)
  * dev_scratch is DEVICE memory of at least forge_*_host_scratch_bytes(...) bytes,
  * 256-byte aligned, owned by the caller.  `lens` is a HOST pointer here.
  */

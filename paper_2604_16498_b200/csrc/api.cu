@@ -2,6 +2,8 @@
 // the device status word, tensor-map encoding and the host-buffer variants.
 #include <atomic>
 #include <cstring>
+#include <mutex>
+#include <vector>
 
 #include "forge_common.cuh"
 #include "tmap.cuh"
@@ -137,6 +139,38 @@ extern "C" int forge_check_status(void* stream) {
 // ------------------------------------------------------------------ host-buffer variants
 namespace {
 inline size_t up256(size_t n) { return (n + 255) & ~(size_t)255; }
+
+// Two library-owned streams per device for the copies of the host-buffer variants (one per direction) and a
+// pool of events to order them against the caller's stream.  A call holds `mu` while it enqueues.
+struct CopyLanes {
+    std::mutex mu;
+    cudaStream_t in = nullptr, out = nullptr;
+    std::vector<cudaEvent_t> ev;
+};
+CopyLanes* copy_lanes(int num_events) {
+    static std::mutex table_mu;
+    static CopyLanes* table[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(table_mu);
+    CopyLanes*& lanes = table[dev];
+    if (!lanes) {
+        CopyLanes* fresh = new CopyLanes();
+        if (cudaStreamCreateWithFlags(&fresh->in, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaStreamCreateWithFlags(&fresh->out, cudaStreamNonBlocking) != cudaSuccess) {
+            delete fresh;
+            return nullptr;
+        }
+        lanes = fresh;
+    }
+    std::lock_guard<std::mutex> lock2(lanes->mu);
+    while ((int)lanes->ev.size() < num_events) {
+        cudaEvent_t e;
+        if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        lanes->ev.push_back(e);
+    }
+    return lanes;
+}
 }  // namespace
 
 extern "C" size_t forge_attn_host_scratch_bytes(int B, int Hq, int Hkv, int Sq, int Skv, int D, int elem_bytes) {
@@ -165,6 +199,48 @@ static int attn_host_impl(bool f32, const void* q, const void* k, const void* v,
     void* dout = p; p += up256(qo);
     int32_t* dlens = reinterpret_cast<int32_t*>(p);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // Several batch entries, 16-bit tensors: one entry's copies in, its kernel and its copy out overlap with
+    // the neighbours' (the two directions of the host link run at the same time).
+    if (!f32 && B >= 2) {
+        CopyLanes* lanes = copy_lanes(2 * B + 2);
+        if (lanes) {
+            std::lock_guard<std::mutex> lock(lanes->mu);
+            const size_t qo1 = qo / B, kv1 = kv / B;
+            cudaEvent_t fork = lanes->ev[2 * B], join = lanes->ev[2 * B + 1];
+            // the library's copy streams start where `stream` is now
+            FORGE_CUDA_TRY(cudaEventRecord(fork, s));
+            FORGE_CUDA_TRY(cudaStreamWaitEvent(lanes->in, fork, 0));
+            FORGE_CUDA_TRY(cudaStreamWaitEvent(lanes->out, fork, 0));
+            if (lens) FORGE_CUDA_TRY(cudaMemcpyAsync(dlens, lens, (size_t)B * 4, cudaMemcpyHostToDevice, lanes->in));
+            int st = FORGE_OK;
+            for (int b = 0; b < B && st == FORGE_OK; ++b) {
+                const char* hq = static_cast<const char*>(q) + b * qo1;
+                const char* hk = static_cast<const char*>(k) + b * kv1;
+                const char* hv = static_cast<const char*>(v) + b * kv1;
+                char* dq1 = static_cast<char*>(dq) + b * qo1;
+                char* dk1 = static_cast<char*>(dk) + b * kv1;
+                char* dv1 = static_cast<char*>(dv) + b * kv1;
+                char* do1 = static_cast<char*>(dout) + b * qo1;
+                FORGE_CUDA_TRY(cudaMemcpyAsync(dq1, hq, qo1, cudaMemcpyHostToDevice, lanes->in));
+                FORGE_CUDA_TRY(cudaMemcpyAsync(dk1, hk, kv1, cudaMemcpyHostToDevice, lanes->in));
+                FORGE_CUDA_TRY(cudaMemcpyAsync(dv1, hv, kv1, cudaMemcpyHostToDevice, lanes->in));
+                FORGE_CUDA_TRY(cudaEventRecord(lanes->ev[2 * b], lanes->in));
+                FORGE_CUDA_TRY(cudaStreamWaitEvent(s, lanes->ev[2 * b], 0));
+                st = forge_attn_fused(dq1, dk1, dv1, do1, 1, Hq, Hkv, Sq, Skv, D, mask_kind, lens ? dlens + b : nullptr,
+                                      scale, stream);
+                if (st != FORGE_OK) break;
+                FORGE_CUDA_TRY(cudaEventRecord(lanes->ev[2 * b + 1], s));
+                FORGE_CUDA_TRY(cudaStreamWaitEvent(lanes->out, lanes->ev[2 * b + 1], 0));
+                FORGE_CUDA_TRY(cudaMemcpyAsync(static_cast<char*>(out) + b * qo1, do1, qo1, cudaMemcpyDeviceToHost, lanes->out));
+            }
+            // `stream` continues after the last copy out (and after everything the copy streams were given)
+            FORGE_CUDA_TRY(cudaEventRecord(join, lanes->in));
+            FORGE_CUDA_TRY(cudaStreamWaitEvent(s, join, 0));
+            FORGE_CUDA_TRY(cudaEventRecord(join, lanes->out));
+            FORGE_CUDA_TRY(cudaStreamWaitEvent(s, join, 0));
+            return st;
+        }
+    }
     FORGE_CUDA_TRY(cudaMemcpyAsync(dq, q, qo, cudaMemcpyHostToDevice, s));
     FORGE_CUDA_TRY(cudaMemcpyAsync(dk, k, kv, cudaMemcpyHostToDevice, s));
     FORGE_CUDA_TRY(cudaMemcpyAsync(dv, v, kv, cudaMemcpyHostToDevice, s));

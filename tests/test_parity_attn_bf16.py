@@ -146,3 +146,21 @@ def test_host_buffer_variant():
     binding.attn_fused_host(q, k, v, out, scratch, w.mask_kind, torch.from_numpy(w.lens), w.scale)
     binding.check_status()
     assert_close_bf16(out, oracle.attn(w.q.values, w.k.values, w.v.values, w.mask_kind, w.lens, w.scale))
+
+
+def test_host_buffer_variant_is_ordered_on_the_callers_stream():
+    """Three batch entries (the entry-by-entry path): work given to the stream after the call sees the result, and
+    the device scratch may be reused by the next call without a synchronisation in between."""
+    w = wl.attention_workload("t", 48, 3, 4, 2, 300, 300, 128, wl.MASK_CAUSAL, 128 ** -0.5, "bf16")
+    q, k, v = to_pinned(w.q), to_pinned(w.k), to_pinned(w.v)
+    out1 = torch.empty_like(q).pin_memory()
+    out2 = torch.empty_like(q).pin_memory()
+    scratch = torch.empty(binding.attn_host_scratch_bytes(3, 4, 2, 300, 300, 128, 2), dtype=torch.uint8, device="cuda")
+    binding.attn_fused_host(q, k, v, out1, scratch, w.mask_kind, None, w.scale)
+    back = torch.empty(out1.shape, dtype=out1.dtype, device="cuda")
+    back.copy_(out1, non_blocking=True)  # same stream, right behind the call
+    binding.attn_fused_host(q, k, v, out2, scratch, w.mask_kind, None, w.scale)
+    binding.check_status()
+    ref = oracle.attn(w.q.values, w.k.values, w.v.values, w.mask_kind, None, w.scale)
+    assert_close_bf16(back.cpu(), ref)
+    assert torch.equal(out1, out2)

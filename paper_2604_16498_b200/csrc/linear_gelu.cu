@@ -20,8 +20,9 @@
 // operand, eight extra warps (10-17) read all of it into registers, meet at a barrier of their own and
 // write the swizzled fp16 operand over it (exact: 1024 + (w ^ 0x80) as fp16 bits, minus 1152); the scale
 // is applied to the accumulator in the epilogue, where it factors out of the sum over K.
-// 8192 x 8192 x 4096: 535 us (1028 TFLOP/s), against 850 us with 192-column tiles and the int8 tile in a
-// buffer of its own converted piece by piece.
+// Four stages (with a single output staging buffer to make room).  8192 x 8192 x 4096: 511 us (1075 TFLOP/s),
+// against 850 us with 192-column tiles, three stages and the int8 tile in a buffer of its own converted
+// piece by piece.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 
@@ -52,9 +53,12 @@ struct LinearSmem {
     // W8: BN rows of 64 int8 weights, which arrive in the upper half of the stage's B operand and are widened in place
     static constexpr int kRawBytes = W8 ? BN * kBK : 0;
     static constexpr int kStageBytes = kABytes + kBBytes;
-    static constexpr int kOutBytes = kBM * 128;          // output staging: 128 rows x 64 bf16, two buffers
+    static constexpr int kOutBytes = kBM * 128;          // output staging: 128 rows x 64 bf16
+    // two buffers; one in the int8 form, whose long k-loops leave the epilogue idle most of the time and whose
+    // fourth stage needs the room
+    static constexpr int kOutBufs = W8 ? 1 : 2;
     static constexpr int kOutOffset = STAGES * kStageBytes;
-    static constexpr int kBarOffset = kOutOffset + 2 * kOutBytes;
+    static constexpr int kBarOffset = kOutOffset + kOutBufs * kOutBytes;
     // barriers: full[S], empty[S], tmem_full[2], tmem_empty[2], raw_full[S]; then the TMEM base, then
     // bias[2][BN] and scale[2][BN]
     static constexpr int kBiasOffset = kBarOffset + (3 * STAGES + 4) * 8 + 16;
@@ -278,7 +282,7 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
             // Two staging buffers: the store of one block drains while the next block is computed.
 #pragma unroll 1
             for (int blk = 0; blk < BNO / 64; ++blk, ++out_blocks) {
-                uint8_t* stage_out = smem + L::kOutOffset + (out_blocks & 1) * L::kOutBytes;
+                uint8_t* stage_out = smem + L::kOutOffset + (out_blocks % L::kOutBufs) * L::kOutBytes;
                 uint32_t r[32];
                 tmem_ld_x32(taddr + blk * 64 + chalf * 32, r);
                 if constexpr (GATED) {  // silu(gate) * up, the up product sits BN / 2 columns further
@@ -290,8 +294,8 @@ linear_bias_gelu_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid
                         r[i] = __float_as_uint(activate<FORGE_ACT_SILU>(__uint_as_float(r[i])) * __uint_as_float(r2[i]));
                 }
                 tmem_ld_wait();
-                // the store issued two blocks ago has finished reading this buffer
-                if (etid == 0) tma_store_wait_read<1>();
+                // the store that last used this buffer (two blocks ago with two buffers) has finished reading it
+                if (etid == 0) tma_store_wait_read<L::kOutBufs - 1>();
                 asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {  // 16-byte chunk chalf*4 + c of the row's 128-byte line
@@ -471,10 +475,10 @@ extern "C" int forge_linear_act_w8a16(const void* x, const void* w_int8, const f
     if ((K % 16) != 0 || (N % 8) != 0) return FORGE_ERR_UNSUPPORTED;  // 16-byte rows of int8 weights and of fp16 outputs
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     switch (act) {
-        case FORGE_ACT_GELU_TANH: return launch_linear<256, 3, FORGE_ACT_GELU_TANH, true, false, true, true>(x, w_int8, b, residual, y, M, N, K, s, nullptr, scale);
-        case FORGE_ACT_GELU_ERF: return launch_linear<256, 3, FORGE_ACT_GELU_ERF, true, false, true, true>(x, w_int8, b, residual, y, M, N, K, s, nullptr, scale);
-        case FORGE_ACT_RELU: return launch_linear<256, 3, FORGE_ACT_RELU, true, false, true, true>(x, w_int8, b, residual, y, M, N, K, s, nullptr, scale);
-        case FORGE_ACT_SILU: return launch_linear<256, 3, FORGE_ACT_SILU, true, false, true, true>(x, w_int8, b, residual, y, M, N, K, s, nullptr, scale);
-        default: return launch_linear<256, 3, FORGE_ACT_NONE, true, false, true, true>(x, w_int8, b, residual, y, M, N, K, s, nullptr, scale);
+        case FORGE_ACT_GELU_TANH: return launch_linear<256, 4, FORGE_ACT_GELU_TANH, true, false, true, true>(x, w_int8, b, residual, y, M, N, K, s, nullptr, scale);
+        case FORGE_ACT_GELU_ERF: return launch_linear<256, 4, FORGE_ACT_GELU_ERF, true, false, true, true>(x, w_int8, b, residual, y, M, N, K, s, nullptr, scale);
+        case FORGE_ACT_RELU: return launch_linear<256, 4, FORGE_ACT_RELU, true, false, true, true>(x, w_int8, b, residual, y, M, N, K, s, nullptr, scale);
+        case FORGE_ACT_SILU: return launch_linear<256, 4, FORGE_ACT_SILU, true, false, true, true>(x, w_int8, b, residual, y, M, N, K, s, nullptr, scale);
+        default: return launch_linear<256, 4, FORGE_ACT_NONE, true, false, true, true>(x, w_int8, b, residual, y, M, N, K, s, nullptr, scale);
     }
 }

@@ -638,6 +638,19 @@ def other_configs(torch, binding, dev, gen, randn, peaks, args):
                lambda d: binding.linear_act_w8a16(d[0], d[1], d[2], None, None, binding.ACT_GELU_TANH, out=d[3]))
     fl = 2 * M * N * K
     other["linear_w8a16_8192x8192x4096"] = {"ms": ms, "tflops": fl / ms / 1e9, "frac_of_fp16_peak": fl / ms / 1e9 / pk}
+    # split-KV decode of a single long sequence (the small-batch case the splits exist for): 128 pieces per
+    # sequence keep every worker warp busy, and groups of sixteen pieces are merged in two levels
+    B1, Hq1, Hkv1, S1, D1, splits1 = 1, 32, 8, 32768, 128, 128
+    lens1 = torch.full((B1,), S1, dtype=torch.int32, device=dev)
+    ws1 = torch.empty(binding.attn_decode_workspace_bytes(B1, Hq1, D1, splits1), dtype=torch.uint8, device=dev)
+    binding.attn_decode_workspace_init(ws1)
+    ms = timed(lambda: (randn((B1, Hq1, D1)), randn((B1, Hkv1, S1, D1)), randn((B1, Hkv1, S1, D1)), empty((B1, Hq1, D1))),
+               lambda d: binding.attn_decode_splitkv(d[0], d[1], d[2], lens1, splits1, D1 ** -0.5, out=d[3], workspace=ws1),
+               nset=5)  # 5 x 134 MB
+    by = 4 * Hkv1 * D1 * S1 + 4 * B1 * Hq1 * D1
+    other["decode_B1_32k_context_128_splits"] = {"ms": ms, "gbs": by / ms / 1e6, "frac_of_hbm_peak": by / ms / 1e6 / peaks["hbm_gbs"],
+                                                 "bytes": by}
+    del ws1
     # a whole decoder layer of the 8B-class shape (QKV projection, causal GQA attention, output projection with
     # residual, SwiGLU MLP, down projection with residual) into its two planned buffers; one set of weights
     # (436 MB, larger than L2), rotating activations

@@ -149,12 +149,15 @@ int forge_attn_fused_f32(const void* q, const void* k, const void* v, void* out,
  * call starts: clear a new workspace once with forge_attn_decode_workspace_init (or
  * any memset); every call that completes leaves the counters at zero, so the same
  * workspace can be passed again and again.  The counters take the first
- * max(64 KiB, 4 * B * Hq bytes): all shapes with B * Hq <= 16384 share that region, so
+ * max(1088 KiB, 68 * B * Hq bytes): all shapes with B * Hq <= 16384 share that region, so
  * a workspace cleared once also serves later calls of other such shapes; after a call
  * with a larger B * Hq, or one that ended in FORGE_ERR_TIMEOUT, clear it again.  The
  * rest needs no initialisation.  Two calls that may overlap on the GPU must not share
  * a workspace.
- * 1 <= num_splits <= 64; D any multiple of 8 up to 128; Hq / Hkv must be between 1 and 8.
+ * 1 <= num_splits <= 256 (FORGE_ERR_UNSUPPORTED beyond); D any multiple of 8 up to 128; Hq / Hkv
+ * must be between 1 and 8.  A piece is streamed by one warp, and a GPU runs seven such warps
+ * per SM: with few (batch, kv head) pairs, allow about 7 * SMs / (B * Hkv) pieces per sequence
+ * (a single sequence with 8 kv heads: 128 or more) or most of the GPU idles.
  */
 int forge_attn_decode_splitkv(const void* q, const void* k_cache, const void* v_cache, void* out,
                               int B, int Hq, int Hkv, int Smax, int D,

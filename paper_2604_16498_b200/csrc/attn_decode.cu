@@ -55,6 +55,11 @@ constexpr int kBlockKeys = 16;             // cached rows per ring stage
 // saturated either way, and what is queued beyond that only adds to the latency of every block, which is what
 // the end of the call (the last blocks of the slowest warps) waits for.
 constexpr int kWarpRingBytes = 16 * 1024;
+constexpr int kSingleLevelPieces = 32;     // up to this many pieces of a sequence are merged by one warp in one go
+                                           // (one (m, l) pair per lane and head)
+constexpr int kMergeGroup = 16;            // beyond that: groups of sixteen, then the (at most sixteen) groups' results
+constexpr int kMaxSplits = kMergeGroup * kMergeGroup;
+constexpr int kPiecesPerLane = 1;          // no merge walks through more than 32 partials
 
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 r;
@@ -213,27 +218,30 @@ __device__ __forceinline__ Item make_item(unsigned idx, const Schedule& sc, cons
     return it;
 }
 
-// Merge of the `pieces` partials of the G heads of one (batch, kv head), done by the warp that completed
-// the last piece.  Lane = D / 32 consecutive output dims.  A function of its own (not inlined): it runs once
-// per (batch, kv head) and must not take registers away from the streaming loop.
+// Merge of `pieces` partials of the G heads of one (batch, kv head), done by the warp that completed the last
+// of them: the partials in slots first, first + stride, ...  With `final` the result is normalised and written
+// to the output rows; otherwise it is written back, unnormalised, as the partial in slot `first` (the first
+// level of a two-level merge).  Lane = D / 32 consecutive output dims.  A function of its own (not inlined):
+// it runs once per (batch, kv head) or group of pieces and must not take registers away from the streaming loop.
 template <int D, int G, bool F16>
-__device__ __noinline__ void merge_pieces(const float* __restrict__ ws_o, const float* __restrict__ ws_ml,
-                                          uint16_t* __restrict__ out, int head0, int pieces, int num_splits,
-                                          int head_dim, int lane) {
+__device__ __forceinline__ void merge_impl(float* __restrict__ ws_o, float* __restrict__ ws_ml,
+                                           uint16_t* __restrict__ out, int head0, int first, int stride, int pieces,
+                                           bool final, int num_splits, int head_dim, int lane) {
     // The merge sits at the very end of the call (all pieces of a sequence end together), so it is
     // arranged for few round trips to L2: the (m, l) pairs of all heads are requested first, then the
     // partial outputs of two heads and sixteen pieces at a time, all before anything is used.
     constexpr int V = D / 32;  // floats per lane
     const int P = pieces;
-    float2 ml[G][2];  // (m, l) of pieces lane and lane + 32 (at most 64 pieces) of every head
+    float2 ml[G][kPiecesPerLane];  // (m, l) of pieces lane, lane + 32, ... of every head
 #pragma unroll
     for (int h = 0; h < G; ++h) {
-        const float2* mlp = reinterpret_cast<const float2*>(ws_ml) + (size_t)(head0 + h) * num_splits;
-        ml[h][0] = (lane < P) ? __ldcg(mlp + lane) : make_float2(-INFINITY, 0.f);
-        ml[h][1] = (lane + 32 < P) ? __ldcg(mlp + lane + 32) : make_float2(-INFINITY, 0.f);
+        const float2* mlp = reinterpret_cast<const float2*>(ws_ml) + (size_t)(head0 + h) * num_splits + first;
+#pragma unroll
+        for (int j = 0; j < kPiecesPerLane; ++j)
+            ml[h][j] = (lane + 32 * j < P) ? __ldcg(mlp + (lane + 32 * j) * stride) : make_float2(-INFINITY, 0.f);
     }
     auto load_part = [&](int h, int sp, float (&dst)[V]) {
-        const float* src = ws_o + ((size_t)(head0 + h) * num_splits + sp) * D + lane * V;
+        const float* src = ws_o + ((size_t)(head0 + h) * num_splits + first + sp * stride) * D + lane * V;
         if constexpr (V == 4) {
             const float4 t4 = __ldcg(reinterpret_cast<const float4*>(src));
             dst[0] = t4.x; dst[1] = t4.y; dst[2] = t4.z; dst[3] = t4.w;
@@ -260,20 +268,26 @@ __device__ __noinline__ void merge_pieces(const float* __restrict__ ws_o, const 
         };
         load_chunk(0);
         // weights of the two heads' pieces: w = 2^(m - M), 0 for a piece without rows
-        float w[2][2], L[2];
+        float w[2][kPiecesPerLane], L[2], Mx[2];
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
             const int h = (h0 + e < G) ? h0 + e : h0;
-            float M = fmaxf(ml[h][0].x, ml[h][1].x);
+            float M = ml[h][0].x;
+#pragma unroll
+            for (int j = 1; j < kPiecesPerLane; ++j) M = fmaxf(M, ml[h][j].x);
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
             const float Mr = (M == -INFINITY) ? 0.f : M;
-            w[e][0] = exp2f(ml[h][0].x - Mr);
-            w[e][1] = exp2f(ml[h][1].x - Mr);
-            float l = w[e][0] * ml[h][0].y + w[e][1] * ml[h][1].y;
+            float l = 0.f;
+#pragma unroll
+            for (int j = 0; j < kPiecesPerLane; ++j) {
+                w[e][j] = exp2f(ml[h][j].x - Mr);
+                l = fmaf(w[e][j], ml[h][j].y, l);
+            }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
             L[e] = l;
+            Mx[e] = M;
         }
         float o_acc[2][V];
 #pragma unroll
@@ -282,12 +296,20 @@ __device__ __noinline__ void merge_pieces(const float* __restrict__ ws_o, const 
             for (int v = 0; v < V; ++v) o_acc[e][v] = 0.f;
         for (int s0 = 0; s0 < P; s0 += kChunk) {
             if (s0 > 0) load_chunk(s0);
+            // the weights of pieces s0 .. s0 + 15 sit in entry s0 / 32 of their lanes (no dynamic indexing)
+            float wsel[2];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                wsel[e] = w[e][0];
+#pragma unroll
+                for (int j = 1; j < kPiecesPerLane; ++j) wsel[e] = ((s0 >> 5) == j) ? w[e][j] : wsel[e];
+            }
 #pragma unroll
             for (int e = 0; e < 2; ++e)
 #pragma unroll
                 for (int i = 0; i < kChunk; ++i) {
                     const int sp = s0 + i;
-                    const float wgt = __shfl_sync(0xffffffffu, (sp & 32) ? w[e][1] : w[e][0], sp & 31);
+                    const float wgt = __shfl_sync(0xffffffffu, wsel[e], sp & 31);
                     if (sp < P && wgt != 0.f) {
 #pragma unroll
                         for (int v = 0; v < V; ++v) o_acc[e][v] = fmaf(wgt, part[e][i][v], o_acc[e][v]);
@@ -297,6 +319,14 @@ __device__ __noinline__ void merge_pieces(const float* __restrict__ ws_o, const 
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
             if (h0 + e >= G) continue;
+            if (!final) {  // the merged partial (M, L, sum of the weighted partial outputs) takes the first slot
+                const size_t slot = (size_t)(head0 + h0 + e) * num_splits + first;
+                float* dst = ws_o + slot * D + lane * V;
+                if constexpr (V == 4) *reinterpret_cast<float4*>(dst) = make_float4(o_acc[e][0], o_acc[e][1], o_acc[e][2], o_acc[e][3]);
+                else *reinterpret_cast<float2*>(dst) = make_float2(o_acc[e][0], o_acc[e][1]);
+                if (lane == 0) *reinterpret_cast<float2*>(ws_ml + slot * 2) = make_float2(Mx[e], L[e]);
+                continue;
+            }
             const float invL = L[e] > 0.f ? 1.f / L[e] : 0.f;
             uint16_t* orow = out + (size_t)(head0 + h0 + e) * head_dim + lane * V;
             if (lane * V < head_dim) {  // head_dim is a multiple of 8, V divides 8: all V dims are inside or none
@@ -310,6 +340,43 @@ __device__ __noinline__ void merge_pieces(const float* __restrict__ ws_o, const 
     }
 }
 
+// The common case: all pieces of a (batch, kv head), at most 32, merged into the output rows.
+template <int D, int G, bool F16>
+__device__ __noinline__ void merge_pieces(float* __restrict__ ws_o, float* __restrict__ ws_ml,
+                                          uint16_t* __restrict__ out, int head0, int pieces, int num_splits,
+                                          int head_dim, int lane) {
+    merge_impl<D, G, F16>(ws_o, ws_ml, out, head0, 0, 1, pieces, true, num_splits, head_dim, lane);
+}
+
+// Arrival and merge for a sequence cut into more than 32 pieces (a long sequence in a small batch): two levels,
+// so that the merge work is spread over as many warps as there are groups of sixteen pieces and no warp walks
+// through more than sixteen partials per level.  The last arrival of a group of sixteen merges them into the
+// group's first slot and then arrives at the (batch, kv head)'s counter; the last of those merges the groups'
+// results.  The arrivals are the same release-acquire read-modify-writes as in the kernel.
+template <int D, int G, bool F16>
+__device__ __noinline__ void arrive_two_level(unsigned int* __restrict__ counters, float* __restrict__ ws_o,
+                                              float* __restrict__ ws_ml, uint16_t* __restrict__ out, int B, int Hkv,
+                                              int b, int kvh, int piece, int pieces, int head0, int num_splits,
+                                              int head_dim, int lane) {
+    auto arrive = [&](unsigned int* counter) {
+        __syncwarp();
+        unsigned int arrived = 0;
+        if (lane == 0)
+            asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(arrived) : "l"(counter) : "memory");
+        return __shfl_sync(0xffffffffu, arrived, 0);
+    };
+    unsigned int* group_counter = counters + b * Hkv + kvh;
+    const int sg = piece / kMergeGroup, n_sg = (pieces + kMergeGroup - 1) / kMergeGroup;
+    const int in_sg = min(kMergeGroup, pieces - sg * kMergeGroup);
+    unsigned int* sg_counter = counters + B * Hkv + (b * Hkv + kvh) * (kMaxSplits / kMergeGroup) + sg;
+    if (arrive(sg_counter) + 1 != (unsigned)in_sg) return;
+    if (lane == 0) *sg_counter = 0;  // as the next call expects it
+    merge_impl<D, G, F16>(ws_o, ws_ml, out, head0, sg * kMergeGroup, 1, in_sg, false, num_splits, head_dim, lane);
+    if (arrive(group_counter) + 1 != (unsigned)n_sg) return;
+    if (lane == 0) *group_counter = 0;
+    merge_impl<D, G, F16>(ws_o, ws_ml, out, head0, 0, kMergeGroup, n_sg, true, num_splits, head_dim, lane);
+}
+
 // Worker w (= warp) takes pieces w, w + workers, ...; consecutive pieces go to different SMs.
 //   S[head, key]  = Q K^T   as m16n8k16 with A = Q (rows = the G heads, padded with zero rows) and
 //                   B = K rows (the contraction runs over the head dimension in whatever order the
@@ -317,7 +384,7 @@ __device__ __noinline__ void merge_pieces(const float* __restrict__ ws_o, const 
 //   online softmax on the accumulator fragment (lane (g, c) owns head g, keys 2c, 2c+1 of each 8);
 //   O^T[dim, head] += V^T P^T  with A = pairs of V rows interleaved with byte permutes and B = the
 //                   probabilities exactly where the first MMA left them.
-// Workspace: counters[B * Hkv] (zero between calls), then ws_o[(b, head, piece)][D] and ws_ml[(b, head, piece)][2]
+// Workspace: counters[B * Hkv] and counters of the groups of sixteen pieces [B * Hkv][16] (zero between calls), then ws_o[(b, head, piece)][D] and ws_ml[(b, head, piece)][2]
 // with num_splits piece slots per (batch, head).
 template <int D, int G, bool F16>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -593,6 +660,11 @@ decode_split_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     make_float4(acc[hb][0][2 + e], acc[hb][1][2 + e], acc[hb][2][2 + e], acc[hb][3][2 + e]);
             }
         }
+        if (it.pieces > kSingleLevelPieces) {
+            arrive_two_level<D, G, F16>(counters, ws_o, ws_ml, out, B, Hkv, it.b, it.kvh, it.piece, it.pieces, head0,
+                                        num_splits, head_dim, lane);
+            continue;
+        }
         // The arrival is a release-acquire read-modify-write at device scope by lane 0, after a warp barrier:
         // the warp's stores of the partial happen before it, and whoever reads the full count has acquired the
         // partials of all earlier arrivals.  (One combined operation instead of fence, atomic, fence: the
@@ -667,12 +739,14 @@ int dispatch_g(int G, const void* q, const void* kc, const void* vc, const int32
 #undef FORGE_DECODE_CASE
 }
 
-// Bytes of the arrival counters at the start of the workspace: one per (batch, kv head), sized for Hkv = Hq.
-// At least 64 KiB, so that every shape with B * Hq <= 16384 keeps its counters (and only counters) in the
+// Bytes of the arrival counters at the start of the workspace: one per (batch, kv head) and, behind those, one
+// per group of sixteen pieces of a (batch, kv head) for the two-level merge; sized for Hkv = Hq.
+// At least 1088 KiB, so that every shape with B * Hq <= 16384 keeps its counters (and only counters) in the
 // same region: a workspace cleared once then serves calls of any such shape.
 inline size_t counter_bytes(int B, int Hq) {
-    const size_t need = ((size_t)B * Hq * sizeof(unsigned int) + 255) & ~(size_t)255;
-    return need > 65536 ? need : 65536;
+    constexpr size_t kPerHead = (1 + kMaxSplits / kMergeGroup) * sizeof(unsigned int);
+    const size_t need = ((size_t)B * Hq * kPerHead + 255) & ~(size_t)255;
+    return need > 16384 * kPerHead ? need : 16384 * kPerHead;
 }
 
 }  // namespace
@@ -704,7 +778,7 @@ int decode_splitkv_impl(const void* q, const void* k_cache, const void* v_cache,
     int st = check_attn_args(q, k_cache, v_cache, out, B, Hq, Hkv, 1, Smax, D, FORGE_MASK_PADDING, lens, /*any_head_dim=*/true);
     if (st != FORGE_OK) return st;
     if (num_splits < 1) return FORGE_ERR_INVALID_ARG;
-    if (num_splits > 64 || Hkv > 65535 || B > 65535) return FORGE_ERR_UNSUPPORTED;
+    if (num_splits > kMaxSplits || Hkv > 65535 || B > 65535) return FORGE_ERR_UNSUPPORTED;
     // the kernel counts 16-row blocks and pieces in 32 bits
     if ((long long)B * Hkv * ((Smax + kBlockKeys - 1) / kBlockKeys) >= (1LL << 31)) return FORGE_ERR_UNSUPPORTED;
     if (!workspace || !aligned16(workspace)) return FORGE_ERR_INVALID_ARG;

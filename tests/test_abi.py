@@ -44,10 +44,11 @@ def test_status_strings(lib):
 
 
 def test_workspace_size(lib):
-    # arrival counters (64 KiB, or 4 bytes per (batch, head) if that is more) + num_splits partial slots per (batch, head)
-    assert lib.forge_attn_decode_workspace_bytes(16, 32, 128, 16) == 65536 + 16 * 32 * 16 * (128 + 2) * 4
-    assert lib.forge_attn_decode_workspace_bytes(3, 8, 40, 5) == 65536 + 3 * 8 * 5 * (64 + 2) * 4
-    assert lib.forge_attn_decode_workspace_bytes(4096, 8, 64, 1) == 4096 * 8 * 4 + 4096 * 8 * (64 + 2) * 4
+    # arrival counters (1088 KiB, or 68 bytes per (batch, head) if that is more) + num_splits partial slots per (batch, head)
+    assert lib.forge_attn_decode_workspace_bytes(16, 32, 128, 16) == 17 * 65536 + 16 * 32 * 16 * (128 + 2) * 4
+    assert lib.forge_attn_decode_workspace_bytes(3, 8, 40, 5) == 17 * 65536 + 3 * 8 * 5 * (64 + 2) * 4
+    assert lib.forge_attn_decode_workspace_bytes(1024, 32, 128, 1) == 68 * 1024 * 32 + 1024 * 32 * (128 + 2) * 4
+    assert lib.forge_attn_decode_workspace_bytes(4096, 8, 64, 1) == 4096 * 8 * 68 + 4096 * 8 * (64 + 2) * 4
     assert lib.forge_attn_decode_workspace_bytes(0, 32, 128, 16) == 0
 
 
@@ -91,7 +92,7 @@ def test_decode_argument_validation(lib):
 
     assert call(lens=None) == binding.ERR_INVALID_ARG
     assert call(splits=0) == binding.ERR_INVALID_ARG
-    assert call(splits=65) == binding.ERR_UNSUPPORTED
+    assert call(splits=257) == binding.ERR_UNSUPPORTED
     assert call(ws=None) == binding.ERR_INVALID_ARG
     assert call(wsb=need - 1) == binding.ERR_WORKSPACE
     assert call(Hq=18, Hkv=2, wsb=1 << 30) == binding.ERR_UNSUPPORTED   # group size 9

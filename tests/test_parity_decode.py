@@ -121,3 +121,15 @@ def test_host_buffer_variant():
     binding.check_status()
     ref = oracle.attn_decode(w.q.values, w.k_cache.values, w.v_cache.values, w.lens, w.scale)
     assert_close_bf16(out, ref)
+
+
+@pytest.mark.parametrize("num_splits", [130, 256])
+def test_single_long_sequence_with_many_pieces(num_splits):
+    """One sequence, two kv heads: the pieces of a sequence number more than 64 (the merge keeps eight (m, l) pairs
+    per lane and head); 257 pieces are refused."""
+    w = wl.decode_workload("t", 33, 1, 8, 2, 20000, 128, num_splits, 1.0 / np.sqrt(128), (19000, 20000))
+    _run(w, num_splits)
+    with pytest.raises(binding.ForgeError) as e:
+        binding.attn_decode_splitkv(to_device(w.q), to_device(w.k_cache), to_device(w.v_cache),
+                                    torch.from_numpy(w.lens).cuda(), 257, w.scale)
+    assert e.value.status == binding.ERR_UNSUPPORTED

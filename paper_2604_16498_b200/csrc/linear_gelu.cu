@@ -402,6 +402,20 @@ int launch_linear(const void* x, const void* w, const void* b, const void* resid
 template <int ACT, bool F16>
 int launch_layout(int w_layout, const void* x, const void* w, const void* b, const void* r, void* y, int M, int N,
                   int K, cudaStream_t s) {
+    // This kernel gets the problems with a single row tile (M <= 128): they stream W once and are bound by HBM, so
+    // what counts is how many SMs pull on it.  When 192-column tiles would leave many SMs without one (and W is
+    // large enough for that to matter: small problems are bound by latency, which more and narrower tiles only
+    // add to), narrower tiles with deeper rings spread the same bytes over more of them: the widest of 192, 128
+    // and 64 columns that gives at least three quarters of the SMs a tile, else 64.
+    const int sms = sm_count();
+    const long long w_bytes = 2LL * N * K;
+    if ((N + 191) / 192 < (3 * sms) / 4 && w_bytes >= (16LL << 20)) {
+        if ((N + 127) / 128 >= (3 * sms) / 4)
+            return w_layout == FORGE_W_NK ? launch_linear<128, 5, ACT, true, false, F16>(x, w, b, r, y, M, N, K, s)
+                                          : launch_linear<128, 5, ACT, false, false, F16>(x, w, b, r, y, M, N, K, s);
+        return w_layout == FORGE_W_NK ? launch_linear<64, 8, ACT, true, false, F16>(x, w, b, r, y, M, N, K, s)
+                                      : launch_linear<64, 8, ACT, false, false, F16>(x, w, b, r, y, M, N, K, s);
+    }
     return w_layout == FORGE_W_NK ? launch_linear<192, 4, ACT, true, false, F16>(x, w, b, r, y, M, N, K, s)
                                   : launch_linear<192, 4, ACT, false, false, F16>(x, w, b, r, y, M, N, K, s);
 }

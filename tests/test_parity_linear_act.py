@@ -61,3 +61,17 @@ def test_argument_validation():
     with pytest.raises(binding.ForgeError) as e:
         binding.linear_act(x, ww, None, None, 7)
     assert e.value.status == binding.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("shape", [(16, 4104, 2112), (100, 14344, 640)])
+@pytest.mark.parametrize("w_layout", [binding.W_KN, binding.W_NK])
+def test_single_row_tile_with_a_large_weight(shape, w_layout):
+    """M <= 128 and a weight of 17-18 MB: the narrow tiles (64 and 128 columns) that spread the weight stream over
+    more SMs; the last column tile is ragged."""
+    M, N, K = shape
+    w, r = _case(M, N, K, seed=55)
+    wdev = to_device(w.w) if w_layout == binding.W_KN else to_device(w.w).t().contiguous()
+    wref = w.w.values if w_layout == binding.W_KN else np.ascontiguousarray(w.w.values.T)
+    y = binding.linear_act(to_device(w.x), wdev, to_device(w.b), to_device(r), binding.ACT_GELU_TANH, w_layout)
+    binding.check_status()
+    assert_close_bf16(y, oracle.linear_act(w.x.values, wref, w.b.values, r.values, oracle.ACT_GELU_TANH, w_layout))

@@ -412,7 +412,12 @@ def run_gpu(args):
     barrier()
     clocks = sampler.stop()
     binding.check_status()
-    in_step_ms = [float(np.median([e[i].elapsed_time(e[i + 1]) for e in evs])) for i in range(len(KERNELS))]
+    per_call = [np.array([e[i].elapsed_time(e[i + 1]) for e in evs]) for i in range(len(KERNELS))]
+    in_step_ms = [float(np.median(pc)) for pc in per_call]
+    # the same samples as a distribution (one call each, events on both sides: launch gaps included)
+    in_step_dist = [{"mean": float(pc.mean() * 1e3), "p50": float(np.percentile(pc, 50) * 1e3),
+                     "p90": float(np.percentile(pc, 90) * 1e3), "p99": float(np.percentile(pc, 99) * 1e3),
+                     "best": float(pc.min() * 1e3), "calls": int(pc.size)} for pc in per_call]
 
     st = stats(step_ms, args.steps)
     ms_per_step = st["median"]
@@ -426,6 +431,7 @@ def run_gpu(args):
         w = work[name]
         ms = ks["median"]
         k = {"ms": ms, "ms_min": ks["min"], "ms_max": ks["max"], "ms_in_step": in_step_ms[i],
+             "in_step_us": in_step_dist[i],
              "tflops": w.flops() / ms / 1e9, "gbs": w.bytes() / ms / 1e6, "bound": bound[name],
              "flops": w.flops(), "bytes": w.bytes()}
         if bound[name] == "tensor":

@@ -18,7 +18,7 @@ from . import binding
 
 def main() -> None:
     ap = argparse.ArgumentParser()
-    ap.add_argument("op", choices=["attention", "attention_f32", "linear", "decode"])
+    ap.add_argument("op", choices=["attention", "attention_f32", "linear", "linear_w8", "decode"])
     ap.add_argument("--B", type=int, default=8)
     ap.add_argument("--Hq", type=int, default=12)
     ap.add_argument("--Hkv", type=int, default=12)
@@ -58,6 +58,12 @@ def main() -> None:
         x, w, b = randn((a.M, a.K)), randn((a.K, a.N), std=0.02), randn((a.N,), std=0.02)
         y = torch.empty((a.M, a.N), dtype=torch.bfloat16, device=dev)
         call = lambda: binding.linear_bias_gelu(x, w, b, out=y)
+    elif a.op == "linear_w8":
+        x = randn((a.M, a.K), torch.float16)
+        wq = torch.randint(-127, 128, (a.N, a.K), generator=g, device=dev, dtype=torch.int8)
+        sc = torch.rand((a.N,), generator=g, device=dev) * 0.01
+        y = torch.empty((a.M, a.N), dtype=torch.float16, device=dev)
+        call = lambda: binding.linear_act_w8a16(x, wq, sc, None, None, binding.ACT_GELU_TANH, out=y)
     else:
         q = randn((a.B, a.Hq, a.D))
         kc = randn((a.B, a.Hkv, a.S, a.D))
